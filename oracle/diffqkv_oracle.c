@@ -1,0 +1,300 @@
+/*
+ * DiffQKV attention oracle: plain, slow, float64 CPU code.
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It exists so that the CUDA
+ * library can be checked element by element against the plain definition of
+ * what the paper's method computes.  It shares no code, header, table or
+ * helper with the CUDA path and must never be called from it; only the test
+ * suite, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * What it follows (paper sections, equations, listings):
+ *   - Section 2, "Formulation of DiffQKV Attention": q, K, V with separate
+ *     head counts n_q, n_k, n_v; scores = softmax over cached positions of
+ *     <q_i, K_(j,i)> / sqrt(d_k); o_i = sum_j alpha_(j,i) V_(j,i).
+ *   - Section 3.2, Eq. (idx): idx_k = idx_q * n_k / n_q, idx_v = idx_q * n_v / n_q
+ *     (read as integer floor; n_k and n_v must divide n_q).
+ *   - Appendix "KV Group Sharing" listing: replicated heads are adjacent,
+ *     which is the same contiguous grouping as the floor in Eq. (idx).
+ *   - Section 3.2: the split kernel produces per-chunk outputs and the combine
+ *     kernel assembles them; oracle_combine is the log-sum-exp merge that makes
+ *     "assemble" exact.
+ *   - Appendix attention listing: augmented Q = W_down(act(W_gate x) * (W_up x))
+ *     with x = h W_Q; the activation is read as SiLU (the model's own MLP is
+ *     SwiGLU), no biases.
+ *
+ * Everything is computed in double from the stored (bf16 or fp32) values, which
+ * convert to double exactly.  Loops are the definition written out: no
+ * blocking, no online softmax, no fusion.  OpenMP is used only to spread
+ * independent (sequence, head) or row work over host cores.
+ *
+ * Pins (tests/test_oracle_pins.py): textbook multi-head attention when
+ * n_q = n_k = n_v (library softmax/matmul), K-replication identity from the
+ * paper's group-sharing listing, identical keys give the mean of V, a dominant
+ * key returns its V row within (len-1)e^-gap, a pure-Python brute force on tiny
+ * shapes, split/combine invariance, page-table invariance, prefill row i equals
+ * decode at length i+1, and hand-worked tiny cases for the augmented Q.
+ * The choice of SiLU as act_fn is a reading of the paper, not pinned by it:
+ * for oracle_augq the activation choice is "parity unpinned" (the rest of the
+ * chain is pinned by closed forms).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORACLE_BF16 = 0, ORACLE_F32 = 1 };
+
+/* Exact widening of a stored element to double. */
+static double load_elt(const void *base, int64_t idx, int dtype) {
+  if (dtype == ORACLE_F32) {
+    return (double)((const float *)base)[idx];
+  } else {
+    uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return (double)f;
+  }
+}
+
+typedef struct {
+  const void *k_cache, *v_cache;
+  int64_t k_stride_blk, k_stride_head, k_stride_tok; /* in elements */
+  int64_t v_stride_blk, v_stride_head, v_stride_tok;
+  const int32_t *seqlens;    /* [batch] */
+  const int32_t *page_table; /* [batch, max_pages_per_seq] or NULL */
+  int32_t page_size, max_pages_per_seq;
+} oracle_cache;
+
+/* Element offset of (sequence b, token j, head, channel 0) in a cache pool.
+ * Contiguous cache: blk = b, slot = j.  Paged cache: blk = page_table[b][j / page_size],
+ * slot = j % page_size.  (The paper defines no page format; this is the
+ * library's own layout rule restated.) */
+static int64_t cache_row(const oracle_cache *c, int is_v, int b, int64_t j, int head) {
+  int64_t blk = b, slot = j;
+  if (c->page_table) {
+    blk = c->page_table[(int64_t)b * c->max_pages_per_seq + j / c->page_size];
+    slot = j % c->page_size;
+  }
+  if (is_v) return blk * c->v_stride_blk + (int64_t)head * c->v_stride_head + slot * c->v_stride_tok;
+  return blk * c->k_stride_blk + (int64_t)head * c->k_stride_head + slot * c->k_stride_tok;
+}
+
+int oracle_set_threads(int n) {
+#ifdef _OPENMP
+  if (n > 0) omp_set_num_threads(n);
+  return omp_get_max_threads();
+#else
+  (void)n;
+  return 1;
+#endif
+}
+
+/* Attention of one query vector q[d_qk] (already double) over tokens [t0, t1) of
+ * sequence b, K head hk, V head hv.  Writes the normalised output o[d_v] and
+ * lse = m + log(l).  Empty range: o = 0, lse = -inf. */
+static void attend_range(const double *q, const oracle_cache *c, int dtype, int b, int hk, int hv,
+                         int64_t t0, int64_t t1, int d_qk, int d_v, double scale,
+                         double *o, double *lse_out) {
+  for (int ch = 0; ch < d_v; ++ch) o[ch] = 0.0;
+  if (t1 <= t0) { *lse_out = -INFINITY; return; }
+  int64_t n = t1 - t0;
+  double *s = (double *)malloc(sizeof(double) * (size_t)n);
+  double m = -INFINITY;
+  for (int64_t j = t0; j < t1; ++j) {
+    int64_t row = cache_row(c, 0, b, j, hk);
+    double acc = 0.0;
+    for (int ch = 0; ch < d_qk; ++ch) acc += q[ch] * load_elt(c->k_cache, row + ch, dtype);
+    acc *= scale;
+    s[j - t0] = acc;
+    if (acc > m) m = acc;
+  }
+  double l = 0.0;
+  for (int64_t i = 0; i < n; ++i) { s[i] = exp(s[i] - m); l += s[i]; }
+  for (int64_t j = t0; j < t1; ++j) {
+    int64_t row = cache_row(c, 1, b, j, hv);
+    double p = s[j - t0];
+    for (int ch = 0; ch < d_v; ++ch) o[ch] += p * load_elt(c->v_cache, row + ch, dtype);
+  }
+  for (int ch = 0; ch < d_v; ++ch) o[ch] /= l;
+  *lse_out = m + log(l);
+  free(s);
+}
+
+/* Decode: one query token per sequence.
+ *   q   [batch, n_q, d_qk] storage dtype, contiguous
+ *   out [batch, n_q, d_v] double; lse [batch, n_q] double
+ *   pairs: optional list of (b, h) pairs (n_pairs of them); when given only those
+ *          rows of out / lse are computed (the others are left untouched).
+ * Returns 0, or -1 when n_k or n_v does not divide n_q. */
+int oracle_decode(const void *q, const oracle_cache *c, int batch, int n_q, int n_k, int n_v,
+                  int d_qk, int d_v, int dtype, double scale, const int32_t *pairs, int n_pairs,
+                  double *out, double *lse) {
+  if (n_k <= 0 || n_v <= 0 || n_q % n_k || n_q % n_v) return -1;
+  int64_t total = pairs ? n_pairs : (int64_t)batch * n_q;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t w = 0; w < total; ++w) {
+    int b = pairs ? pairs[2 * w] : (int)(w / n_q);
+    int h = pairs ? pairs[2 * w + 1] : (int)(w % n_q);
+    int hk = (int)(((int64_t)h * n_k) / n_q); /* Eq. (idx), floor */
+    int hv = (int)(((int64_t)h * n_v) / n_q);
+    double *qd = (double *)malloc(sizeof(double) * (size_t)d_qk);
+    for (int ch = 0; ch < d_qk; ++ch) qd[ch] = load_elt(q, ((int64_t)b * n_q + h) * d_qk + ch, dtype);
+    attend_range(qd, c, dtype, b, hk, hv, 0, c->seqlens[b], d_qk, d_v, scale,
+                 out + ((int64_t)b * n_q + h) * d_v, lse + (int64_t)b * n_q + h);
+    free(qd);
+  }
+  return 0;
+}
+
+/* Decode restricted to an explicit token range per split: cuts [n_splits + 1]
+ * ascending token positions shared by all sequences (clamped to each length).
+ * o_partial [batch, n_q, n_splits, d_v], lse_partial [batch, n_q, n_splits]:
+ * per-split normalised outputs and log-sum-exps, the objects the combine step merges. */
+int oracle_decode_splits(const void *q, const oracle_cache *c, int batch, int n_q, int n_k, int n_v,
+                         int d_qk, int d_v, int dtype, double scale, const int64_t *cuts, int n_splits,
+                         double *o_partial, double *lse_partial) {
+  if (n_k <= 0 || n_v <= 0 || n_q % n_k || n_q % n_v) return -1;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t w = 0; w < (int64_t)batch * n_q; ++w) {
+    int b = (int)(w / n_q), h = (int)(w % n_q);
+    int hk = (int)(((int64_t)h * n_k) / n_q);
+    int hv = (int)(((int64_t)h * n_v) / n_q);
+    double *qd = (double *)malloc(sizeof(double) * (size_t)d_qk);
+    for (int ch = 0; ch < d_qk; ++ch) qd[ch] = load_elt(q, w * d_qk + ch, dtype);
+    int64_t len = c->seqlens[b];
+    for (int s = 0; s < n_splits; ++s) {
+      int64_t t0 = cuts[s] < len ? cuts[s] : len;
+      int64_t t1 = cuts[s + 1] < len ? cuts[s + 1] : len;
+      attend_range(qd, c, dtype, b, hk, hv, t0, t1, d_qk, d_v, scale,
+                   o_partial + (w * n_splits + s) * d_v, lse_partial + w * n_splits + s);
+    }
+    free(qd);
+  }
+  return 0;
+}
+
+/* Combine (Section 3.2, "combine kernel"): merge per-split normalised outputs.
+ *   lse = log sum_s exp(lse_s) over splits with lse_s > -inf,
+ *   out = sum_s exp(lse_s - lse) o_s.   All splits empty: out = 0, lse = -inf. */
+void oracle_combine(const double *o_partial, const double *lse_partial, int64_t rows /* batch*n_q */,
+                    int n_splits, int d_v, double *out, double *lse) {
+  for (int64_t r = 0; r < rows; ++r) {
+    double m = -INFINITY;
+    for (int s = 0; s < n_splits; ++s)
+      if (lse_partial[r * n_splits + s] > m) m = lse_partial[r * n_splits + s];
+    for (int ch = 0; ch < d_v; ++ch) out[r * d_v + ch] = 0.0;
+    if (m == -INFINITY) { lse[r] = -INFINITY; continue; }
+    double sum = 0.0;
+    for (int s = 0; s < n_splits; ++s) {
+      double ls = lse_partial[r * n_splits + s];
+      if (ls == -INFINITY) continue;
+      sum += exp(ls - m);
+    }
+    double total = m + log(sum);
+    for (int s = 0; s < n_splits; ++s) {
+      double ls = lse_partial[r * n_splits + s];
+      if (ls == -INFINITY) continue;
+      double w = exp(ls - total);
+      for (int ch = 0; ch < d_v; ++ch) out[r * d_v + ch] += w * o_partial[(r * n_splits + s) * d_v + ch];
+    }
+    lse[r] = total;
+  }
+}
+
+/* Cache append done by prefill (attention listing: past_key_value.update):
+ * copy rows k_new [batch, q_len, n_k, d_qk], v_new [batch, q_len, n_v, d_v] into the
+ * cache at token positions past_b + i, past_b = seqlens[b] on entry.  Pure byte
+ * movement; the cache pointers are written through a non-const alias. */
+void oracle_cache_append(const void *k_new, const void *v_new, int q_len, const oracle_cache *c,
+                         int batch, int n_k, int n_v, int d_qk, int d_v, int dtype) {
+  size_t es = dtype == ORACLE_F32 ? 4 : 2;
+  for (int b = 0; b < batch; ++b)
+    for (int i = 0; i < q_len; ++i) {
+      int64_t j = (int64_t)c->seqlens[b] + i;
+      for (int h = 0; h < n_k; ++h)
+        memcpy((char *)(uintptr_t)c->k_cache + es * (size_t)cache_row(c, 0, b, j, h),
+               (const char *)k_new + es * (size_t)((((int64_t)b * q_len + i) * n_k + h) * d_qk), es * d_qk);
+      for (int h = 0; h < n_v; ++h)
+        memcpy((char *)(uintptr_t)c->v_cache + es * (size_t)cache_row(c, 1, b, j, h),
+               (const char *)v_new + es * (size_t)((((int64_t)b * q_len + i) * n_v + h) * d_v), es * d_v);
+    }
+}
+
+/* Causal prefill attention over a cache that already holds the new rows.
+ *   q [batch, q_len, n_q, d_qk]; query row i of sequence b sits at absolute position
+ *   past_b + i and sees tokens 0 .. past_b + i (bottom-right aligned causal mask);
+ *   past [batch] = number of tokens that were cached before this call.
+ *   rows: optional list of (b, i, h) triples (n_rows of them); out is then
+ *   [n_rows, d_v] and lse [n_rows] in list order.  Without a list out is
+ *   [batch, q_len, n_q, d_v] and lse [batch, q_len, n_q]. */
+int oracle_prefill(const void *q, int q_len, const int32_t *past, const oracle_cache *c, int batch,
+                   int n_q, int n_k, int n_v, int d_qk, int d_v, int dtype, double scale,
+                   const int32_t *rows, int64_t n_rows, double *out, double *lse) {
+  if (n_k <= 0 || n_v <= 0 || n_q % n_k || n_q % n_v) return -1;
+  int64_t total = rows ? n_rows : (int64_t)batch * q_len * n_q;
+#pragma omp parallel for schedule(dynamic, 4)
+  for (int64_t w = 0; w < total; ++w) {
+    int b, i, h;
+    if (rows) { b = rows[3 * w]; i = rows[3 * w + 1]; h = rows[3 * w + 2]; }
+    else { b = (int)(w / ((int64_t)q_len * n_q)); i = (int)((w / n_q) % q_len); h = (int)(w % n_q); }
+    int hk = (int)(((int64_t)h * n_k) / n_q);
+    int hv = (int)(((int64_t)h * n_v) / n_q);
+    double *qd = (double *)malloc(sizeof(double) * (size_t)d_qk);
+    int64_t qrow = (((int64_t)b * q_len + i) * n_q + h) * d_qk;
+    for (int ch = 0; ch < d_qk; ++ch) qd[ch] = load_elt(q, qrow + ch, dtype);
+    attend_range(qd, c, dtype, b, hk, hv, 0, (int64_t)past[b] + i + 1, d_qk, d_v, scale,
+                 out + w * d_v, lse + w);
+    free(qd);
+  }
+  return 0;
+}
+
+/* Augmented Q (attention listing: q_proj, then q_down_proj(act(q_gate_proj(x)) * q_up_proj(x))).
+ * Weights use the nn.Linear layout [out_features, in_features], y = x W^T, no bias:
+ *   W_Q [d_q0, d_model], W_gate, W_up [d_aug, d_q0], W_down [d_out, d_aug].
+ *   h [T, d_model].  rows: optional list of n_rows token indices; q_out is
+ *   [n_rows or T, d_out] double.  No intermediate rounding. */
+void oracle_augq(const void *h, const void *W_Q, const void *W_gate, const void *W_up, const void *W_down,
+                 int64_t T, int d_model, int d_q0, int d_aug, int d_out, int dtype,
+                 const int64_t *rows, int64_t n_rows, double *q_out) {
+  int64_t total = rows ? n_rows : T;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t w = 0; w < total; ++w) {
+    int64_t t = rows ? rows[w] : w;
+    double *x = (double *)malloc(sizeof(double) * (size_t)d_q0);
+    double *a = (double *)malloc(sizeof(double) * (size_t)d_aug);
+    for (int o = 0; o < d_q0; ++o) {
+      double acc = 0.0;
+      for (int i = 0; i < d_model; ++i)
+        acc += load_elt(h, t * d_model + i, dtype) * load_elt(W_Q, (int64_t)o * d_model + i, dtype);
+      x[o] = acc;
+    }
+    for (int o = 0; o < d_aug; ++o) {
+      double g = 0.0, u = 0.0;
+      for (int i = 0; i < d_q0; ++i) {
+        g += x[i] * load_elt(W_gate, (int64_t)o * d_q0 + i, dtype);
+        u += x[i] * load_elt(W_up, (int64_t)o * d_q0 + i, dtype);
+      }
+      double silu = g / (1.0 + exp(-g));
+      a[o] = silu * u;
+    }
+    for (int o = 0; o < d_out; ++o) {
+      double acc = 0.0;
+      for (int i = 0; i < d_aug; ++i) acc += a[i] * load_elt(W_down, (int64_t)o * d_aug + i, dtype);
+      q_out[w * d_out + o] = acc;
+    }
+    free(x);
+    free(a);
+  }
+}
+
+/* KV-cache cost model, Eq. (cache_0) with alpha = element size, beta = 0:
+ * bytes moved to stream the cache once for the given lengths. */
+double oracle_kv_bytes(const int32_t *seqlens, int batch, int n_k, int n_v, int d_qk, int d_v, int elt_bytes) {
+  double tokens = 0.0;
+  for (int b = 0; b < batch; ++b) tokens += seqlens[b];
+  return tokens * ((double)n_k * d_qk + (double)n_v * d_v) * elt_bytes;
+}
