@@ -1,0 +1,178 @@
+/*
+ * diffqkv.h -- C ABI of libdiffqkv: DiffQKV attention over a KV cache on NVIDIA B200 (sm_100a).
+ *
+ * DiffQKV attention (paper Section 2, "Formulation of DiffQKV Attention") is softmax
+ * attention in which Q, K and V have their own head counts n_q, n_k, n_v.  Query head h
+ * reads K head  hk = floor(h * n_k / n_q)  and V head  hv = floor(h * n_v / n_q)
+ * (Section 3.2, Eq. (idx); n_k and n_v must divide n_q, so hk = h / (n_q/n_k)).  For one
+ * query vector q_h and the visible cached tokens j:
+ *
+ *     s_j = scale * <q_h, K[j, hk]>          m = max_j s_j
+ *     p_j = exp(s_j - m)                     l = sum_j p_j
+ *     out_h = (sum_j p_j * V[j, hv]) / l     lse_h = m + log(l)
+ *
+ * K and V live in two separate pools (Section 3.1: the key cache and the value cache have
+ * different shapes), streamed once per call; that traffic, b*s*(n_k*d_k + n_v*d_v) elements
+ * (Eq. (cache_0)), is what bounds decoding.
+ *
+ * General rules for every call
+ *   - Every pointer in the argument lists and structs is a DEVICE pointer unless it is marked
+ *     "host".  The structs themselves (diffqkv_cache, diffqkv_shape) are read on the host.
+ *   - The library borrows all buffers, owns nothing and, unless an entry point says otherwise,
+ *     allocates nothing: scratch memory is a caller-provided workspace.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return without
+ *     synchronising.  Buffers must stay valid until the stream has run the work.
+ *   - Errors the host can see (null pointers, head counts that do not divide, unsupported head
+ *     dimensions, misaligned pointers, a workspace that is too small, a failed launch) return a
+ *     status and launch nothing.  Conditions only the device can see (a page id outside the
+ *     pool, a bounded wait that ran out) OR the bit (1 << diffqkv_status value) into *dev_status
+ *     (when given) and the affected block skips that work; nothing traps.
+ *   - Tensors are dense in their last (channel) dimension.  bf16 tensors must be 16-byte
+ *     aligned with strides that are multiples of 8 elements; fp32 tensors 16-byte aligned with
+ *     strides that are multiples of 4 elements.
+ */
+#ifndef DIFFQKV_H_
+#define DIFFQKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DIFFQKV_OK = 0,
+  DIFFQKV_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, n_k or n_v not dividing n_q ... */
+  DIFFQKV_ERR_UNSUPPORTED = 2, /* a shape or dtype no kernel covers                                */
+  DIFFQKV_ERR_ALIGNMENT = 3,   /* a pointer or stride violates the alignment rules above           */
+  DIFFQKV_ERR_WORKSPACE = 4,   /* workspace missing or smaller than the *_workspace_bytes answer   */
+  DIFFQKV_ERR_CUDA = 5,        /* a CUDA runtime or driver call failed                             */
+  DIFFQKV_ERR_TIMEOUT = 6,     /* device: a bounded wait on a copy ran out                         */
+  DIFFQKV_ERR_INDEX = 7        /* device: page id outside [0, num_blocks)                          */
+} diffqkv_status;
+
+typedef enum { DIFFQKV_BF16 = 0, DIFFQKV_F32 = 1 } diffqkv_dtype;
+
+/*
+ * The KV cache: two pools addressed through the same rule.  Token j of sequence b, head hd,
+ * channel c of the K pool sits at element offset
+ *     blk * k_stride_blk + hd * k_stride_head + slot * k_stride_tok + c
+ * with (blk, slot) = (b, j) for a contiguous cache (page_table == NULL) and
+ * (blk, slot) = (page_table[b * max_pages_per_seq + j / page_size], j % page_size) for a paged
+ * one; likewise for V.  One page table serves both pools.  The paper fixes only the logical
+ * shapes (b, s, n_h, d_h) (Section 3.1); strides make head-major and token-major storage
+ * both expressible, and the page format is this library's own.
+ */
+typedef struct {
+  void *k_cache;             /* K pool, element type = shape.dtype                                  */
+  void *v_cache;             /* V pool                                                              */
+  int64_t k_stride_blk, k_stride_head, k_stride_tok; /* in elements                                 */
+  int64_t v_stride_blk, v_stride_head, v_stride_tok;
+  const int32_t *seqlens;    /* [batch] visible tokens per sequence (decode: includes the new one)  */
+  const int32_t *page_table; /* [batch, max_pages_per_seq] physical page ids, or NULL = contiguous  */
+  int32_t page_size;         /* tokens per page (paged only; a multiple of 16 for the TMA kernels)  */
+  int32_t max_pages_per_seq; /* row length of page_table                                            */
+  int32_t num_blocks;        /* extent of the blk dimension: pages in the pool, or batch            */
+  int32_t max_seqlen;        /* host-known upper bound of seqlens[]; contiguous: also the token     */
+                             /* extent of each (blk, head) slab, so reads never pass it             */
+} diffqkv_cache;
+
+typedef struct {
+  int32_t batch, n_q, n_k, n_v; /* n_q % n_k == 0 and n_q % n_v == 0                                */
+  int32_t d_qk, d_v;            /* channels per head of Q/K and of V                                */
+  diffqkv_dtype dtype;          /* storage type of q, K and V; accumulation is always fp32          */
+  diffqkv_dtype out_dtype;      /* storage type of `out`                                            */
+  float scale;                  /* multiplies the inner product; the paper uses 1/sqrt(d_k)         */
+} diffqkv_shape;
+
+/*
+ * Split planning for decode (Section 3.2: the split kernel divides K and V into chunks along
+ * the sequence).  The sequence axis is cut into chunks of one fixed length; sequence b uses
+ * ceil(seqlens[b] / chunk) of the at most S splits.
+ *   diffqkv_decode_num_splits: S the library would choose for num_splits = 0 (always >= 1).
+ *   diffqkv_decode_workspace_bytes: bytes of workspace diffqkv_decode / gqa_decode need for
+ *   this shape, max_seqlen and num_splits (0 = the automatic choice).  Returns 0 on bad input.
+ */
+int32_t diffqkv_decode_num_splits(const diffqkv_shape *shape, int32_t max_seqlen);
+size_t diffqkv_decode_workspace_bytes(const diffqkv_shape *shape, int32_t max_seqlen, int32_t num_splits);
+
+/*
+ * diffqkv_decode -- one query token per sequence against the cache (Section 2 formulation with
+ * the head map of Eq. (idx); split-sequence execution per Section 3.2).
+ *   q          [batch, n_q, d_qk]  shape.dtype, contiguous
+ *   cache      see diffqkv_cache; seqlens[b] == 0 gives out = 0 and lse = -inf for that sequence
+ *   num_splits maximum splits per sequence, 0 = automatic
+ *   workspace  at least diffqkv_decode_workspace_bytes(...) bytes, 256-byte aligned; holds the
+ *              per-split partial outputs (fp32 [batch, n_q, S, d_v]) and log-sum-exps
+ *              (fp32 [batch, n_q, S]); contents on entry are ignored
+ *   out        [batch, n_q, d_v]   shape.out_dtype
+ *   lse        [batch, n_q] fp32 natural-log log-sum-exp of the scaled scores, or NULL
+ *   dev_status one int32 the kernels OR (1 << diffqkv_status) bits into, or NULL; the caller zeroes it
+ * Runs the split kernel and then the combine kernel on `stream`.
+ */
+diffqkv_status diffqkv_decode(const void *q, const diffqkv_cache *cache, const diffqkv_shape *shape,
+                              int32_t num_splits, void *workspace, size_t workspace_bytes, void *out,
+                              float *lse, int32_t *dev_status, void *stream);
+
+/*
+ * gqa_decode -- grouped-query attention, the comparison point of the paper (Appendix B.1: GQA is
+ * the special case n_k == n_v).  Same arguments and the same kernels as diffqkv_decode; returns
+ * DIFFQKV_ERR_INVALID_ARG when shape.n_k != shape.n_v.
+ */
+diffqkv_status gqa_decode(const void *q, const diffqkv_cache *cache, const diffqkv_shape *shape,
+                          int32_t num_splits, void *workspace, size_t workspace_bytes, void *out,
+                          float *lse, int32_t *dev_status, void *stream);
+
+/*
+ * diffqkv_combine -- merge per-split partial results (Section 3.2: the combine kernel assembles
+ * the output chunks).  With o_s the NORMALISED output of split s and lse_s its log-sum-exp:
+ *     lse = log sum_s exp(lse_s),   out = sum_s exp(lse_s - lse) * o_s,
+ * splits with lse_s == -inf are skipped; if all are, out = 0 and lse = -inf.
+ *   o_partial   [rows, S, d_v] fp32     lse_partial [rows, S] fp32     (rows = batch * n_q)
+ *   out         [rows, d_v] out_dtype   lse [rows] fp32 or NULL
+ */
+diffqkv_status diffqkv_combine(const float *o_partial, const float *lse_partial, int32_t batch, int32_t n_q,
+                               int32_t d_v, int32_t num_splits, diffqkv_dtype out_dtype, void *out,
+                               float *lse, void *stream);
+
+/*
+ * diffqkv_prefill -- causal attention for q_len new tokens per sequence, writing their K and V
+ * rows into the cache first (appendix attention listing: cache update, then the causal
+ * flash-attention call; head map of Eq. (idx)).
+ *   q      [batch, q_len, n_q, d_qk]   k_new [batch, q_len, n_k, d_qk]   v_new [batch, q_len, n_v, d_v]
+ *   cache  seqlens[b] = tokens already cached (past_b) on entry; rows past_b .. past_b + q_len - 1 of
+ *          both pools are overwritten; seqlens itself is not modified (the caller adds q_len)
+ *   out    [batch, q_len, n_q, d_v] out_dtype; query row i sees tokens 0 .. past_b + i
+ *   lse    [batch, q_len, n_q] fp32 or NULL
+ * Requires bf16, d_qk == d_v == 128 (tensor-core tiles).
+ */
+diffqkv_status diffqkv_prefill(const void *q, const void *k_new, const void *v_new, int32_t q_len,
+                               const diffqkv_cache *cache, const diffqkv_shape *shape, void *out, float *lse,
+                               int32_t *dev_status, void *stream);
+
+/*
+ * diffqkv_augq -- the augmented-Q projection that produces the queries (Section 2, Observation 3;
+ * appendix attention listing: q_proj followed by q_down_proj(act(q_gate_proj(x)) * q_up_proj(x))).
+ * act is read as SiLU, there are no biases, and weights use the nn.Linear layout [out, in]:
+ *     x = h W_Q^T,   a = silu(x W_gate^T) * (x W_up^T),   q = a W_down^T
+ *   h [T, d_model]   W_Q [d_q0, d_model]   W_gate, W_up [d_aug, d_q0]   W_down [d_out, d_aug]   all bf16
+ *   workspace  diffqkv_augq_workspace_bytes(T, d_q0, d_aug) bytes for x and a (bf16)
+ *   q_out [T, d_out] bf16
+ * All dimensions must be multiples of 128 except T.
+ */
+size_t diffqkv_augq_workspace_bytes(int64_t T, int32_t d_q0, int32_t d_aug);
+diffqkv_status diffqkv_augq(const void *h, const void *W_Q, const void *W_gate, const void *W_up,
+                            const void *W_down, int64_t T, int32_t d_model, int32_t d_q0, int32_t d_aug,
+                            int32_t d_out, void *workspace, size_t workspace_bytes, void *q_out, void *stream);
+
+/* Static, never-null description of a status value. */
+const char *diffqkv_status_string(diffqkv_status status);
+
+/* Kernels launched by this library since it was loaded (host counter, for benchmarks). */
+int64_t diffqkv_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DIFFQKV_H_ */

@@ -1,0 +1,246 @@
+"""ctypes binding of ``libdiffqkv.so``: same entry-point names as ``include/diffqkv.h``.
+
+Argument marshalling only.  Every step of the attention path runs in the library's CUDA
+kernels; torch is used for device memory, streams and host<->device copies.  Importing this
+module loads the library and raises if it has not been built -- there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdiffqkv.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2501_13629_b200.build` "
+        "(there is no CPU or PyTorch fallback)")
+_lib = C.CDLL(LIB_PATH)
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_INDEX = range(8)
+BF16, F32 = 0, 1
+
+EXPORTS = (
+    "diffqkv_decode_num_splits", "diffqkv_decode_workspace_bytes", "diffqkv_decode", "gqa_decode",
+    "diffqkv_combine", "diffqkv_prefill", "diffqkv_augq_workspace_bytes", "diffqkv_augq",
+    "diffqkv_status_string", "diffqkv_launch_count",
+)
+
+
+class CacheStruct(C.Structure):
+    _fields_ = [
+        ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+        ("k_stride_blk", C.c_int64), ("k_stride_head", C.c_int64), ("k_stride_tok", C.c_int64),
+        ("v_stride_blk", C.c_int64), ("v_stride_head", C.c_int64), ("v_stride_tok", C.c_int64),
+        ("seqlens", C.c_void_p), ("page_table", C.c_void_p),
+        ("page_size", C.c_int32), ("max_pages_per_seq", C.c_int32),
+        ("num_blocks", C.c_int32), ("max_seqlen", C.c_int32),
+    ]
+
+
+class ShapeStruct(C.Structure):
+    _fields_ = [
+        ("batch", C.c_int32), ("n_q", C.c_int32), ("n_k", C.c_int32), ("n_v", C.c_int32),
+        ("d_qk", C.c_int32), ("d_v", C.c_int32),
+        ("dtype", C.c_int), ("out_dtype", C.c_int), ("scale", C.c_float),
+    ]
+
+
+_lib.diffqkv_decode_num_splits.restype = C.c_int32
+_lib.diffqkv_decode_num_splits.argtypes = [C.POINTER(ShapeStruct), C.c_int32]
+_lib.diffqkv_decode_workspace_bytes.restype = C.c_size_t
+_lib.diffqkv_decode_workspace_bytes.argtypes = [C.POINTER(ShapeStruct), C.c_int32, C.c_int32]
+_DECODE_ARGS = [C.c_void_p, C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_int32, C.c_void_p, C.c_size_t,
+                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+for _name in ("diffqkv_decode", "gqa_decode"):
+    getattr(_lib, _name).restype = C.c_int
+    getattr(_lib, _name).argtypes = _DECODE_ARGS
+_lib.diffqkv_combine.restype = C.c_int
+_lib.diffqkv_combine.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int,
+                                 C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.diffqkv_prefill.restype = C.c_int
+_lib.diffqkv_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(CacheStruct),
+                                 C.POINTER(ShapeStruct), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.diffqkv_augq_workspace_bytes.restype = C.c_size_t
+_lib.diffqkv_augq_workspace_bytes.argtypes = [C.c_int64, C.c_int32, C.c_int32]
+_lib.diffqkv_augq.restype = C.c_int
+_lib.diffqkv_augq.argtypes = [C.c_void_p] * 5 + [C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                                 C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+_lib.diffqkv_status_string.restype = C.c_char_p
+_lib.diffqkv_status_string.argtypes = [C.c_int]
+_lib.diffqkv_launch_count.restype = C.c_int64
+
+
+class DiffQKVError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def status_string(status: int) -> str:
+    return _lib.diffqkv_status_string(int(status)).decode()
+
+
+def launch_count() -> int:
+    return int(_lib.diffqkv_launch_count())
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.bfloat16:
+        return BF16
+    if dt == torch.float32:
+        return F32
+    raise TypeError(f"unsupported dtype {dt}")
+
+
+def _p(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+@dataclass
+class KVCache:
+    """Device-side cache description (see ``diffqkv_cache`` in the header).
+
+    ``k`` / ``v`` are the pools: contiguous ``[batch, heads, max_seqlen, d]`` or paged
+    ``[pages, heads, page_size, d]`` by default; any other layout by passing explicit
+    (blk, head, tok) element strides.
+    """
+    k: torch.Tensor
+    v: torch.Tensor
+    seqlens: torch.Tensor                      # int32 [batch], device
+    max_seqlen: int
+    page_table: Optional[torch.Tensor] = None  # int32 [batch, max_pages_per_seq], device
+    page_size: int = 0
+    k_strides: Optional[Tuple[int, int, int]] = None
+    v_strides: Optional[Tuple[int, int, int]] = None
+    num_blocks: Optional[int] = None
+
+    def c_struct(self) -> CacheStruct:
+        ks = self.k_strides or (self.k.stride(0), self.k.stride(1), self.k.stride(2))
+        vs = self.v_strides or (self.v.stride(0), self.v.stride(1), self.v.stride(2))
+        assert self.seqlens.dtype == torch.int32 and self.seqlens.is_contiguous()
+        pt = self.page_table
+        if pt is not None:
+            assert pt.dtype == torch.int32 and pt.is_contiguous() and pt.dim() == 2
+        nb = self.num_blocks if self.num_blocks is not None else self.k.shape[0]
+        return CacheStruct(
+            self.k.data_ptr(), self.v.data_ptr(), *map(int, ks), *map(int, vs),
+            self.seqlens.data_ptr(), None if pt is None else pt.data_ptr(),
+            int(self.page_size), 0 if pt is None else int(pt.shape[1]), int(nb), int(self.max_seqlen))
+
+
+def make_shape(batch, n_q, n_k, n_v, d_qk, d_v, dtype: torch.dtype, out_dtype: torch.dtype, scale: float):
+    return ShapeStruct(batch, n_q, n_k, n_v, d_qk, d_v, _dtype_code(dtype), _dtype_code(out_dtype), float(scale))
+
+
+def diffqkv_decode_num_splits(shape: ShapeStruct, max_seqlen: int) -> int:
+    return int(_lib.diffqkv_decode_num_splits(C.byref(shape), max_seqlen))
+
+
+def diffqkv_decode_workspace_bytes(shape: ShapeStruct, max_seqlen: int, num_splits: int = 0) -> int:
+    return int(_lib.diffqkv_decode_workspace_bytes(C.byref(shape), max_seqlen, num_splits))
+
+
+def _decode(fn_name, q, cache: KVCache, n_k, n_v, scale, num_splits, workspace, out, lse, dev_status,
+            out_dtype, stream):
+    batch, n_q, d_qk = q.shape
+    d_v = cache.v.shape[-1]
+    out_dtype = out_dtype or (out.dtype if out is not None else q.dtype)
+    shape = make_shape(batch, n_q, n_k, n_v, d_qk, d_v, q.dtype, out_dtype, scale)
+    if workspace is None:
+        nbytes = diffqkv_decode_workspace_bytes(shape, cache.max_seqlen, num_splits)
+        workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
+    if out is None:
+        out = torch.empty((batch, n_q, d_v), dtype=out_dtype, device=q.device)
+    cs = cache.c_struct()
+    st = getattr(_lib, fn_name)(_p(q), C.byref(cs), C.byref(shape), int(num_splits), _p(workspace),
+                                workspace.numel() * workspace.element_size(), _p(out), _p(lse),
+                                _p(dev_status), _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, fn_name)
+    return out
+
+
+def diffqkv_decode(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: float, num_splits: int = 0,
+                   workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                   lse: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                   out_dtype: Optional[torch.dtype] = None, stream: Optional[torch.cuda.Stream] = None):
+    """q [batch, n_q, d_qk] against the cache; returns out [batch, n_q, d_v] (enqueued on the stream)."""
+    return _decode("diffqkv_decode", q, cache, n_k, n_v, scale, num_splits, workspace, out, lse, dev_status,
+                   out_dtype, stream)
+
+
+def gqa_decode(q: torch.Tensor, cache: KVCache, n_kv: int, scale: float, num_splits: int = 0,
+               workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+               lse: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+               out_dtype: Optional[torch.dtype] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Grouped-query attention (n_k == n_v == n_kv) through the same kernels."""
+    return _decode("gqa_decode", q, cache, n_kv, n_kv, scale, num_splits, workspace, out, lse, dev_status,
+                   out_dtype, stream)
+
+
+def diffqkv_combine(o_partial: torch.Tensor, lse_partial: torch.Tensor, out_dtype: torch.dtype = torch.float32,
+                    out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                    stream: Optional[torch.cuda.Stream] = None):
+    """o_partial [batch, n_q, S, d_v] fp32, lse_partial [batch, n_q, S] fp32 -> out [batch, n_q, d_v]."""
+    batch, n_q, S, d_v = o_partial.shape
+    assert o_partial.dtype == torch.float32 and lse_partial.dtype == torch.float32
+    assert o_partial.is_contiguous() and lse_partial.is_contiguous()
+    if out is None:
+        out = torch.empty((batch, n_q, d_v), dtype=out_dtype, device=o_partial.device)
+    st = _lib.diffqkv_combine(_p(o_partial), _p(lse_partial), batch, n_q, d_v, S, _dtype_code(out.dtype),
+                              _p(out), _p(lse), _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_combine")
+    return out
+
+
+def diffqkv_prefill(q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, cache: KVCache, scale: float,
+                    out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                    dev_status: Optional[torch.Tensor] = None, out_dtype: Optional[torch.dtype] = None,
+                    stream: Optional[torch.cuda.Stream] = None):
+    """q [batch, q_len, n_q, d_qk]; writes k_new / v_new into the cache, returns out [batch, q_len, n_q, d_v]."""
+    batch, q_len, n_q, d_qk = q.shape
+    n_k, n_v, d_v = k_new.shape[2], v_new.shape[2], v_new.shape[3]
+    out_dtype = out_dtype or (out.dtype if out is not None else q.dtype)
+    shape = make_shape(batch, n_q, n_k, n_v, d_qk, d_v, q.dtype, out_dtype, scale)
+    if out is None:
+        out = torch.empty((batch, q_len, n_q, d_v), dtype=out_dtype, device=q.device)
+    cs = cache.c_struct()
+    st = _lib.diffqkv_prefill(_p(q), _p(k_new), _p(v_new), q_len, C.byref(cs), C.byref(shape), _p(out), _p(lse),
+                              _p(dev_status), _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_prefill")
+    return out
+
+
+def diffqkv_augq_workspace_bytes(T: int, d_q0: int, d_aug: int) -> int:
+    return int(_lib.diffqkv_augq_workspace_bytes(T, d_q0, d_aug))
+
+
+def diffqkv_augq(h: torch.Tensor, W_Q: torch.Tensor, W_gate: torch.Tensor, W_up: torch.Tensor,
+                 W_down: torch.Tensor, workspace: Optional[torch.Tensor] = None,
+                 q_out: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """h [T, d_model] bf16, weights in nn.Linear layout [out, in]; returns q [T, d_out] bf16."""
+    T, d_model = h.shape
+    d_q0, d_aug, d_out = W_Q.shape[0], W_gate.shape[0], W_down.shape[0]
+    if workspace is None:
+        workspace = torch.empty(max(diffqkv_augq_workspace_bytes(T, d_q0, d_aug), 256), dtype=torch.uint8,
+                                device=h.device)
+    if q_out is None:
+        q_out = torch.empty((T, d_out), dtype=torch.bfloat16, device=h.device)
+    st = _lib.diffqkv_augq(_p(h), _p(W_Q), _p(W_gate), _p(W_up), _p(W_down), T, d_model, d_q0, d_aug, d_out,
+                           _p(workspace), workspace.numel(), _p(q_out), _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_augq")
+    return q_out

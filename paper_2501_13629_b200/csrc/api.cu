@@ -1,0 +1,195 @@
+// C-ABI entry points of libdiffqkv: argument checks, split planning, kernel selection.
+#include <atomic>
+
+#include "common.cuh"
+
+namespace diffqkv {
+
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+DecodePlan plan_decode(const diffqkv_shape& shape, int max_seqlen, int num_splits) {
+  (void)shape;
+  if (max_seqlen < 1) max_seqlen = 1;
+  int want = num_splits;
+  if (want <= 0) want = (max_seqlen + 511) / 512;  // automatic: chunks of about 512 tokens
+  if (want < 1) want = 1;
+  int chunk = (max_seqlen + want - 1) / want;
+  chunk = (chunk + kChunkQuantum - 1) / kChunkQuantum * kChunkQuantum;
+  DecodePlan pl;
+  pl.chunk = chunk;
+  pl.splits = (max_seqlen + chunk - 1) / chunk;
+  return pl;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static diffqkv_status check_shape(const diffqkv_shape* s) {
+  if (!s) return DIFFQKV_ERR_INVALID_ARG;
+  if (s->batch < 0 || s->n_q <= 0 || s->n_k <= 0 || s->n_v <= 0 || s->d_qk <= 0 || s->d_v <= 0)
+    return DIFFQKV_ERR_INVALID_ARG;
+  if (s->n_q % s->n_k != 0 || s->n_q % s->n_v != 0) return DIFFQKV_ERR_INVALID_ARG;
+  if (s->dtype != DIFFQKV_BF16 && s->dtype != DIFFQKV_F32) return DIFFQKV_ERR_INVALID_ARG;
+  if (s->out_dtype != DIFFQKV_BF16 && s->out_dtype != DIFFQKV_F32) return DIFFQKV_ERR_INVALID_ARG;
+  if (!(s->scale == s->scale)) return DIFFQKV_ERR_INVALID_ARG;
+  if (s->batch > 65535 || s->n_q > 65535) return DIFFQKV_ERR_UNSUPPORTED;
+  const int vec = s->dtype == DIFFQKV_BF16 ? 8 : 4;
+  if (s->d_qk % vec != 0 || s->d_v % vec != 0) return DIFFQKV_ERR_UNSUPPORTED;
+  if (s->d_v > 512 || s->d_qk > 8192) return DIFFQKV_ERR_UNSUPPORTED;
+  return DIFFQKV_OK;
+}
+
+static diffqkv_status check_cache(const diffqkv_cache* c, const diffqkv_shape* s) {
+  if (!c || !c->k_cache || !c->v_cache || !c->seqlens) return DIFFQKV_ERR_INVALID_ARG;
+  if (c->max_seqlen < 0 || c->num_blocks < 0) return DIFFQKV_ERR_INVALID_ARG;
+  if (c->page_table) {
+    if (c->page_size <= 0 || c->max_pages_per_seq <= 0) return DIFFQKV_ERR_INVALID_ARG;
+    if ((long long)c->max_pages_per_seq * c->page_size < c->max_seqlen) return DIFFQKV_ERR_INVALID_ARG;
+  } else if (c->num_blocks < s->batch) {
+    return DIFFQKV_ERR_INVALID_ARG;
+  }
+  const int vec = s->dtype == DIFFQKV_BF16 ? 8 : 4;
+  const long long strides[6] = {c->k_stride_blk, c->k_stride_head, c->k_stride_tok,
+                                c->v_stride_blk, c->v_stride_head, c->v_stride_tok};
+  for (long long st : strides)
+    if (st < 0 || st % vec != 0) return DIFFQKV_ERR_ALIGNMENT;
+  if (c->k_stride_tok < s->d_qk || c->v_stride_tok < s->d_v) return DIFFQKV_ERR_INVALID_ARG;
+  if (!aligned16(c->k_cache) || !aligned16(c->v_cache)) return DIFFQKV_ERR_ALIGNMENT;
+  return DIFFQKV_OK;
+}
+
+static CacheView view_of(const diffqkv_cache* c) {
+  CacheView v;
+  v.k = c->k_cache;
+  v.v = c->v_cache;
+  v.k_sb = c->k_stride_blk; v.k_sh = c->k_stride_head; v.k_st = c->k_stride_tok;
+  v.v_sb = c->v_stride_blk; v.v_sh = c->v_stride_head; v.v_st = c->v_stride_tok;
+  v.seqlens = c->seqlens;
+  v.page_table = c->page_table;
+  v.page_size = c->page_size;
+  v.max_pages_per_seq = c->max_pages_per_seq;
+  v.num_blocks = c->num_blocks;
+  v.max_seqlen = c->max_seqlen;
+  return v;
+}
+
+static size_t decode_workspace_bytes(const diffqkv_shape& s, const DecodePlan& pl) {
+  const size_t rows = (size_t)s.batch * s.n_q;
+  return align_up(rows * pl.splits * s.d_v * sizeof(float), 256) + align_up(rows * pl.splits * sizeof(float), 256);
+}
+
+static diffqkv_status decode_impl(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape,
+                                  int32_t num_splits, void* workspace, size_t workspace_bytes, void* out,
+                                  float* lse, int32_t* dev_status, cudaStream_t stream) {
+  diffqkv_status st = check_shape(shape);
+  if (st != DIFFQKV_OK) return st;
+  if (!q || !out) return DIFFQKV_ERR_INVALID_ARG;
+  st = check_cache(cache, shape);
+  if (st != DIFFQKV_OK) return st;
+  if (!aligned16(q) || !aligned16(out)) return DIFFQKV_ERR_ALIGNMENT;
+  if (num_splits < 0) return DIFFQKV_ERR_INVALID_ARG;
+  if (shape->batch == 0) return DIFFQKV_OK;
+  const DecodePlan pl = plan_decode(*shape, cache->max_seqlen, num_splits);
+  const size_t need = decode_workspace_bytes(*shape, pl);
+  if (!workspace || workspace_bytes < need) return DIFFQKV_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DIFFQKV_ERR_ALIGNMENT;
+
+  const size_t rows = (size_t)shape->batch * shape->n_q;
+  DecodeParams p;
+  p.q = q;
+  p.cache = view_of(cache);
+  p.batch = shape->batch; p.n_q = shape->n_q; p.n_k = shape->n_k; p.n_v = shape->n_v;
+  p.d_qk = shape->d_qk; p.d_v = shape->d_v;
+  p.scale_log2 = shape->scale * kLog2e;
+  p.chunk = pl.chunk;
+  p.splits = pl.splits;
+  p.o_partial = reinterpret_cast<float*>(workspace);
+  p.lse_partial = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) +
+                                           align_up(rows * pl.splits * shape->d_v * sizeof(float), 256));
+  p.dev_status = dev_status;
+
+  cudaError_t err = launch_decode_generic(p, shape->dtype, stream);
+  if (err != cudaSuccess) return DIFFQKV_ERR_CUDA;
+  err = launch_combine(p.o_partial, p.lse_partial, (int)rows, shape->d_v, pl.splits, shape->out_dtype, out, lse,
+                       stream);
+  return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
+}
+
+}  // namespace diffqkv
+
+using namespace diffqkv;
+
+extern "C" {
+
+int32_t diffqkv_decode_num_splits(const diffqkv_shape* shape, int32_t max_seqlen) {
+  if (check_shape(shape) != DIFFQKV_OK) return 1;
+  return plan_decode(*shape, max_seqlen, 0).splits;
+}
+
+size_t diffqkv_decode_workspace_bytes(const diffqkv_shape* shape, int32_t max_seqlen, int32_t num_splits) {
+  if (check_shape(shape) != DIFFQKV_OK || max_seqlen < 0 || num_splits < 0) return 0;
+  return decode_workspace_bytes(*shape, plan_decode(*shape, max_seqlen, num_splits));
+}
+
+diffqkv_status diffqkv_decode(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape,
+                              int32_t num_splits, void* workspace, size_t workspace_bytes, void* out, float* lse,
+                              int32_t* dev_status, void* stream) {
+  return decode_impl(q, cache, shape, num_splits, workspace, workspace_bytes, out, lse, dev_status,
+                     static_cast<cudaStream_t>(stream));
+}
+
+diffqkv_status gqa_decode(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape, int32_t num_splits,
+                          void* workspace, size_t workspace_bytes, void* out, float* lse, int32_t* dev_status,
+                          void* stream) {
+  if (shape && shape->n_k != shape->n_v) return DIFFQKV_ERR_INVALID_ARG;
+  return decode_impl(q, cache, shape, num_splits, workspace, workspace_bytes, out, lse, dev_status,
+                     static_cast<cudaStream_t>(stream));
+}
+
+diffqkv_status diffqkv_combine(const float* o_partial, const float* lse_partial, int32_t batch, int32_t n_q,
+                               int32_t d_v, int32_t num_splits, diffqkv_dtype out_dtype, void* out, float* lse,
+                               void* stream) {
+  if (!o_partial || !lse_partial || !out) return DIFFQKV_ERR_INVALID_ARG;
+  if (batch < 0 || n_q <= 0 || d_v <= 0 || num_splits <= 0) return DIFFQKV_ERR_INVALID_ARG;
+  if (out_dtype != DIFFQKV_BF16 && out_dtype != DIFFQKV_F32) return DIFFQKV_ERR_INVALID_ARG;
+  if (num_splits > 8192) return DIFFQKV_ERR_UNSUPPORTED;
+  if ((long long)batch * n_q > 0x7fffffffLL) return DIFFQKV_ERR_UNSUPPORTED;
+  cudaError_t err = launch_combine(o_partial, lse_partial, batch * n_q, d_v, num_splits, out_dtype, out, lse,
+                                   static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
+}
+
+diffqkv_status diffqkv_prefill(const void*, const void*, const void*, int32_t, const diffqkv_cache*,
+                               const diffqkv_shape*, void*, float*, int32_t*, void*) {
+  return DIFFQKV_ERR_UNSUPPORTED;
+}
+
+size_t diffqkv_augq_workspace_bytes(int64_t T, int32_t d_q0, int32_t d_aug) {
+  if (T < 0 || d_q0 <= 0 || d_aug <= 0) return 0;
+  return align_up((size_t)T * d_q0 * 2, 256) + align_up((size_t)T * d_aug * 2, 256);
+}
+
+diffqkv_status diffqkv_augq(const void*, const void*, const void*, const void*, const void*, int64_t, int32_t,
+                            int32_t, int32_t, int32_t, void*, size_t, void*, void*) {
+  return DIFFQKV_ERR_UNSUPPORTED;
+}
+
+const char* diffqkv_status_string(diffqkv_status status) {
+  switch (status) {
+    case DIFFQKV_OK: return "ok";
+    case DIFFQKV_ERR_INVALID_ARG: return "invalid argument";
+    case DIFFQKV_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case DIFFQKV_ERR_ALIGNMENT: return "pointer or stride alignment";
+    case DIFFQKV_ERR_WORKSPACE: return "workspace missing or too small";
+    case DIFFQKV_ERR_CUDA: return "CUDA call failed";
+    case DIFFQKV_ERR_TIMEOUT: return "device wait ran out";
+    case DIFFQKV_ERR_INDEX: return "page id out of range";
+  }
+  return "unknown status";
+}
+
+int64_t diffqkv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

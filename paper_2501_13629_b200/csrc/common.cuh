@@ -1,0 +1,61 @@
+// Shared device/host helpers of libdiffqkv (CUDA side only; the CPU oracle shares nothing with this).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "diffqkv.h"
+
+namespace diffqkv {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Host-side decode plan: the sequence axis is cut into chunks of `chunk` tokens (a multiple of
+// kChunkQuantum); sequence b uses ceil(len_b / chunk) of the `splits` partial slots.
+constexpr int kChunkQuantum = 64;
+struct DecodePlan {
+  int chunk;
+  int splits;
+};
+DecodePlan plan_decode(const diffqkv_shape& shape, int max_seqlen, int num_splits);
+
+struct CacheView {  // device copy of the addressing part of diffqkv_cache
+  const void* k;
+  const void* v;
+  long long k_sb, k_sh, k_st;
+  long long v_sb, v_sh, v_st;
+  const int* seqlens;
+  const int* page_table;
+  int page_size, max_pages_per_seq, num_blocks, max_seqlen;
+};
+
+struct DecodeParams {
+  const void* q;
+  CacheView cache;
+  int batch, n_q, n_k, n_v, d_qk, d_v;
+  float scale_log2;  // scale * log2(e): scores are kept in the base-2 domain
+  int chunk, splits;
+  float* o_partial;    // [batch, n_q, splits, d_v]
+  float* lse_partial;  // [batch, n_q, splits]   natural log
+  int* dev_status;
+};
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void store_out(float* p, float x) { *p = x; }
+__device__ __forceinline__ void store_out(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+
+// Device-side conditions are reported as bit (1 << diffqkv_status) so that several can coexist.
+__device__ __forceinline__ void report(int* dev_status, int code) {
+  if (dev_status) atomicOr(dev_status, 1 << code);
+}
+
+// Launchers (defined next to their kernels).
+cudaError_t launch_decode_generic(const DecodeParams& p, diffqkv_dtype dtype, cudaStream_t stream);
+cudaError_t launch_combine(const float* o_partial, const float* lse_partial, int rows, int d_v, int splits,
+                           diffqkv_dtype out_dtype, void* out, float* lse, cudaStream_t stream);
+void count_launch(int n = 1);
+
+}  // namespace diffqkv

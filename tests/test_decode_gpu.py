@@ -1,0 +1,191 @@
+"""GPU parity of diffqkv_decode / gqa_decode / diffqkv_combine against the float64 oracle,
+called through the C ABI on the same seeded inputs."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2501_13629_b200 import workloads as W
+from helpers import check_bf16, check_f32, check_lse, device_cache, run_decode, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2501_13629_b200 import api as _api
+    assert torch.cuda.is_available()
+    return _api
+
+
+def test_cfg1_fp32_small(api, oracle):
+    """Config 1: batch 1, 16/2/4 heads, d 64, 512 tokens, fp32 cache, seed 0, scale 1/8."""
+    inp = W.make_decode_inputs(W.CFG1)
+    ref, lse_ref = run_oracle(oracle, inp)
+    for splits in (0, 1, 3, 8):
+        out, lse, st = run_decode(api, inp, num_splits=splits)
+        assert st == 0
+        check_f32(out, ref, f"cfg1 splits={splits}")
+        check_lse(lse, lse_ref, 1e-5 * np.abs(lse_ref).max())
+
+
+@pytest.mark.parametrize("cfg", [W.CFG2, W.CFG3], ids=lambda c: c.name)
+def test_full_size_bf16_and_gqa_twin(api, oracle, cfg):
+    """Configs 2 and 3 at full size, DiffQKV and the n_k = n_v twin, every output element."""
+    for c in (cfg, cfg.gqa_twin()):
+        inp = W.make_decode_inputs(c)
+        ref, lse_ref = run_oracle(oracle, inp)
+        gqa = c.n_k == c.n_v
+        out, lse, st = run_decode(api, inp, gqa=gqa)
+        assert st == 0
+        check_bf16(out, ref, c.name)
+        check_lse(lse, lse_ref, 2e-2, c.name)
+        out_b, _, _ = run_decode(api, inp, out_dtype=torch.bfloat16, gqa=gqa, want_lse=False)
+        check_bf16(out_b, ref, c.name + " bf16 out")
+
+
+SMALL = W.DecodeConfig("small", batch=3, n_q=16, n_k=2, n_v=4, d_qk=128, d_v=128, kv_len=700, seed=42)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("heads", [(16, 2, 4), (8, 8, 8), (8, 1, 1), (8, 1, 8), (12, 6, 2), (32, 4, 16), (4, 4, 2)])
+@pytest.mark.parametrize("d", [64, 128])
+def test_head_configurations(api, oracle, dtype, heads, d):
+    n_q, n_k, n_v = heads
+    cfg = dataclasses.replace(SMALL, n_q=n_q, n_k=n_k, n_v=n_v, d_qk=d, d_v=d, dtype=dtype)
+    inp = W.make_decode_inputs(cfg, seqlens=np.array([700, 1, 333], dtype=np.int32))
+    ref, lse_ref = run_oracle(oracle, inp)
+    out, lse, st = run_decode(api, inp)
+    assert st == 0
+    (check_bf16 if dtype == "bf16" else check_f32)(out, ref, str(heads))
+    check_lse(lse, lse_ref, 2e-2 if dtype == "bf16" else 1e-4)
+
+
+def test_mixed_head_dims(api, oracle):
+    cfg = dataclasses.replace(SMALL, d_qk=64, d_v=128)
+    inp = W.make_decode_inputs(cfg, seqlens=np.array([700, 65, 64], dtype=np.int32))
+    ref, _ = run_oracle(oracle, inp)
+    out, _, st = run_decode(api, inp)
+    assert st == 0
+    check_bf16(out, ref)
+
+
+@pytest.mark.parametrize("lens", [[0, 0, 0], [0, 5, 700], [63, 64, 65], [127, 128, 129], [1, 2, 3]])
+def test_ragged_and_empty_lengths(api, oracle, lens):
+    inp = W.make_decode_inputs(SMALL, seqlens=np.array(lens, dtype=np.int32))
+    ref, lse_ref = run_oracle(oracle, inp)
+    for splits in (0, 1, 5):
+        out, lse, st = run_decode(api, inp, num_splits=splits)
+        assert st == 0
+        check_bf16(out, ref, f"{lens} splits={splits}")
+        check_lse(lse, lse_ref, 2e-2)
+        for b, n in enumerate(lens):
+            if n == 0:
+                assert np.all(out[b] == 0.0) and np.all(np.isneginf(lse[b]))
+
+
+def test_split_count_invariance(api, oracle):
+    """Any split count gives the same result up to fp32 reassociation."""
+    inp = W.make_decode_inputs(dataclasses.replace(SMALL, kv_len=3000), seqlens=np.array([3000, 1500, 77], np.int32))
+    ref, _ = run_oracle(oracle, inp)
+    outs = []
+    for splits in (1, 2, 7, 16, 47):
+        out, _, st = run_decode(api, inp, num_splits=splits)
+        assert st == 0
+        check_bf16(out, ref, f"splits={splits}")
+        outs.append(out)
+    for o in outs[1:]:
+        assert np.abs(o - outs[0]).max() <= 5e-3
+
+
+@pytest.mark.parametrize("page_size", [16, 64])
+def test_paged_equals_contiguous_bitwise(api, oracle, page_size):
+    """Paging is pure addressing: identity table, shuffled table and the contiguous cache give
+    bit-identical outputs for the same chunking."""
+    inp = W.make_decode_inputs(dataclasses.replace(SMALL, kv_len=1024), seqlens=np.array([1024, 500, 17], np.int32))
+    ref, _ = run_oracle(oracle, inp)
+    base, lse0, st = run_decode(api, inp, num_splits=4)
+    assert st == 0
+    check_bf16(base, ref)
+    for identity in (True, False):
+        pg = W.paginate(inp, page_size, seed=9, identity=identity)
+        out, lse, st = run_decode(api, pg, num_splits=4)
+        assert st == 0
+        assert np.array_equal(out, base) and np.array_equal(lse, lse0)
+
+
+def test_token_major_layout(api, oracle):
+    """The (b, s, n_h, d_h) layout of the paper's cache, expressed through strides."""
+    inp = W.make_decode_inputs(SMALL, seqlens=np.array([700, 300, 64], np.int32))
+    base, _, _ = run_decode(api, inp)
+    c = inp.cfg
+    S = c.kv_len
+    tm = dataclasses.replace(
+        inp, k=np.ascontiguousarray(inp.k.transpose(0, 2, 1, 3)), v=np.ascontiguousarray(inp.v.transpose(0, 2, 1, 3)),
+        k_strides=(S * c.n_k * c.d_qk, c.d_qk, c.n_k * c.d_qk), v_strides=(S * c.n_v * c.d_v, c.d_v, c.n_v * c.d_v))
+    ref, _ = run_oracle(oracle, tm)
+    out, _, st = run_decode(api, tm)
+    assert st == 0
+    check_bf16(out, ref)
+    assert np.abs(out - base).max() <= 5e-3
+
+
+def test_out_of_range_page_is_reported_not_read(api):
+    """A page id outside the pool sets the INDEX bit in dev_status; the kernel skips the read."""
+    inp = W.make_decode_inputs(dataclasses.replace(SMALL, kv_len=256), seqlens=np.array([256, 256, 256], np.int32))
+    pg = W.paginate(inp, 16, seed=3)
+    pg.page_table[1, 3] = pg.num_pages + 5
+    pg.page_table[2, 0] = -1
+    out, lse, st = run_decode(api, pg)
+    assert st == (1 << api.ERR_INDEX)
+    assert np.all(np.isfinite(out))
+
+
+def test_paged_varlen_config5_shape_reduced(api, oracle):
+    """Config 5's structure (16-token pages, shuffled table, uniform lengths) at a reduced length range."""
+    cfg = dataclasses.replace(W.CFG5, batch=8, kv_len=4096, len_range=(64, 4096))
+    inp = W.make_decode_inputs(cfg)
+    ref, lse_ref = run_oracle(oracle, inp)
+    out, lse, st = run_decode(api, inp)
+    assert st == 0
+    check_bf16(out, ref)
+    check_lse(lse, lse_ref, 2e-2)
+
+
+def test_combine_entry_point(api, oracle):
+    rng = np.random.Generator(np.random.Philox(key=5))
+    o = rng.standard_normal((3, 8, 11, 128)).astype(np.float32)
+    l = (3 * rng.standard_normal((3, 8, 11))).astype(np.float32)
+    l[0, 0, :] = -np.inf
+    l[1, 2, 3:] = -np.inf
+    o[1, 2, 3:] = np.nan  # skipped splits must not be read into the result
+    ref, lse_ref = oracle.combine(o.astype(np.float64), l.astype(np.float64))
+    to, tl = torch.from_numpy(o).cuda(), torch.from_numpy(l).cuda()
+    lse = torch.empty((3, 8), dtype=torch.float32, device="cuda")
+    out = api.diffqkv_combine(to, tl, out_dtype=torch.float32, lse=lse)
+    torch.cuda.synchronize()
+    check_f32(out.cpu().numpy().astype(np.float64), ref)
+    check_lse(lse.cpu().numpy().astype(np.float64), lse_ref, 1e-5)
+    out_b = api.diffqkv_combine(to, tl, out_dtype=torch.bfloat16)
+    check_bf16(out_b.float().cpu().numpy().astype(np.float64), ref)
+
+
+def test_dominant_and_uniform_softmax(api, oracle):
+    """Structured inputs: identical keys (uniform weights) and one dominant key (peaked weights)."""
+    cfg = dataclasses.replace(SMALL, batch=2, kv_len=600)
+    inp = W.make_decode_inputs(cfg, seqlens=np.array([600, 431], np.int32))
+    inp.k[:] = inp.k[:, :, :1]  # every token has the same key
+    ref, _ = run_oracle(oracle, inp)
+    out, _, _ = run_decode(api, inp)
+    check_bf16(out, ref, "uniform")
+    vf = W.as_f64(inp.v)
+    for b, n in enumerate([600, 431]):
+        for h in range(cfg.n_q):
+            assert np.abs(out[b, h] - vf[b, h // 4, :n].mean(axis=0)).max() <= 2e-2
+    inp2 = W.make_decode_inputs(cfg, seqlens=np.array([600, 431], np.int32))
+    qf = W.bf16_bits_to_f32(inp2.q)
+    inp2.k[:, :, 300] = W.f32_to_bf16_bits(4.0 * qf[:, ::8])  # dominant for the first head of each K group
+    ref2, _ = run_oracle(oracle, inp2)
+    out2, _, _ = run_decode(api, inp2)
+    check_bf16(out2, ref2, "dominant")
