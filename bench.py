@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the DiffQKV decode path on B200: KV-cache GB/s and fraction of the HBM roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--quick]
+
+Headline workload: long-context DiffQKV decode (batch 4, 32/4/8 heads, d 128, 32768 cached tokens,
+bf16).  One step = one ``diffqkv_decode`` call (split kernel + combine kernel) over the whole batch.
+The line printed by rank 0 also carries the GQA twin (n_k = n_v), the other decode configurations,
+the roofline of the split kernel and the CPU oracle timed on the host cores.
+
+With N > 1 every rank runs the same workload on its own GPU (the path has no exchange step:
+replicas only), the timed region is bracketed by barriers and the slowest rank's time is used.
+``--impl reference`` times the float64 CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_kv_cache_bandwidth"
+UNIT = "GB/s"
+L2_BYTES = 126 * 1024 * 1024
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def kv_bytes(cfg, seqlens) -> float:
+    """Algorithmic bytes of one decode step: every cached K and V element once."""
+    return float(np.sum(seqlens.astype(np.int64))) * (cfg.n_k * cfg.d_qk + cfg.n_v * cfg.d_v) * \
+        (2 if cfg.dtype == "bf16" else 4)
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.01)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------- GPU arm
+class DecodeCase:
+    """One decode workload resident on the device, with `rotate` distinct copies of the cache so that
+    consecutive steps never find their cache lines in L2."""
+
+    def __init__(self, api, cfg, device, host_inputs=None, rotate=None):
+        import torch
+        from paper_2501_13629_b200 import workloads as W
+        self.api, self.cfg, self.torch = api, cfg, torch
+        if host_inputs is not None:
+            inp = host_inputs
+            self.seqlens_host = inp.seqlens
+            k, v = W.to_torch(inp.k, device), W.to_torch(inp.v, device)
+            q = W.to_torch(inp.q, device)
+            pt = None if inp.page_table is None else torch.from_numpy(inp.page_table).to(device)
+            num_blocks = inp.num_pages if pt is not None else cfg.batch
+            max_seqlen, ks, vs = inp.max_seqlen, inp.k_strides, inp.v_strides
+        else:  # large pools: same recipe (i.i.d. N(0,1) rounded to bf16), drawn on the device
+            g = torch.Generator(device=device)
+            g.manual_seed(cfg.seed)
+            self.seqlens_host = W.draw_lengths(cfg)
+            q = torch.randn((cfg.batch, cfg.n_q, cfg.d_qk), generator=g, device=device).to(torch.bfloat16)
+            if cfg.page_size:
+                table, num_blocks = W.shuffled_page_table(self.seqlens_host, cfg.page_size, cfg.seed)
+                pt = torch.from_numpy(table).to(device)
+                k = torch.empty((num_blocks, cfg.n_k, cfg.page_size, cfg.d_qk), dtype=torch.bfloat16, device=device)
+                v = torch.empty((num_blocks, cfg.n_v, cfg.page_size, cfg.d_v), dtype=torch.bfloat16, device=device)
+                max_seqlen = int(table.shape[1]) * cfg.page_size
+            else:
+                pt, num_blocks, max_seqlen = None, cfg.batch, cfg.kv_len
+                k = torch.empty((cfg.batch, cfg.n_k, cfg.kv_len, cfg.d_qk), dtype=torch.bfloat16, device=device)
+                v = torch.empty((cfg.batch, cfg.n_v, cfg.kv_len, cfg.d_v), dtype=torch.bfloat16, device=device)
+            for t in (k, v):  # fill in slices to bound temporary memory
+                flat = t.view(-1)
+                step = 1 << 28
+                for lo in range(0, flat.numel(), step):
+                    n = min(step, flat.numel() - lo)
+                    flat[lo:lo + n] = torch.randn(n, generator=g, device=device).to(torch.bfloat16)
+            ks = (k.stride(0), k.stride(1), k.stride(2))
+            vs = (v.stride(0), v.stride(1), v.stride(2))
+        self.bytes = kv_bytes(cfg, self.seqlens_host)
+        pool_bytes = (k.numel() + v.numel()) * k.element_size()
+        if rotate is None:
+            rotate = 1 if pool_bytes > 4 * L2_BYTES else min(64, int(np.ceil(4 * L2_BYTES / pool_bytes)))
+        self.rotate = rotate
+        seqlens = torch.from_numpy(self.seqlens_host).to(device)
+        self.caches = []
+        for r in range(rotate):
+            kk, vv = (k, v) if r == 0 else (k.clone(), v.clone())
+            self.caches.append(api.KVCache(kk, vv, seqlens, int(max_seqlen), page_table=pt,
+                                           page_size=cfg.page_size, k_strides=ks, v_strides=vs,
+                                           num_blocks=num_blocks))
+        self.q = q
+        self.shape = api.make_shape(cfg.batch, cfg.n_q, cfg.n_k, cfg.n_v, cfg.d_qk, cfg.d_v, q.dtype,
+                                    torch.bfloat16, cfg.scale)
+        nbytes = api.diffqkv_decode_workspace_bytes(self.shape, int(max_seqlen), 0)
+        self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+        self.out = torch.empty((cfg.batch, cfg.n_q, cfg.d_v), dtype=torch.bfloat16, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.working_set = pool_bytes * rotate
+        self._i = 0
+
+    def step(self, q=None, out=None):
+        cfg = self.cfg
+        cache = self.caches[self._i % self.rotate]
+        self._i += 1
+        fn = self.api.gqa_decode if cfg.n_k == cfg.n_v else None
+        if fn is not None:
+            fn(self.q if q is None else q, cache, cfg.n_k, cfg.scale, workspace=self.workspace,
+               out=self.out if out is None else out, dev_status=self.status)
+        else:
+            self.api.diffqkv_decode(self.q if q is None else q, cache, cfg.n_k, cfg.n_v, cfg.scale,
+                                    workspace=self.workspace, out=self.out if out is None else out,
+                                    dev_status=self.status)
+
+    def time_steps(self, steps, warmup, barrier=None):
+        """Device time of `steps` consecutive steps, in ms (CUDA events on the launching stream)."""
+        torch = self.torch
+        for _ in range(warmup):
+            self.step()
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(steps):
+            self.step()
+        end.record()
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+        return start.elapsed_time(end)
+
+    def time_split_kernel(self, steps):
+        """Average duration of the split kernel alone: the library records an event pair around it."""
+        torch, api = self.torch, self.api
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in pairs:
+            a.record()  # creates the underlying CUDA events
+            b.record()
+        torch.cuda.synchronize()
+        for a, b in pairs:
+            api.set_split_events(a, b)
+            self.step()
+        api.set_split_events(None, None)
+        torch.cuda.synchronize()
+        return float(np.mean([a.elapsed_time(b) for a, b in pairs]))
+
+    def time_e2e(self, steps, warmup):
+        """Same step through the binding with HOST buffers: pinned q and seqlens copied to the device and
+        the output read back inside the timed region (the KV cache is decode state and stays resident)."""
+        torch = self.torch
+        q_host = self.q.cpu().pin_memory()
+        out_host = torch.empty(self.out.shape, dtype=self.out.dtype).pin_memory()
+        q_dev = torch.empty_like(self.q)
+        for i in range(warmup + steps):
+            if i == warmup:
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+            q_dev.copy_(q_host, non_blocking=True)
+            self.step(q=q_dev)
+            out_host.copy_(self.out, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+        dt = time.perf_counter() - t0
+        return dt * 1e3, q_host.numel() * q_host.element_size(), out_host.numel() * out_host.element_size()
+
+
+def run_ours(args):
+    import torch
+    from paper_2501_13629_b200 import api, workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    barrier = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+        barrier = lambda: (dist.barrier(), torch.cuda.synchronize())  # noqa: E731
+    peaks = measured_peaks()
+
+    cfg = W.CFG3
+    host = W.make_decode_inputs(cfg)
+    case = DecodeCase(api, cfg, device, host_inputs=host)
+    launches0 = api.launch_count()
+    with ClockSampler(local_rank) as clocks:
+        ms = case.time_steps(args.steps, args.warmup, barrier)
+    launches = api.launch_count() - launches0 - 0
+    launches_timed = launches * args.steps // (args.steps + args.warmup)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    assert int(case.status.item()) == 0, "device status reported an error"
+    ms_per_step = ms / args.steps
+    value = world * case.bytes / (ms_per_step * 1e-3) / 1e9
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "cfg3: DiffQKV decode batch 4, n_q 32, n_k 4, n_v 8, d 128, KV length 32768, bf16 "
+                               "cache [batch, head, seq, dim], one query token per sequence",
+                   "kv_bytes_per_step": case.bytes, "parallelism": "replicas" if world > 1 else "single",
+                   "l2": f"inputs larger than L2: {case.rotate} distinct cache copies rotated, "
+                         f"working set {case.working_set / 1e6:.0f} MB"},
+        "gpu_launches": launches_timed,
+        "clocks": clocks.summary(),
+        "tokens_per_s_per_layer": world * cfg.batch / (ms_per_step * 1e-3),
+        "frac_of_8TBs_nominal": value / world / 8000.0,
+        "frac_of_measured_hbm": value / world / peaks["hbm_gbs"],
+    }
+
+    if rank == 0:
+        # roofline of the dominant (split) kernel, timed alone by events the library records around it
+        k_ms = case.time_split_kernel(min(args.steps, 200))
+        ach = case.bytes / (k_ms * 1e-3) / 1e9
+        line["roofline"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                            "frac": ach / peaks["hbm_gbs"], "traffic": None, "kernel": "decode split kernel",
+                            "kernel_ms": k_ms, "peak_source": peaks["source"] + " (burst copy)"}
+        e2e_ms, h2d, d2h = case.time_e2e(min(args.steps, 500), min(args.warmup, 20))
+        e2e_step = e2e_ms / min(args.steps, 500)
+        line["e2e"] = {"value": world * case.bytes / (e2e_step * 1e-3) / 1e9, "unit": UNIT,
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_step,
+                       "note": "pinned q copied in and out copied back each step; the KV cache is resident state"}
+        others = {}
+        if not args.quick and world == 1:
+            twin = DecodeCase(api, cfg.gqa_twin(), device, host_inputs=W.make_decode_inputs(cfg.gqa_twin()))
+            t_ms = twin.time_steps(args.steps, args.warmup) / args.steps
+            others["cfg3_gqa_twin"] = {"ms_per_step": t_ms, "GB/s": twin.bytes / t_ms / 1e6,
+                                       "tokens_per_s_per_layer": cfg.batch / (t_ms * 1e-3)}
+            line["diffqkv_vs_gqa_speedup_32k"] = t_ms / ms_per_step
+            del twin
+            for c in (W.CFG2, W.CFG2.gqa_twin(), W.CFG1):
+                cs = DecodeCase(api, c, device, host_inputs=W.make_decode_inputs(c))
+                c_ms = cs.time_steps(args.steps, args.warmup) / args.steps
+                others[c.name] = {"ms_per_step": c_ms, "GB/s": cs.bytes / c_ms / 1e6, "rotate": cs.rotate}
+                del cs
+            torch.cuda.empty_cache()
+            c5 = DecodeCase(api, W.CFG5, device)
+            n5 = max(5, min(args.steps, 30))
+            c5_ms = c5.time_steps(n5, 3) / n5
+            others[W.CFG5.name] = {"ms_per_step": c5_ms, "GB/s": c5.bytes / c5_ms / 1e6,
+                                   "kv_bytes": c5.bytes, "frac_of_measured_hbm": c5.bytes / c5_ms / 1e6 / peaks["hbm_gbs"]}
+            del c5
+        line["others"] = others
+        line["cpu_baseline"] = cpu_baseline(host, budget_s=12.0)
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- oracle arm
+def _time_oracle_pairs(oracle, host, pairs):
+    cfg = host.cfg
+    cache = oracle.Cache(host.k, host.v, host.k_strides, host.v_strides, host.seqlens, host.page_table,
+                         cfg.page_size)
+    t0 = time.perf_counter()
+    oracle.decode(host.q, cache, cfg.n_q, cfg.n_k, cfg.n_v, cfg.d_qk, cfg.d_v, cfg.scale, pairs=pairs)
+    return time.perf_counter() - t0
+
+
+def _all_pairs(cfg):
+    return np.array([(b, h) for b in range(cfg.batch) for h in range(cfg.n_q)], dtype=np.int32)
+
+
+def cpu_baseline(host, budget_s=20.0):
+    """The float64 oracle, as it stands, on the host cores, on a bounded sample of the same workload."""
+    import oracle
+    cores = oracle.set_threads(0)
+    cfg = host.cfg
+    pairs = _all_pairs(cfg)
+    t1 = _time_oracle_pairs(oracle, host, pairs)  # the whole workload once (also warms the page cache)
+    reps = int(max(1, min(200, budget_s / max(t1, 1e-6))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        _time_oracle_pairs(oracle, host, pairs)
+    dt = (time.perf_counter() - t0) / reps
+    return {"value": kv_bytes(cfg, host.seqlens) / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"all {len(pairs)} (sequence, query head) rows of cfg3 at the full 32768-token context, "
+                      f"{reps} repetitions, {dt:.3f} s each", "seconds": dt * reps}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2501_13629_b200 import workloads as W
+    oracle.build()
+    cores = oracle.set_threads(0)
+    cfg = W.CFG3
+    host = W.make_decode_inputs(cfg)
+    pairs = _all_pairs(cfg)
+    t_row = _time_oracle_pairs(oracle, host, pairs[:cores]) / 1.0  # wall time of `cores` rows in parallel
+    budget = 150.0
+    total_steps = args.steps + args.warmup
+    per_step_rows = int(max(1, min(len(pairs), (budget / total_steps / max(t_row, 1e-6)) * cores)))
+    sample = pairs[:per_step_rows]
+    for _ in range(args.warmup):
+        _time_oracle_pairs(oracle, host, sample)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        _time_oracle_pairs(oracle, host, sample)
+    dt = time.perf_counter() - t0
+    ms_per_step = dt / args.steps * 1e3
+    value = (per_step_rows / len(pairs)) * kv_bytes(cfg, host.seqlens) / (ms_per_step * 1e-3) / 1e9
+    desc = (f"each step: {per_step_rows} of {len(pairs)} (sequence, query head) rows of cfg3 at the full "
+            f"32768-token context")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "cfg3: DiffQKV decode batch 4, n_q 32, n_k 4, n_v 8, d 128, KV length 32768, bf16 "
+                               "cache [batch, head, seq, dim], one query token per sequence", "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--quick", action="store_true", help="headline workload only")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -169,6 +169,14 @@ diffqkv_status diffqkv_augq(const void *h, const void *W_Q, const void *W_gate, 
 /* Static, never-null description of a status value. */
 const char *diffqkv_status_string(diffqkv_status status);
 
+/*
+ * Profiling hook for benchmarks (process-wide host state, not thread-safe).  While both arguments
+ * are non-NULL cudaEvent_t handles, every decode call records `before_split` just before and
+ * `after_split` just after its split kernel on the call's stream, so the split kernel can be timed
+ * apart from the combine kernel.  Pass NULL, NULL to switch it off.
+ */
+void diffqkv_profile_split_events(void *before_split, void *after_split);
+
 /* Kernels launched by this library since it was loaded (host counter, for benchmarks). */
 int64_t diffqkv_launch_count(void);
 

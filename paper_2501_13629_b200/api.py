@@ -28,7 +28,7 @@ BF16, F32 = 0, 1
 EXPORTS = (
     "diffqkv_decode_num_splits", "diffqkv_decode_workspace_bytes", "diffqkv_decode", "gqa_decode",
     "diffqkv_combine", "diffqkv_prefill", "diffqkv_augq_workspace_bytes", "diffqkv_augq",
-    "diffqkv_status_string", "diffqkv_launch_count",
+    "diffqkv_status_string", "diffqkv_launch_count", "diffqkv_profile_split_events",
 )
 
 
@@ -74,6 +74,8 @@ _lib.diffqkv_augq.argtypes = [C.c_void_p] * 5 + [C.c_int64, C.c_int32, C.c_int32
 _lib.diffqkv_status_string.restype = C.c_char_p
 _lib.diffqkv_status_string.argtypes = [C.c_int]
 _lib.diffqkv_launch_count.restype = C.c_int64
+_lib.diffqkv_profile_split_events.restype = None
+_lib.diffqkv_profile_split_events.argtypes = [C.c_void_p, C.c_void_p]
 
 
 class DiffQKVError(RuntimeError):
@@ -88,6 +90,12 @@ def status_string(status: int) -> str:
 
 def launch_count() -> int:
     return int(_lib.diffqkv_launch_count())
+
+
+def set_split_events(before: Optional[torch.cuda.Event], after: Optional[torch.cuda.Event]) -> None:
+    """Benchmark hook: have decode calls record these events around their split kernel (None, None = off)."""
+    _lib.diffqkv_profile_split_events(None if before is None else C.c_void_p(before.cuda_event),
+                                      None if after is None else C.c_void_p(after.cuda_event))
 
 
 def _dtype_code(dt: torch.dtype) -> int:

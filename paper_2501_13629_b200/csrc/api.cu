@@ -22,6 +22,8 @@ DecodePlan plan_decode(const diffqkv_shape& shape, int max_seqlen, int num_split
   return pl;
 }
 
+static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
+
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -110,7 +112,10 @@ static diffqkv_status decode_impl(const void* q, const diffqkv_cache* cache, con
                                            align_up(rows * pl.splits * shape->d_v * sizeof(float), 256));
   p.dev_status = dev_status;
 
+  const bool timed = g_ev_before && g_ev_after;
+  if (timed) cudaEventRecord(g_ev_before, stream);
   cudaError_t err = launch_decode_generic(p, shape->dtype, stream);
+  if (timed) cudaEventRecord(g_ev_after, stream);
   if (err != cudaSuccess) return DIFFQKV_ERR_CUDA;
   err = launch_combine(p.o_partial, p.lse_partial, (int)rows, shape->d_v, pl.splits, shape->out_dtype, out, lse,
                        stream);
@@ -188,6 +193,11 @@ const char* diffqkv_status_string(diffqkv_status status) {
     case DIFFQKV_ERR_INDEX: return "page id out of range";
   }
   return "unknown status";
+}
+
+void diffqkv_profile_split_events(void* before_split, void* after_split) {
+  g_ev_before = static_cast<cudaEvent_t>(before_split);
+  g_ev_after = static_cast<cudaEvent_t>(after_split);
 }
 
 int64_t diffqkv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
