@@ -116,6 +116,29 @@ diffqkv_status diffqkv_decode(const void *q, const diffqkv_cache *cache, const d
                               float *lse, int32_t *dev_status, void *stream);
 
 /*
+ * diffqkv_decode_static -- diffqkv_decode for callers that cannot provide or allocate a workspace.
+ * (The paper has no counterpart; this is a deployment convenience of this library.)
+ * Some hosts cannot call cudaMalloc when they decode: all device memory already belongs to their own
+ * pool, or they sit behind an interface with no workspace argument, or an allocation would stall a
+ * latency-critical loop.  For them the split kernel's partial results go to a fixed 8 MiB array built
+ * into the library (each GPU that loads the library carries those 8 MiB until the process exits).
+ * Arguments and results are those of diffqkv_decode without `workspace` / `workspace_bytes`.
+ *   - Returns DIFFQKV_ERR_WORKSPACE, launching nothing, when
+ *     diffqkv_decode_workspace_bytes(shape, cache->max_seqlen, num_splits) exceeds 8 MiB (8388608 bytes);
+ *     choose fewer splits or a smaller batch, or use diffqkv_decode with your own buffer.
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - The first call on each device resolves the array's device address (the device of `stream` must be
+ *     the current device); make that first call outside any stream capture.
+ *   - All calls on one device share the one array: two calls whose kernels may overlap on the GPU
+ *     (different streams without ordering, or several host threads) race on it.  Calls on one stream
+ *     are safe.  The array keeps the previous call's partials; nothing in it needs clearing because a
+ *     call reads only what it has itself written.
+ */
+diffqkv_status diffqkv_decode_static(const void *q, const diffqkv_cache *cache, const diffqkv_shape *shape,
+                                     int32_t num_splits, void *out, float *lse, int32_t *dev_status,
+                                     void *stream);
+
+/*
  * gqa_decode -- grouped-query attention, the comparison point of the paper (Appendix B.1: GQA is
  * the special case n_k == n_v).  Same arguments and the same kernels as diffqkv_decode; returns
  * DIFFQKV_ERR_INVALID_ARG when shape.n_k != shape.n_v.

@@ -28,7 +28,7 @@ BF16, F32 = 0, 1
 EXPORTS = (
     "diffqkv_decode_num_splits", "diffqkv_decode_workspace_bytes", "diffqkv_decode", "gqa_decode",
     "diffqkv_combine", "diffqkv_prefill", "diffqkv_augq_workspace_bytes", "diffqkv_augq",
-    "diffqkv_status_string", "diffqkv_launch_count", "diffqkv_profile_split_events",
+    "diffqkv_status_string", "diffqkv_launch_count", "diffqkv_profile_split_events", "diffqkv_decode_static",
 )
 
 
@@ -60,6 +60,9 @@ _DECODE_ARGS = [C.c_void_p, C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_
 for _name in ("diffqkv_decode", "gqa_decode"):
     getattr(_lib, _name).restype = C.c_int
     getattr(_lib, _name).argtypes = _DECODE_ARGS
+_lib.diffqkv_decode_static.restype = C.c_int
+_lib.diffqkv_decode_static.argtypes = [C.c_void_p, C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_int32,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.diffqkv_combine.restype = C.c_int
 _lib.diffqkv_combine.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int,
                                  C.c_void_p, C.c_void_p, C.c_void_p]
@@ -186,6 +189,26 @@ def diffqkv_decode(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: f
     """q [batch, n_q, d_qk] against the cache; returns out [batch, n_q, d_v] (enqueued on the stream)."""
     return _decode("diffqkv_decode", q, cache, n_k, n_v, scale, num_splits, workspace, out, lse, dev_status,
                    out_dtype, stream)
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def diffqkv_decode_static(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: float, out: torch.Tensor,
+                          num_splits: int = 0, lse: Optional[torch.Tensor] = None,
+                          dev_status: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """diffqkv_decode for callers that must not allocate: the split partials go to the 8 MiB array built
+    into the library, and ``out`` has to be passed in (this wrapper allocates nothing either).  Raises
+    DiffQKVError(ERR_WORKSPACE) when the shape needs more than STATIC_SCRATCH_BYTES.  Calls on one stream
+    are ordered; calls that can overlap on the GPU share the array and race."""
+    batch, n_q, d_qk = q.shape
+    shape = make_shape(batch, n_q, n_k, n_v, d_qk, cache.v.shape[-1], q.dtype, out.dtype, scale)
+    cs = cache.c_struct()
+    st = _lib.diffqkv_decode_static(_p(q), C.byref(cs), C.byref(shape), int(num_splits), _p(out), _p(lse),
+                                    _p(dev_status), _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_decode_static")
+    return out
 
 
 def gqa_decode(q: torch.Tensor, cache: KVCache, n_kv: int, scale: float, num_splits: int = 0,
