@@ -102,7 +102,10 @@ size_t diffqkv_decode_workspace_bytes(const diffqkv_shape *shape, int32_t max_se
  * the head map of Eq. (idx); split-sequence execution per Section 3.2).
  *   q          [batch, n_q, d_qk]  shape.dtype, contiguous
  *   cache      see diffqkv_cache; seqlens[b] == 0 gives out = 0 and lse = -inf for that sequence
- *   num_splits maximum splits per sequence, 0 = automatic
+ *   num_splits 0 = automatic (recommended): bf16 caches that a TMA tensor map can describe use the
+ *              persistent TMA kernel, which divides all (sequence, head group, 64-token tile) work
+ *              evenly over one block per SM and cuts sequences wherever a block's share ends; other
+ *              inputs use fixed chunks.  > 0 = fixed chunks, at most that many per sequence (generic kernel)
  *   workspace  at least diffqkv_decode_workspace_bytes(...) bytes, 256-byte aligned; holds the
  *              per-split partial outputs (fp32 [batch, n_q, S, d_v]) and log-sum-exps
  *              (fp32 [batch, n_q, S]); contents on entry are ignored
@@ -191,6 +194,16 @@ diffqkv_status diffqkv_augq(const void *h, const void *W_Q, const void *W_gate, 
 
 /* Static, never-null description of a status value. */
 const char *diffqkv_status_string(diffqkv_status status);
+
+/*
+ * Tuning hook (process-wide host state): cap the number of persistent blocks the TMA decode kernel
+ * launches; 0 restores the default of one block per SM.  Workspace sizes must be queried after the
+ * cap is set.  Mainly for tests, which use it to move the places where sequences are cut.
+ */
+void diffqkv_set_max_blocks(int32_t max_blocks);
+
+/* Which split kernel the most recent decode call launched: 0 none yet, 1 generic, 2 TMA (for tests). */
+int32_t diffqkv_last_decode_kernel(void);
 
 /*
  * Profiling hook for benchmarks (process-wide host state, not thread-safe).  While both arguments

@@ -29,6 +29,7 @@ EXPORTS = (
     "diffqkv_decode_num_splits", "diffqkv_decode_workspace_bytes", "diffqkv_decode", "gqa_decode",
     "diffqkv_combine", "diffqkv_prefill", "diffqkv_augq_workspace_bytes", "diffqkv_augq",
     "diffqkv_status_string", "diffqkv_launch_count", "diffqkv_profile_split_events", "diffqkv_decode_static",
+    "diffqkv_set_max_blocks", "diffqkv_last_decode_kernel",
 )
 
 
@@ -77,6 +78,8 @@ _lib.diffqkv_augq.argtypes = [C.c_void_p] * 5 + [C.c_int64, C.c_int32, C.c_int32
 _lib.diffqkv_status_string.restype = C.c_char_p
 _lib.diffqkv_status_string.argtypes = [C.c_int]
 _lib.diffqkv_launch_count.restype = C.c_int64
+_lib.diffqkv_set_max_blocks.restype = None
+_lib.diffqkv_set_max_blocks.argtypes = [C.c_int32]
 _lib.diffqkv_profile_split_events.restype = None
 _lib.diffqkv_profile_split_events.argtypes = [C.c_void_p, C.c_void_p]
 
@@ -99,6 +102,19 @@ def set_split_events(before: Optional[torch.cuda.Event], after: Optional[torch.c
     """Benchmark hook: have decode calls record these events around their split kernel (None, None = off)."""
     _lib.diffqkv_profile_split_events(None if before is None else C.c_void_p(before.cuda_event),
                                       None if after is None else C.c_void_p(after.cuda_event))
+
+
+def set_max_blocks(n: int) -> None:
+    """Cap the persistent blocks of the TMA decode kernel (0 = one per SM); see diffqkv_set_max_blocks."""
+    _lib.diffqkv_set_max_blocks(int(n))
+
+
+KERNEL_NONE, KERNEL_GENERIC, KERNEL_TMA = 0, 1, 2
+
+
+def last_decode_kernel() -> int:
+    """0 none yet, 1 generic split kernel, 2 TMA split kernel."""
+    return int(_lib.diffqkv_last_decode_kernel())
 
 
 def _dtype_code(dt: torch.dtype) -> int:

@@ -12,7 +12,10 @@ DecodePlan plan_decode(const diffqkv_shape& shape, int max_seqlen, int num_split
   (void)shape;
   if (max_seqlen < 1) max_seqlen = 1;
   int want = num_splits;
-  if (want <= 0) want = (max_seqlen + 511) / 512;  // automatic: chunks of about 512 tokens
+  if (want <= 0) {  // automatic: chunks of about 512 tokens, at most 32 splits
+    want = (max_seqlen + 511) / 512;
+    if (want > 32) want = 32;
+  }
   if (want < 1) want = 1;
   int chunk = (max_seqlen + want - 1) / want;
   chunk = (chunk + kChunkQuantum - 1) / kChunkQuantum * kChunkQuantum;
@@ -23,6 +26,7 @@ DecodePlan plan_decode(const diffqkv_shape& shape, int max_seqlen, int num_split
 }
 
 static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
+static int g_last_kernel = 0;  // 0 none, 1 generic, 2 TMA
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -82,6 +86,26 @@ static size_t decode_workspace_bytes(const diffqkv_shape& s, const DecodePlan& p
   return align_up(rows * pl.splits * s.d_v * sizeof(float), 256) + align_up(rows * pl.splits * sizeof(float), 256);
 }
 
+// Workspace for either schedule.  The TMA path needs little, but whether a given cache layout can be
+// described by a tensor map is only known at the call, so the answer covers the generic kernel too.
+static size_t workspace_need(const diffqkv_shape& s, int max_seqlen, int num_splits) {
+  size_t need = decode_workspace_bytes(s, plan_decode(s, max_seqlen, num_splits));
+  if (num_splits == 0) {
+    diffqkv_cache fake = {};
+    fake.max_seqlen = max_seqlen;
+    TmaPlan tp;
+    if (tma_decode_supported(s, fake, &tp)) {
+      const size_t t = tma_decode_workspace_bytes(s, tp);
+      if (t > need) need = t;
+    }
+  }
+  return need;
+}
+
+void profile_after_split(cudaStream_t stream) {
+  if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_after, stream);
+}
+
 static diffqkv_status decode_impl(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape,
                                   int32_t num_splits, void* workspace, size_t workspace_bytes, void* out,
                                   float* lse, int32_t* dev_status, cudaStream_t stream) {
@@ -94,9 +118,22 @@ static diffqkv_status decode_impl(const void* q, const diffqkv_cache* cache, con
   if (num_splits < 0) return DIFFQKV_ERR_INVALID_ARG;
   if (shape->batch == 0) return DIFFQKV_OK;
   const DecodePlan pl = plan_decode(*shape, cache->max_seqlen, num_splits);
-  const size_t need = decode_workspace_bytes(*shape, pl);
+  const size_t need = workspace_need(*shape, cache->max_seqlen, num_splits);
   if (!workspace || workspace_bytes < need) return DIFFQKV_ERR_WORKSPACE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DIFFQKV_ERR_ALIGNMENT;
+  const bool timed = g_ev_before && g_ev_after;
+
+  // bf16 caches a tensor map can describe go to the TMA kernel (automatic schedule only)
+  TmaPlan tp;
+  if (num_splits == 0 && tma_decode_supported(*shape, *cache, &tp)) {
+    if (timed) cudaEventRecord(g_ev_before, stream);
+    const cudaError_t terr = launch_decode_tma(q, *cache, *shape, tp, workspace, out, lse, dev_status, stream);
+    if (terr == cudaSuccess) {
+      g_last_kernel = 2;
+      return DIFFQKV_OK;
+    }
+    if (terr != cudaErrorNotSupported) return DIFFQKV_ERR_CUDA;
+  }
 
   const size_t rows = (size_t)shape->batch * shape->n_q;
   DecodeParams p;
@@ -112,10 +149,10 @@ static diffqkv_status decode_impl(const void* q, const diffqkv_cache* cache, con
                                            align_up(rows * pl.splits * shape->d_v * sizeof(float), 256));
   p.dev_status = dev_status;
 
-  const bool timed = g_ev_before && g_ev_after;
   if (timed) cudaEventRecord(g_ev_before, stream);
   cudaError_t err = launch_decode_generic(p, shape->dtype, stream);
-  if (timed) cudaEventRecord(g_ev_after, stream);
+  g_last_kernel = 1;
+  profile_after_split(stream);
   if (err != cudaSuccess) return DIFFQKV_ERR_CUDA;
   err = launch_combine(p.o_partial, p.lse_partial, (int)rows, shape->d_v, pl.splits, shape->out_dtype, out, lse,
                        stream);
@@ -135,8 +172,12 @@ int32_t diffqkv_decode_num_splits(const diffqkv_shape* shape, int32_t max_seqlen
 
 size_t diffqkv_decode_workspace_bytes(const diffqkv_shape* shape, int32_t max_seqlen, int32_t num_splits) {
   if (check_shape(shape) != DIFFQKV_OK || max_seqlen < 0 || num_splits < 0) return 0;
-  return decode_workspace_bytes(*shape, plan_decode(*shape, max_seqlen, num_splits));
+  return workspace_need(*shape, max_seqlen, num_splits);
 }
+
+void diffqkv_set_max_blocks(int32_t max_blocks) { set_tma_max_blocks(max_blocks); }
+
+int32_t diffqkv_last_decode_kernel(void) { return g_last_kernel; }
 
 diffqkv_status diffqkv_decode(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape,
                               int32_t num_splits, void* workspace, size_t workspace_bytes, void* out, float* lse,

@@ -57,5 +57,19 @@ cudaError_t launch_decode_generic(const DecodeParams& p, diffqkv_dtype dtype, cu
 cudaError_t launch_combine(const float* o_partial, const float* lse_partial, int rows, int d_v, int splits,
                            diffqkv_dtype out_dtype, void* out, float* lse, cudaStream_t stream);
 void count_launch(int n = 1);
+void profile_after_split(cudaStream_t stream);  // records the benchmark hook's second event, if armed
+
+// TMA decode path (decode_tma.cu): persistent blocks over a flat (sequence, unit, tile) list.
+struct TmaPlan {
+  int U, kpu, vpu;   // query heads, K heads and V heads per unit
+  int box_tok;       // tokens per TMA box
+  int stages, grid, smem;
+  long long slots;   // partial-result slots: grid + batch * units
+};
+bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPlan* plan);
+size_t tma_decode_workspace_bytes(const diffqkv_shape& s, const TmaPlan& plan);
+cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, const TmaPlan& plan,
+                              void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream);
+void set_tma_max_blocks(int n);
 
 }  // namespace diffqkv

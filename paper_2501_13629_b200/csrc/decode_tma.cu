@@ -1,0 +1,655 @@
+// DiffQKV split-sequence decode for bf16 caches on sm_100a: TMA-fed shared-memory ring, warp-level
+// tensor-core scoring, probabilities reused across the group's V heads.
+//
+// Work decomposition.  Query heads are handled in "units": U = n_q / min(n_k, n_v) consecutive query
+// heads that share K heads and V heads among themselves only (Eq. (idx) of the paper makes the head
+// maps contiguous blocks).  A unit holds KPU = n_k / min K heads and VPU = n_v / min V heads, one of
+// the two being 1.  The sequence axis is cut into tiles of 64 tokens.  All (sequence, unit, tile)
+// triples, in that order, form one flat list that is divided evenly over the persistent blocks of
+// the grid; a maximal run of one block's tiles inside one (sequence, unit) is a segment and yields
+// one partial result (or the final result when the segment covers the whole sequence).
+//
+// Per block: one producer warp issues TMA loads of the K tile(s) and V tile(s) of each 64-token tile
+// into a ring of stages (128-byte swizzle, completion counted on an mbarrier per stage); four
+// consumer warps each own 16 tokens of a tile:
+//   S^T[16 tok x 8 heads] = K[16 tok x d] . Q^T        mma.sync m16n8k16, K rows via ldmatrix
+//   online softmax over tokens per head column         warp shuffles across the 8 row groups
+//   O^T[d x 8 heads] += V^T[d x 16 tok] . P^T          V via ldmatrix.trans, P^T via movmatrix
+// so every K and V byte is read from shared memory exactly once and scored against all query
+// heads of its unit.  Accumulation is fp32; P is rounded to bf16 for the second product and the
+// softmax denominator sums the rounded values.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace diffqkv {
+namespace {
+
+constexpr int kTT = 64;             // tokens per tile
+constexpr int kConsumerWarps = 4;   // 16 tokens each
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kSubTileBytes = kTT * 128;  // 64 rows of 128 bytes (64 bf16 channels), swizzled
+constexpr int kHeadsPerMma = 8;
+constexpr int kMaxBatchTma = 2048;  // the per-sequence tile prefix lives in shared memory
+int g_max_blocks = 0;               // tuning / test hook: 0 = one block per SM
+
+struct TmaParams {
+  const __nv_bfloat16* q;
+  const int* seqlens;
+  const int* page_table;
+  int page_size, max_pages_per_seq, num_blocks, max_seqlen;
+  int batch, n_q, n_units, U;
+  int hk_per_unit, hv_per_unit;  // KPU, VPU
+  int box_tok;                   // tokens per TMA box (64, or the page size when smaller)
+  int stages;
+  float scale_log2;
+  float* o_partial;    // [slots][U][d_v] normalised partial outputs
+  float* lse_partial;  // [slots][U] base-2 log-sum-exp of the scaled scores
+  int* meta;           // [batch + 1] exclusive prefix of tiles per sequence
+  void* out;
+  float* lse;
+  int out_is_f32;
+  int* dev_status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+// Position in the flat (sequence, unit, tile) list.
+struct Walker {
+  long long g;  // flat tile index
+  int b, u, t, nt;
+  __device__ void seek(long long g0, const int* prefix, int batch, int n_units) {
+    g = g0;
+    int lo = 0, hi = batch;  // smallest b' with n_units * prefix[b'] > g; answer b = b' - 1
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if ((long long)n_units * prefix[mid] > g0) hi = mid; else lo = mid + 1;
+    }
+    b = lo - 1;
+    nt = prefix[b + 1] - prefix[b];
+    const long long rem = g0 - (long long)n_units * prefix[b];
+    u = (int)(rem / nt);
+    t = (int)(rem % nt);
+  }
+  __device__ void next_sequence(const int* prefix, int batch) {
+    do {
+      ++b;
+      nt = b < batch ? prefix[b + 1] - prefix[b] : 1;
+    } while (b < batch && nt == 0);
+  }
+};
+
+template <int D_QK, int D_V, int KPU, int VPU>
+__global__ void __launch_bounds__(kThreads, 1)
+decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+                  const TmaParams p) {
+  constexpr int K_SUB = KPU * (D_QK / 64);  // 8 KB sub-tiles of K per stage
+  constexpr int V_SUB = VPU * (D_V / 64);
+  constexpr int STAGE_BYTES = (K_SUB + V_SUB) * kSubTileBytes;
+  constexpr int KS = D_QK / 16;  // k-steps of the score product
+  constexpr int MT = D_V / 16;   // 16-channel blocks of the output
+  constexpr int OROW = D_V + 4;  // padded row of the merge buffer (bank-conflict free)
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* stage_base = smem;
+  float* obuf = reinterpret_cast<float*>(smem + (size_t)p.stages * STAGE_BYTES);  // [warps][8][OROW]
+  float* mbuf = obuf + kConsumerWarps * kHeadsPerMma * OROW;                      // [warps][8]
+  float* lbuf = mbuf + kConsumerWarps * kHeadsPerMma;                             // [warps][8]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(lbuf + kConsumerWarps * kHeadsPerMma);  // full[s], empty[s]
+  volatile int* abort_flag = reinterpret_cast<int*>(bars + 2 * p.stages);         // set when a wait ran out
+  int* prefix = const_cast<int*>(abort_flag) + 2;                                 // [batch + 1]
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t full0 = ptx::smem_u32(bars), empty0 = ptx::smem_u32(bars + p.stages);
+
+  if (tid == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < p.stages; ++s) {
+      ptx::mbar_init(full0 + 8 * s, 1);
+      ptx::mbar_init(empty0 + 8 * s, kConsumerWarps);
+    }
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmap_k);
+    ptx::prefetch_tmap(&tmap_v);
+  }
+  // exclusive prefix of tiles per sequence (warp 0: per-lane chunks, then a warp scan)
+  if (warp == 0) {
+    const int per = (p.batch + 31) / 32;
+    const int lo = lane * per, hi = min(p.batch, lo + per);
+    int sum = 0;
+    for (int b = lo; b < hi; ++b) sum += (min(max(p.seqlens[b], 0), p.max_seqlen) + kTT - 1) / kTT;
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    int run = incl - sum;
+    for (int b = lo; b < hi; ++b) {
+      prefix[b] = run;
+      run += (min(max(p.seqlens[b], 0), p.max_seqlen) + kTT - 1) / kTT;
+    }
+    if (lane == 31) prefix[p.batch] = incl;
+  }
+  __syncthreads();
+  if (blockIdx.x == 0)
+    for (int b = tid; b <= p.batch; b += kThreads) p.meta[b] = prefix[b];
+
+  const long long total = (long long)p.n_units * prefix[p.batch];
+  // Only min(grid, total) blocks take part, so that every participating block owns at least one tile
+  // (the combine kernel relies on the blocks between a row's first and last owner all having written).
+  const long long nblk = min((long long)gridDim.x, total);
+  if (blockIdx.x >= nblk) return;
+  const long long g_begin = (total * blockIdx.x) / nblk;
+  const long long g_end = (total * (blockIdx.x + 1)) / nblk;
+
+  Walker w;
+  w.seek(g_begin, prefix, p.batch, p.n_units);
+
+  if (warp == kConsumerWarps) {
+    // ------------------------------------------------------------------ producer warp
+    const int parts = kTT / p.box_tok;  // TMA boxes along the token axis per sub-tile
+    const int boxes = (K_SUB + V_SUB) * parts;
+    const uint32_t box_bytes = (uint32_t)p.box_tok * 128u;
+    int stage = 0;
+    uint32_t phase = 0;
+    int issued = 0;
+    bool ok = true;
+    for (; w.g < g_end && ok; ++w.g) {
+      if (issued >= p.stages) {
+        if (!ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) {
+          report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+          ok = false;
+          break;
+        }
+      }
+      const int len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
+      const int tok0 = w.t * kTT;
+      const int parts_valid = min(parts, (len - tok0 + p.box_tok - 1) / p.box_tok);
+      const uint32_t dst0 = ptx::smem_u32(stage_base + (size_t)stage * STAGE_BYTES);
+      const uint32_t bar = full0 + 8 * stage;
+      if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)((K_SUB + V_SUB) * parts_valid) * box_bytes);
+      __syncwarp();
+      for (int x = lane; x < boxes; x += 32) {
+        const int sub = x / parts, part = x % parts;
+        if (part >= parts_valid) continue;
+        const int tok = tok0 + part * p.box_tok;
+        int blk = w.b, slot = tok;
+        if (p.page_table) {
+          blk = p.page_table[(long long)w.b * p.max_pages_per_seq + tok / p.page_size];
+          slot = tok % p.page_size;
+          if (blk < 0 || blk >= p.num_blocks) {  // never read outside the pool: flag it, read page 0 instead
+            report(p.dev_status, DIFFQKV_ERR_INDEX);
+            blk = 0;
+          }
+        }
+        const uint32_t dst = dst0 + sub * kSubTileBytes + part * box_bytes;
+        if (sub < K_SUB) {
+          const int head = w.u * KPU + sub / (D_QK / 64);
+          ptx::tma_load_4d(dst, &tmap_k, bar, (sub % (D_QK / 64)) * 64, slot, head, blk);
+        } else {
+          const int sv = sub - K_SUB;
+          const int head = w.u * VPU + sv / (D_V / 64);
+          ptx::tma_load_4d(dst, &tmap_v, bar, (sv % (D_V / 64)) * 64, slot, head, blk);
+        }
+      }
+      ++issued;
+      if (++stage == p.stages) { stage = 0; phase ^= 1; }
+      if (++w.t == w.nt) {
+        w.t = 0;
+        if (++w.u == p.n_units) { w.u = 0; w.next_sequence(prefix, p.batch); }
+      }
+    }
+    if (!ok) {
+      // Give copies already in flight a bounded chance to land before the block's shared memory is released.
+      for (int s = 0; s < min(issued, p.stages); ++s) {
+        const int uses = (issued - s + p.stages - 1) / p.stages;
+        ptx::mbar_wait(full0 + 8 * s, (uint32_t)(uses - 1) & 1u, nullptr);
+      }
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- consumer warps
+  const int g8 = lane >> 2, t4 = lane & 3;  // row group and column pair of the mma fragments
+  const int heads_per_k = p.U / KPU, heads_per_v = p.U / VPU;
+  const int row0 = warp * 16;  // this warp's token rows inside a tile
+  int stage = 0;
+  uint32_t phase = 0;
+  bool dead = false;
+
+  while (w.g < g_end) {
+    // ---- one segment: tiles [w.t, w.t + seg_tiles) of (sequence w.b, unit w.u)
+    const int seg_tiles = (int)min((long long)(w.nt - w.t), g_end - w.g);
+    const bool whole = (w.t == 0 && seg_tiles == w.nt);
+    const int len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
+    const long long wlin = (long long)w.b * p.n_units + w.u;
+
+    // Q^T fragments (B operand): column g8 = head g8 of the unit, masked per K head of the unit
+    uint32_t qf[KPU][KS][2];
+    {
+      const bool head_ok = g8 < p.U;
+      const __nv_bfloat16* qrow = p.q + ((long long)w.b * p.n_q + (long long)w.u * p.U + (head_ok ? g8 : 0)) * D_QK;
+#pragma unroll
+      for (int i = 0; i < KPU; ++i) {
+        const bool use = head_ok && (g8 / heads_per_k == i);
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+          qf[i][ks][0] = use ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t4) : 0u;
+          qf[i][ks][1] = use ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t4 + 8) : 0u;
+        }
+      }
+    }
+    float m_run[2] = {-INFINITY, -INFINITY};
+    float l_run[2] = {0.f, 0.f};
+    float acc[VPU][MT][4];
+#pragma unroll
+    for (int j = 0; j < VPU; ++j)
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[j][mt][e] = 0.f;
+
+    for (int it = 0; it < seg_tiles; ++it) {
+      // A wait that runs out marks the block dead: the warp stops waiting and computing but keeps
+      // walking, so that it still meets the other warps at the named barriers below.
+      if (!dead && !ptx::mbar_wait(full0 + 8 * stage, phase, abort_flag)) {
+        report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+        dead = true;
+      }
+      const int n_valid = dead ? 0 : min(kTT, len - (w.t + it) * kTT);
+      unsigned char* st = stage_base + (size_t)stage * STAGE_BYTES;
+      const uint32_t st_u32 = ptx::smem_u32(st);
+      if (row0 < n_valid) {
+        if (row0 + 16 > n_valid) {
+          // ragged tail: rows past the sequence end hold whatever followed in memory; zero the V rows
+          // (0 * NaN would poison the product) -- the scores of those rows are masked below.
+          for (int x = lane; x < V_SUB * 16 * 8; x += 32) {
+            const int sub = x / 128, r = (x % 128) / 8, c = x % 8;
+            if (row0 + r >= n_valid)
+              *reinterpret_cast<uint4*>(st + (K_SUB + sub) * kSubTileBytes + (row0 + r) * 128 + c * 16) =
+                  make_uint4(0, 0, 0, 0);
+          }
+          __syncwarp();
+        }
+        // ---- scores S^T = K . Q^T (two accumulators to shorten the dependent mma chain)
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+          const int r = row0 + (lane & 7) + 8 * ((lane >> 3) & 1);
+          const int csel = lane >> 4;
+#pragma unroll
+          for (int i = 0; i < KPU; ++i) {
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+              const int sub = i * (D_QK / 64) + ks / 4;
+              const int chunk = (ks % 4) * 2 + csel;
+              uint32_t a[4];
+              ptx::ldmatrix_x4(st_u32 + sub * kSubTileBytes + r * 128 + ((chunk ^ (r & 7)) << 4), a);
+              if (ks & 1) ptx::mma_bf16_16816(s1, a, qf[i][ks][0], qf[i][ks][1]);
+              else ptx::mma_bf16_16816(s0, a, qf[i][ks][0], qf[i][ks][1]);
+            }
+          }
+        }
+        // ---- online softmax; thread holds rows g8, g8+8 and head columns 2*t4, 2*t4+1
+        const bool v0 = row0 + g8 < n_valid, v1 = row0 + g8 + 8 < n_valid;
+        float x[4];
+        x[0] = v0 ? (s0[0] + s1[0]) * p.scale_log2 : -INFINITY;
+        x[1] = v0 ? (s0[1] + s1[1]) * p.scale_log2 : -INFINITY;
+        x[2] = v1 ? (s0[2] + s1[2]) * p.scale_log2 : -INFINITY;
+        x[3] = v1 ? (s0[3] + s1[3]) * p.scale_log2 : -INFINITY;
+        float mx[2] = {fmaxf(x[0], x[2]), fmaxf(x[1], x[3])};
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+          mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], o));
+          mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], o));
+        }
+        float alpha[2];
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const float m_new = fmaxf(m_run[c], mx[c]);  // finite: row0 < n_valid means a visible token
+          alpha[c] = exp2f(m_run[c] - m_new);
+          m_run[c] = m_new;
+        }
+        const uint32_t p_lo = pack_bf16(exp2f(x[0] - m_run[0]), exp2f(x[1] - m_run[1]));
+        const uint32_t p_hi = pack_bf16(exp2f(x[2] - m_run[0]), exp2f(x[3] - m_run[1]));
+        l_run[0] = l_run[0] * alpha[0] + bf16_lo(p_lo) + bf16_lo(p_hi);
+        l_run[1] = l_run[1] * alpha[1] + bf16_hi(p_lo) + bf16_hi(p_hi);
+        if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
+#pragma unroll
+          for (int j = 0; j < VPU; ++j)
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+              acc[j][mt][0] *= alpha[0]; acc[j][mt][1] *= alpha[1];
+              acc[j][mt][2] *= alpha[0]; acc[j][mt][3] *= alpha[1];
+            }
+        }
+        const uint32_t b0 = ptx::movmatrix_trans(p_lo);  // P^T: tokens 2*t4, 2*t4+1 of head g8
+        const uint32_t b1 = ptx::movmatrix_trans(p_hi);  //      tokens 2*t4+8, 2*t4+9
+        // ---- O^T += V^T . P^T for every V head of the unit
+        {
+          const int r = row0 + (lane & 7) + 8 * (lane >> 4);
+          const int csel = (lane >> 3) & 1;
+#pragma unroll
+          for (int j = 0; j < VPU; ++j) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+              const int sub = K_SUB + j * (D_V / 64) + mt / 4;
+              const int chunk = (mt % 4) * 2 + csel;
+              uint32_t a[4];
+              ptx::ldmatrix_x4_trans(st_u32 + sub * kSubTileBytes + r * 128 + ((chunk ^ (r & 7)) << 4), a);
+              ptx::mma_bf16_16816(acc[j][mt], a, b0, b1);
+            }
+          }
+        }
+        if (row0 + 16 > n_valid) ptx::fence_proxy_async();  // the zero fill above vs. the next TMA write
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(empty0 + 8 * stage);
+      if (++stage == p.stages) { stage = 0; phase ^= 1; }
+    }
+
+    // ---- merge the four warps' (m, l, O) and write the segment's result
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+      l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], o);
+      l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], o);
+    }
+    if (g8 == 0) {
+      mbuf[warp * kHeadsPerMma + 2 * t4] = m_run[0];
+      mbuf[warp * kHeadsPerMma + 2 * t4 + 1] = m_run[1];
+      lbuf[warp * kHeadsPerMma + 2 * t4] = l_run[0];
+      lbuf[warp * kHeadsPerMma + 2 * t4 + 1] = l_run[1];
+    }
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const int col = 2 * t4 + c;
+      if (col < p.U) {
+        const int jv = col / heads_per_v;
+        float* orow = obuf + (warp * kHeadsPerMma + col) * OROW;
+#pragma unroll
+        for (int j = 0; j < VPU; ++j) {
+          if (j == jv) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+              orow[mt * 16 + g8] = acc[j][mt][c];
+              orow[mt * 16 + g8 + 8] = acc[j][mt][2 + c];
+            }
+          }
+        }
+      }
+    }
+    ptx::named_barrier_sync(1, kConsumerWarps * 32);
+    {
+      constexpr int TPH = (kConsumerWarps * 32) / kHeadsPerMma;  // 16 threads per head
+      constexpr int CPT = D_V / TPH;                             // channels per thread
+      const int col = tid / TPH, ch0 = (tid % TPH) * CPT;
+      if (col < p.U) {
+        float mw[kConsumerWarps], M = -INFINITY;
+#pragma unroll
+        for (int ww = 0; ww < kConsumerWarps; ++ww) {
+          mw[ww] = mbuf[ww * kHeadsPerMma + col];
+          M = fmaxf(M, mw[ww]);
+        }
+        float L = 0.f, o[CPT];
+#pragma unroll
+        for (int e = 0; e < CPT; ++e) o[e] = 0.f;
+#pragma unroll
+        for (int ww = 0; ww < kConsumerWarps; ++ww) {
+          const float wgt = mw[ww] == -INFINITY ? 0.f : exp2f(mw[ww] - M);
+          L += wgt * lbuf[ww * kHeadsPerMma + col];
+          if (wgt != 0.f) {
+            const float* src = obuf + (ww * kHeadsPerMma + col) * OROW + ch0;
+#pragma unroll
+            for (int e = 0; e < CPT; ++e) o[e] = fmaf(wgt, src[e], o[e]);
+          }
+        }
+        const float inv = 1.f / L;
+        const float lse2 = M + log2f(L);
+        if (whole) {
+          const long long orow = ((long long)w.b * p.n_q + (long long)w.u * p.U + col) * D_V + ch0;
+          if (p.out_is_f32) {
+            float* dst = reinterpret_cast<float*>(p.out) + orow;
+#pragma unroll
+            for (int e = 0; e < CPT; ++e) dst[e] = o[e] * inv;
+          } else {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + orow;
+#pragma unroll
+            for (int e = 0; e < CPT; ++e) dst[e] = __float2bfloat16_rn(o[e] * inv);
+          }
+          if (p.lse && ch0 == 0) p.lse[(long long)w.b * p.n_q + (long long)w.u * p.U + col] = lse2 * kLn2;
+        } else {
+          const long long slot = blockIdx.x + wlin;
+          float* dst = p.o_partial + (slot * p.U + col) * D_V + ch0;
+#pragma unroll
+          for (int e = 0; e < CPT; ++e) dst[e] = o[e] * inv;
+          if (ch0 == 0) p.lse_partial[slot * p.U + col] = lse2;
+        }
+      }
+    }
+    ptx::named_barrier_sync(1, kConsumerWarps * 32);
+
+    // advance to the next (sequence, unit)
+    w.g += seg_tiles;
+    w.t += seg_tiles;
+    if (w.t == w.nt) {
+      w.t = 0;
+      if (++w.u == p.n_units) { w.u = 0; w.next_sequence(prefix, p.batch); }
+    }
+  }
+}
+
+// Merge of the segment partials written above.  One warp per output row (sequence, query head).
+// A row whose sequence fits inside one block was already written in final form by the decode kernel.
+__global__ void __launch_bounds__(128)
+combine_segments_kernel(const float* __restrict__ o_partial, const float* __restrict__ lse_partial,
+                        const int* __restrict__ meta, int batch, int n_q, int n_units, int U, int d_v, int grid_decode,
+                        void* __restrict__ out, float* __restrict__ lse, int out_is_f32) {
+  const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (row >= (long long)batch * n_q) return;
+  const int lane = threadIdx.x & 31;
+  const int b = (int)(row / n_q), h = (int)(row % n_q);
+  const int u = h / U, col = h % U;
+  const int nt = meta[b + 1] - meta[b];
+  const long long total = (long long)n_units * meta[batch];
+  long long first = 0, last = -1;
+  if (nt > 0) {
+    const long long base = (long long)n_units * meta[b] + (long long)u * nt;
+    const long long nblk = min((long long)grid_decode, total);  // blocks that took part
+    first = ((base + 1) * nblk - 1) / total;  // block that owns flat tile `base`
+    last = ((base + nt) * nblk - 1) / total;
+    if (first == last) return;  // single segment: final result already in place
+  }
+  const long long wlin = (long long)b * n_units + u;
+  float M = -INFINITY;
+  for (long long c = first + lane; c <= last; c += 32) M = fmaxf(M, lse_partial[(c + wlin) * U + col]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  float L = 0.f;
+  for (long long c = first + lane; c <= last; c += 32) L += exp2f(lse_partial[(c + wlin) * U + col] - M);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+  const float inv = nt > 0 ? 1.f / L : 0.f;
+  for (int ch = lane; ch < d_v; ch += 32) {
+    float a = 0.f;
+    for (long long c = first; c <= last; ++c) {
+      const float wgt = exp2f(lse_partial[(c + wlin) * U + col] - M);
+      a = fmaf(wgt, o_partial[((c + wlin) * U + col) * d_v + ch], a);
+    }
+    if (out_is_f32) reinterpret_cast<float*>(out)[row * d_v + ch] = a * inv;
+    else reinterpret_cast<__nv_bfloat16*>(out)[row * d_v + ch] = __float2bfloat16_rn(a * inv);
+  }
+  if (lse && lane == 0) lse[row] = nt > 0 ? (M + log2f(L)) * kLn2 : -INFINITY;
+}
+
+// ---------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      ptr = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(ptr);
+  }();
+  return fn;
+}
+
+// Tensor map over one cache pool: dims (channel, token slot, head, block), box 64 channels x box_tok tokens.
+bool make_pool_map(CUtensorMap* map, const void* base, int d, long long tok_extent, int heads, long long blocks,
+                   long long st_tok, long long st_head, long long st_blk, int box_tok) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)tok_extent, (cuuint64_t)heads, (cuuint64_t)blocks};
+  const cuuint64_t strides[3] = {(cuuint64_t)st_tok * 2, (cuuint64_t)st_head * 2, (cuuint64_t)st_blk * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)box_tok, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  for (int i = 0; i < 3; ++i)
+    if (strides[i] == 0 || strides[i] % 16 != 0 || strides[i] >= (1ull << 40)) return false;
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct DeviceInfo {
+  int sms = 0;
+  int max_smem = 0;
+};
+DeviceInfo device_info() {
+  static std::mutex mu;
+  static DeviceInfo info[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DeviceInfo();
+  std::lock_guard<std::mutex> lock(mu);
+  if (info[dev].sms == 0) {
+    cudaDeviceGetAttribute(&info[dev].sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&info[dev].max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  }
+  return info[dev];
+}
+
+using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const TmaParams);
+struct Variant {
+  KernelFn fn;
+  int stage_bytes;
+  int d_v;
+};
+
+template <int D_QK, int D_V, int KPU, int VPU>
+Variant variant() {
+  return Variant{decode_tma_kernel<D_QK, D_V, KPU, VPU>, (KPU * (D_QK / 64) + VPU * (D_V / 64)) * kSubTileBytes, D_V};
+}
+
+bool pick_variant(int d_qk, int d_v, int kpu, int vpu, Variant* v) {
+#define DIFFQKV_CASE(DQ, DV, KP, VP) \
+  if (d_qk == DQ && d_v == DV && kpu == KP && vpu == VP) { *v = variant<DQ, DV, KP, VP>(); return true; }
+  DIFFQKV_CASE(128, 128, 1, 1) DIFFQKV_CASE(128, 128, 1, 2) DIFFQKV_CASE(128, 128, 1, 4)
+  DIFFQKV_CASE(128, 128, 2, 1) DIFFQKV_CASE(128, 128, 4, 1)
+  DIFFQKV_CASE(64, 64, 1, 1) DIFFQKV_CASE(64, 64, 1, 2) DIFFQKV_CASE(64, 64, 1, 4)
+  DIFFQKV_CASE(64, 64, 2, 1) DIFFQKV_CASE(64, 64, 4, 1)
+  DIFFQKV_CASE(64, 128, 1, 1) DIFFQKV_CASE(64, 128, 1, 2)
+#undef DIFFQKV_CASE
+  return false;
+}
+
+}  // namespace
+
+bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPlan* plan) {
+  if (s.dtype != DIFFQKV_BF16) return false;
+  const int mn = s.n_k < s.n_v ? s.n_k : s.n_v;
+  if (s.n_k % mn != 0 || s.n_v % mn != 0) return false;
+  const int U = s.n_q / mn, kpu = s.n_k / mn, vpu = s.n_v / mn;
+  if (U > kHeadsPerMma || s.batch > kMaxBatchTma || s.batch < 1) return false;
+  Variant v;
+  if (!pick_variant(s.d_qk, s.d_v, kpu, vpu, &v)) return false;
+  int box_tok = kTT;
+  if (c.page_table) {
+    if (c.page_size % 16 != 0) return false;
+    if (c.page_size < kTT) { if (kTT % c.page_size != 0) return false; box_tok = c.page_size; }
+    else if (c.page_size % kTT != 0) return false;
+  }
+  const DeviceInfo di = device_info();
+  if (di.sms <= 0) return false;
+  const int fixed = 1024 + kConsumerWarps * kHeadsPerMma * (s.d_v + 4 + 2) * 4 + 2 * 16 * 8 + (s.batch + 1) * 4 + 64;
+  int stages = (di.max_smem - fixed) / v.stage_bytes;
+  if (stages > 8) stages = 8;
+  if (stages < 2) return false;
+  const long long tiles_max = (long long)s.batch * (s.n_q / U) * ((c.max_seqlen + kTT - 1) / kTT);
+  long long grid = di.sms;
+  if (g_max_blocks > 0 && grid > g_max_blocks) grid = g_max_blocks;
+  if (grid > tiles_max) grid = tiles_max;
+  if (grid < 1) grid = 1;
+  plan->U = U; plan->kpu = kpu; plan->vpu = vpu; plan->box_tok = box_tok; plan->stages = stages;
+  plan->grid = (int)grid;
+  plan->smem = fixed + stages * v.stage_bytes;
+  plan->slots = grid + (long long)s.batch * (s.n_q / U);
+  return true;
+}
+
+void set_tma_max_blocks(int n) { g_max_blocks = n > 0 ? n : 0; }
+
+size_t tma_decode_workspace_bytes(const diffqkv_shape& s, const TmaPlan& plan) {
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  return up((size_t)plan.slots * plan.U * s.d_v * 4) + up((size_t)plan.slots * plan.U * 4) + up((size_t)(s.batch + 1) * 4);
+}
+
+// Returns cudaErrorNotSupported when no tensor map can describe the cache (the caller then falls back to
+// the generic kernel); any other error is a real launch failure.
+cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, const TmaPlan& plan,
+                              void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream) {
+  Variant v;
+  if (!pick_variant(s.d_qk, s.d_v, plan.kpu, plan.vpu, &v)) return cudaErrorNotSupported;
+  CUtensorMap mk, mv;
+  const long long tok_extent = c.page_table ? c.page_size : c.max_seqlen;
+  if (!make_pool_map(&mk, c.k_cache, s.d_qk, tok_extent, s.n_k, c.num_blocks, c.k_stride_tok, c.k_stride_head,
+                     c.k_stride_blk, plan.box_tok) ||
+      !make_pool_map(&mv, c.v_cache, s.d_v, tok_extent, s.n_v, c.num_blocks, c.v_stride_tok, c.v_stride_head,
+                     c.v_stride_blk, plan.box_tok))
+    return cudaErrorNotSupported;
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  TmaParams p;
+  p.q = reinterpret_cast<const __nv_bfloat16*>(q);
+  p.seqlens = c.seqlens;
+  p.page_table = c.page_table;
+  p.page_size = c.page_size; p.max_pages_per_seq = c.max_pages_per_seq;
+  p.num_blocks = c.num_blocks; p.max_seqlen = c.max_seqlen;
+  p.batch = s.batch; p.n_q = s.n_q; p.n_units = s.n_q / plan.U; p.U = plan.U;
+  p.hk_per_unit = plan.kpu; p.hv_per_unit = plan.vpu;
+  p.box_tok = plan.box_tok; p.stages = plan.stages;
+  p.scale_log2 = s.scale * kLog2e;
+  char* ws = reinterpret_cast<char*>(workspace);
+  p.o_partial = reinterpret_cast<float*>(ws);
+  ws += up((size_t)plan.slots * plan.U * s.d_v * 4);
+  p.lse_partial = reinterpret_cast<float*>(ws);
+  ws += up((size_t)plan.slots * plan.U * 4);
+  p.meta = reinterpret_cast<int*>(ws);
+  p.out = out; p.lse = lse; p.out_is_f32 = s.out_dtype == DIFFQKV_F32;
+  p.dev_status = dev_status;
+
+  cudaError_t err = cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem);
+  if (err != cudaSuccess) return err;
+  v.fn<<<plan.grid, kThreads, plan.smem, stream>>>(mk, mv, p);
+  count_launch();
+  err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  profile_after_split(stream);
+  const long long rows = (long long)s.batch * s.n_q;
+  combine_segments_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, stream>>>(
+      p.o_partial, p.lse_partial, p.meta, s.batch, s.n_q, p.n_units, plan.U, s.d_v, plan.grid, out, lse, p.out_is_f32);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace diffqkv

@@ -137,9 +137,10 @@ def test_out_of_range_page_is_reported_not_read(api):
     pg = W.paginate(inp, 16, seed=3)
     pg.page_table[1, 3] = pg.num_pages + 5
     pg.page_table[2, 0] = -1
-    out, lse, st = run_decode(api, pg)
-    assert st == (1 << api.ERR_INDEX)
-    assert np.all(np.isfinite(out))
+    for splits in (0, 2):  # TMA kernel and generic kernel
+        out, lse, st = run_decode(api, pg, num_splits=splits)
+        assert st == (1 << api.ERR_INDEX)
+        assert np.all(np.isfinite(out))
 
 
 def test_paged_varlen_config5_shape_reduced(api, oracle):
@@ -151,6 +152,73 @@ def test_paged_varlen_config5_shape_reduced(api, oracle):
     assert st == 0
     check_bf16(out, ref)
     check_lse(lse, lse_ref, 2e-2)
+
+
+@pytest.fixture
+def blocks(api):
+    """Sets the persistent-block cap of the TMA kernel and always restores the default."""
+    yield api.set_max_blocks
+    api.set_max_blocks(0)
+
+
+def test_tma_kernel_is_the_bf16_path(api):
+    inp = W.make_decode_inputs(SMALL)
+    run_decode(api, inp)
+    assert api.last_decode_kernel() == api.KERNEL_TMA
+    run_decode(api, inp, num_splits=3)
+    assert api.last_decode_kernel() == api.KERNEL_GENERIC
+    run_decode(api, W.make_decode_inputs(W.CFG1))
+    assert api.last_decode_kernel() == api.KERNEL_GENERIC  # fp32 mode
+
+
+@pytest.mark.parametrize("heads", [(16, 2, 4), (32, 4, 16), (8, 8, 8), (8, 4, 1), (8, 2, 4)])
+@pytest.mark.parametrize("d", [64, 128])
+def test_tma_block_partition_invariance(api, oracle, blocks, heads, d):
+    """The flat tile list is cut differently for every block count; results agree with the oracle
+    and with each other up to fp32 reassociation."""
+    n_q, n_k, n_v = heads
+    cfg = dataclasses.replace(SMALL, batch=5, n_q=n_q, n_k=n_k, n_v=n_v, d_qk=d, d_v=d, kv_len=1500)
+    inp = W.make_decode_inputs(cfg, seqlens=np.array([1500, 64, 0, 777, 1], dtype=np.int32))
+    ref, lse_ref = run_oracle(oracle, inp)
+    outs = []
+    for nb in (1, 2, 3, 7, 40, 0):
+        blocks(nb)
+        out, lse, st = run_decode(api, inp)
+        assert st == 0 and api.last_decode_kernel() == api.KERNEL_TMA
+        check_bf16(out, ref, f"{heads} d={d} blocks={nb}")
+        check_lse(lse, lse_ref, 2e-2)
+        assert np.all(out[2] == 0) and np.all(np.isneginf(lse[2]))
+        outs.append(out)
+    for o in outs[1:]:
+        assert np.abs(o - outs[0]).max() <= 5e-3
+
+
+@pytest.mark.parametrize("page_size", [16, 32, 64, 128])
+def test_tma_paged_equals_contiguous_bitwise(api, oracle, blocks, page_size):
+    inp = W.make_decode_inputs(dataclasses.replace(SMALL, kv_len=1024), seqlens=np.array([1024, 500, 17], np.int32))
+    ref, _ = run_oracle(oracle, inp)
+    for nb in (0, 5):
+        blocks(nb)
+        base, lse0, st = run_decode(api, inp)
+        assert st == 0 and api.last_decode_kernel() == api.KERNEL_TMA
+        check_bf16(base, ref)
+        for identity in (True, False):
+            pg = W.paginate(inp, page_size, seed=9, identity=identity)
+            out, lse, st = run_decode(api, pg)
+            assert st == 0 and api.last_decode_kernel() == api.KERNEL_TMA
+            assert np.array_equal(out, base) and np.array_equal(lse, lse0)
+
+
+def test_tma_tail_rows_with_nan_garbage(api, oracle):
+    """Cache rows past a sequence's end may hold anything, NaN bit patterns included."""
+    inp = W.make_decode_inputs(SMALL, seqlens=np.array([700, 333, 5], np.int32))
+    for b, n in enumerate([700, 333, 5]):
+        inp.k[b, :, n:] = 0x7FC0  # bf16 NaN
+        inp.v[b, :, n:] = 0x7FC0
+    ref, _ = run_oracle(oracle, inp)
+    out, _, st = run_decode(api, inp)
+    assert st == 0 and api.last_decode_kernel() == api.KERNEL_TMA
+    check_bf16(out, ref)
 
 
 def test_combine_entry_point(api, oracle):
