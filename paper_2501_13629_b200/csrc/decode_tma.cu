@@ -31,7 +31,9 @@ namespace {
 constexpr int kTT = 64;             // tokens per tile
 constexpr int kConsumerWarps = 4;   // 16 tokens each
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kSubTileBytes = kTT * 128;  // 64 rows of 128 bytes (64 bf16 channels), swizzled
+// Shared-memory layout of one head's 64-token tile with D channels: rows of 128 bytes (64 channels,
+// 128-byte swizzle).  One TMA box brings `box_tok` tokens of all D/64 channel halves, so the tile is
+// [token part][channel half][box_tok rows]; with box_tok = 64 that is simply [half][64 rows].
 constexpr int kHeadsPerMma = 8;
 constexpr int kMaxBatchTma = 2048;  // the per-sequence tile prefix lives in shared memory
 int g_max_blocks = 0;               // tuning / test hook: 0 = one block per SM
@@ -91,9 +93,10 @@ template <int D_QK, int D_V, int KPU, int VPU>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                   const TmaParams p) {
-  constexpr int K_SUB = KPU * (D_QK / 64);  // 8 KB sub-tiles of K per stage
-  constexpr int V_SUB = VPU * (D_V / 64);
-  constexpr int STAGE_BYTES = (K_SUB + V_SUB) * kSubTileBytes;
+  constexpr int HK = D_QK / 64, HV = D_V / 64;  // 64-channel halves per row
+  constexpr int K_TILE = kTT * D_QK * 2;        // bytes of one K head tile
+  constexpr int V_TILE = kTT * D_V * 2;
+  constexpr int STAGE_BYTES = KPU * K_TILE + VPU * V_TILE;
   constexpr int KS = D_QK / 16;  // k-steps of the score product
   constexpr int MT = D_V / 16;   // 16-channel blocks of the output
   constexpr int OROW = D_V + 4;  // padded row of the merge buffer (bank-conflict free)
@@ -141,6 +144,9 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     if (lane == 31) prefix[p.batch] = incl;
   }
   __syncthreads();
+  // Let the combine kernel (launched with programmatic stream serialisation) get resident early; it
+  // still waits for this whole grid to finish before it reads any partial.
+  ptx::grid_launch_dependents();
   if (blockIdx.x == 0)
     for (int b = tid; b <= p.batch; b += kThreads) p.meta[b] = prefix[b];
 
@@ -157,14 +163,28 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer warp
-    const int parts = kTT / p.box_tok;  // TMA boxes along the token axis per sub-tile
-    const int boxes = (K_SUB + V_SUB) * parts;
-    const uint32_t box_bytes = (uint32_t)p.box_tok * 128u;
+    // One TMA box per (head tile, token part): lane x < boxes owns box x of every tile.
+    const int parts = kTT / p.box_tok;
+    const int boxes = (KPU + VPU) * parts;
+    const int my_tile = lane / parts, my_part = lane % parts;
+    const bool my_is_k = my_tile < KPU;
+    const uint32_t my_off = my_is_k ? my_tile * K_TILE + my_part * (p.box_tok * 128 * HK)
+                                    : KPU * K_TILE + (my_tile - KPU) * V_TILE + my_part * (p.box_tok * 128 * HV);
+    const uint32_t tile_part_bytes = (uint32_t)p.box_tok * 128u * (KPU * HK + VPU * HV);
     int stage = 0;
     uint32_t phase = 0;
     int issued = 0;
     bool ok = true;
-    for (; w.g < g_end && ok; ++w.g) {
+    int len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
+    // page id of this lane's box for the tile about to be issued (fetched one tile ahead)
+    auto fetch_blk = [&]() -> int {
+      if (!p.page_table) return w.b;
+      const int tok = w.t * kTT + my_part * p.box_tok;
+      if (lane >= boxes || tok >= len) return 0;
+      return p.page_table[(long long)w.b * p.max_pages_per_seq + tok / p.page_size];
+    };
+    int blk = fetch_blk();
+    for (; w.g < g_end; ++w.g) {
       if (issued >= p.stages) {
         if (!ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) {
           report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
@@ -172,42 +192,33 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
           break;
         }
       }
-      const int len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
       const int tok0 = w.t * kTT;
       const int parts_valid = min(parts, (len - tok0 + p.box_tok - 1) / p.box_tok);
-      const uint32_t dst0 = ptx::smem_u32(stage_base + (size_t)stage * STAGE_BYTES);
       const uint32_t bar = full0 + 8 * stage;
-      if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)((K_SUB + V_SUB) * parts_valid) * box_bytes);
+      if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)parts_valid * tile_part_bytes);
       __syncwarp();
-      for (int x = lane; x < boxes; x += 32) {
-        const int sub = x / parts, part = x % parts;
-        if (part >= parts_valid) continue;
-        const int tok = tok0 + part * p.box_tok;
-        int blk = w.b, slot = tok;
-        if (p.page_table) {
-          blk = p.page_table[(long long)w.b * p.max_pages_per_seq + tok / p.page_size];
-          slot = tok % p.page_size;
-          if (blk < 0 || blk >= p.num_blocks) {  // never read outside the pool: flag it, read page 0 instead
-            report(p.dev_status, DIFFQKV_ERR_INDEX);
-            blk = 0;
-          }
+      if (lane < boxes && my_part < parts_valid) {
+        const int tok = tok0 + my_part * p.box_tok;
+        const int slot = p.page_table ? tok % p.page_size : tok;
+        if (blk < 0 || blk >= p.num_blocks) {  // never read outside the pool: flag it, read block 0 instead
+          report(p.dev_status, DIFFQKV_ERR_INDEX);
+          blk = 0;
         }
-        const uint32_t dst = dst0 + sub * kSubTileBytes + part * box_bytes;
-        if (sub < K_SUB) {
-          const int head = w.u * KPU + sub / (D_QK / 64);
-          ptx::tma_load_4d(dst, &tmap_k, bar, (sub % (D_QK / 64)) * 64, slot, head, blk);
-        } else {
-          const int sv = sub - K_SUB;
-          const int head = w.u * VPU + sv / (D_V / 64);
-          ptx::tma_load_4d(dst, &tmap_v, bar, (sv % (D_V / 64)) * 64, slot, head, blk);
-        }
+        const uint32_t dst = ptx::smem_u32(stage_base + (size_t)stage * STAGE_BYTES) + my_off;
+        if (my_is_k) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, 0, w.u * KPU + my_tile, blk);
+        else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, 0, w.u * VPU + (my_tile - KPU), blk);
       }
       ++issued;
       if (++stage == p.stages) { stage = 0; phase ^= 1; }
       if (++w.t == w.nt) {
         w.t = 0;
-        if (++w.u == p.n_units) { w.u = 0; w.next_sequence(prefix, p.batch); }
+        if (++w.u == p.n_units) {
+          w.u = 0;
+          w.next_sequence(prefix, p.batch);
+          if (w.b < p.batch) len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
+        }
       }
+      if (w.g + 1 < g_end) blk = fetch_blk();
     }
     if (!ok) {
       // Give copies already in flight a bounded chance to land before the block's shared memory is released.
@@ -223,6 +234,9 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   const int g8 = lane >> 2, t4 = lane & 3;  // row group and column pair of the mma fragments
   const int heads_per_k = p.U / KPU, heads_per_v = p.U / VPU;
   const int row0 = warp * 16;  // this warp's token rows inside a tile
+  const int bt_shift = 31 - __clz(p.box_tok), bt_mask = p.box_tok - 1;
+  // 128-byte row index of (token row r, channel half h) inside a head tile with H halves
+  auto row_index = [&](int r, int h, int H) { return (((r >> bt_shift) * H + h) << bt_shift) + (r & bt_mask); };
   int stage = 0;
   uint32_t phase = 0;
   bool dead = false;
@@ -273,11 +287,11 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         if (row0 + 16 > n_valid) {
           // ragged tail: rows past the sequence end hold whatever followed in memory; zero the V rows
           // (0 * NaN would poison the product) -- the scores of those rows are masked below.
-          for (int x = lane; x < V_SUB * 16 * 8; x += 32) {
-            const int sub = x / 128, r = (x % 128) / 8, c = x % 8;
-            if (row0 + r >= n_valid)
-              *reinterpret_cast<uint4*>(st + (K_SUB + sub) * kSubTileBytes + (row0 + r) * 128 + c * 16) =
-                  make_uint4(0, 0, 0, 0);
+          for (int x = lane; x < VPU * HV * 16 * 8; x += 32) {
+            const int sub = x / 128, r = row0 + (x % 128) / 8, c = x % 8;
+            if (r >= n_valid)
+              *reinterpret_cast<uint4*>(st + KPU * K_TILE + (sub / HV) * V_TILE + row_index(r, sub % HV, HV) * 128 +
+                                        c * 16) = make_uint4(0, 0, 0, 0);
           }
           __syncwarp();
         }
@@ -286,14 +300,16 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         {
           const int r = row0 + (lane & 7) + 8 * ((lane >> 3) & 1);
           const int csel = lane >> 4;
+          uint32_t rbase[HK];
+#pragma unroll
+          for (int h = 0; h < HK; ++h) rbase[h] = st_u32 + row_index(r, h, HK) * 128;
 #pragma unroll
           for (int i = 0; i < KPU; ++i) {
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
-              const int sub = i * (D_QK / 64) + ks / 4;
               const int chunk = (ks % 4) * 2 + csel;
               uint32_t a[4];
-              ptx::ldmatrix_x4(st_u32 + sub * kSubTileBytes + r * 128 + ((chunk ^ (r & 7)) << 4), a);
+              ptx::ldmatrix_x4(rbase[ks / 4] + i * K_TILE + ((chunk ^ (r & 7)) << 4), a);
               if (ks & 1) ptx::mma_bf16_16816(s1, a, qf[i][ks][0], qf[i][ks][1]);
               else ptx::mma_bf16_16816(s0, a, qf[i][ks][0], qf[i][ks][1]);
             }
@@ -338,14 +354,16 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         {
           const int r = row0 + (lane & 7) + 8 * (lane >> 4);
           const int csel = (lane >> 3) & 1;
+          uint32_t rbase[HV];
+#pragma unroll
+          for (int h = 0; h < HV; ++h) rbase[h] = st_u32 + KPU * K_TILE + row_index(r, h, HV) * 128;
 #pragma unroll
           for (int j = 0; j < VPU; ++j) {
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
-              const int sub = K_SUB + j * (D_V / 64) + mt / 4;
               const int chunk = (mt % 4) * 2 + csel;
               uint32_t a[4];
-              ptx::ldmatrix_x4_trans(st_u32 + sub * kSubTileBytes + r * 128 + ((chunk ^ (r & 7)) << 4), a);
+              ptx::ldmatrix_x4_trans(rbase[mt / 4] + j * V_TILE + ((chunk ^ (r & 7)) << 4), a);
               ptx::mma_bf16_16816(acc[j][mt], a, b0, b1);
             }
           }
@@ -449,45 +467,108 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
 
 // Merge of the segment partials written above.  One warp per output row (sequence, query head).
 // A row whose sequence fits inside one block was already written in final form by the decode kernel.
+// Launched with programmatic stream serialisation: everything before grid_dependency_wait() only
+// touches inputs of the call (seqlens), so it overlaps the decode kernel's tail.
+constexpr int kCombineSmallBatch = 256;
 __global__ void __launch_bounds__(128)
 combine_segments_kernel(const float* __restrict__ o_partial, const float* __restrict__ lse_partial,
-                        const int* __restrict__ meta, int batch, int n_q, int n_units, int U, int d_v, int grid_decode,
-                        void* __restrict__ out, float* __restrict__ lse, int out_is_f32) {
+                        const int* __restrict__ meta, const int* __restrict__ seqlens, int max_seqlen, int batch,
+                        int n_q, int n_units, int U, int d_v, int grid_decode, void* __restrict__ out,
+                        float* __restrict__ lse, int out_is_f32) {
   const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
-  if (row >= (long long)batch * n_q) return;
+  const bool active = row < (long long)batch * n_q;
   const int lane = threadIdx.x & 31;
-  const int b = (int)(row / n_q), h = (int)(row % n_q);
+  const int b = active ? (int)(row / n_q) : 0, h = active ? (int)(row % n_q) : 0;
   const int u = h / U, col = h % U;
-  const int nt = meta[b + 1] - meta[b];
-  const long long total = (long long)n_units * meta[batch];
-  long long first = 0, last = -1;
-  if (nt > 0) {
-    const long long base = (long long)n_units * meta[b] + (long long)u * nt;
-    const long long nblk = min((long long)grid_decode, total);  // blocks that took part
-    first = ((base + 1) * nblk - 1) / total;  // block that owns flat tile `base`
-    last = ((base + nt) * nblk - 1) / total;
-    if (first == last) return;  // single segment: final result already in place
+  int nt = 0;
+  long long before = 0, all = 0;  // tiles of earlier sequences / of all sequences
+  const bool small = batch <= kCombineSmallBatch;
+  if (small) {
+    for (int bb = lane; bb < batch; bb += 32) {
+      const int t = (min(max(seqlens[bb], 0), max_seqlen) + kTT - 1) / kTT;
+      all += t;
+      if (bb < b) before += t;
+      if (bb == b) nt = t;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      all += __shfl_xor_sync(0xffffffffu, all, o);
+      before += __shfl_xor_sync(0xffffffffu, before, o);
+      nt += __shfl_xor_sync(0xffffffffu, nt, o);
+    }
   }
+  ptx::grid_dependency_wait();
+  if (!active) return;
+  if (!small) {
+    nt = meta[b + 1] - meta[b];
+    before = meta[b];
+    all = meta[batch];
+  }
+  const long long total = (long long)n_units * all;
+  float4* out4 = reinterpret_cast<float4*>(out);
+  if (nt == 0) {  // empty sequence: the decode kernel never touched this row
+    for (int ch = lane * 4; ch < d_v; ch += 128) {
+      if (out_is_f32) out4[(row * d_v + ch) >> 2] = make_float4(0.f, 0.f, 0.f, 0.f);
+      else *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + row * d_v + ch) = make_uint2(0u, 0u);
+    }
+    if (lse && lane == 0) lse[row] = -INFINITY;
+    return;
+  }
+  const long long base = (long long)n_units * before + (long long)u * nt;
+  const long long nblk = min((long long)grid_decode, total);  // blocks that took part
+  const long long first = ((base + 1) * nblk - 1) / total;    // block that owns flat tile `base`
+  const long long last = ((base + nt) * nblk - 1) / total;
+  if (first == last) return;  // single segment: final result already in place
   const long long wlin = (long long)b * n_units + u;
+  const int n = (int)(last - first + 1);
+  const float* lp = lse_partial + (first + wlin) * U + col;  // partial c at lp[c * U]
+  const float* op = o_partial + ((first + wlin) * U + col) * d_v;  // partial c at op[c * U * d_v]
   float M = -INFINITY;
-  for (long long c = first + lane; c <= last; c += 32) M = fmaxf(M, lse_partial[(c + wlin) * U + col]);
+  for (int c = lane; c < n; c += 32) M = fmaxf(M, lp[(long long)c * U]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-  float L = 0.f;
-  for (long long c = first + lane; c <= last; c += 32) L += exp2f(lse_partial[(c + wlin) * U + col] - M);
+  float wreg = 0.f, L = 0.f;  // lane c keeps the weight of partial c (first 32 partials)
+  for (int c = lane; c < n; c += 32) {
+    const float e = exp2f(lp[(long long)c * U] - M);
+    if (c < 32) wreg = e;
+    L += e;
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
-  const float inv = nt > 0 ? 1.f / L : 0.f;
-  for (int ch = lane; ch < d_v; ch += 32) {
-    float a = 0.f;
-    for (long long c = first; c <= last; ++c) {
-      const float wgt = exp2f(lse_partial[(c + wlin) * U + col] - M);
-      a = fmaf(wgt, o_partial[((c + wlin) * U + col) * d_v + ch], a);
+  const float inv = 1.f / L;
+  for (int ch0 = 0; ch0 < d_v; ch0 += 128) {  // uniform trip count: the shuffles need all lanes
+    const int ch = ch0 + lane * 4;
+    const bool in = ch < d_v;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int n32 = min(n, 32);
+#pragma unroll 4
+    for (int c = 0; c < n32; ++c) {
+      const float wgt = __shfl_sync(0xffffffffu, wreg, c);
+      if (in) {
+        const float4 v = *reinterpret_cast<const float4*>(op + (long long)c * U * d_v + ch);
+        a.x = fmaf(wgt, v.x, a.x); a.y = fmaf(wgt, v.y, a.y); a.z = fmaf(wgt, v.z, a.z); a.w = fmaf(wgt, v.w, a.w);
+      }
     }
-    if (out_is_f32) reinterpret_cast<float*>(out)[row * d_v + ch] = a * inv;
-    else reinterpret_cast<__nv_bfloat16*>(out)[row * d_v + ch] = __float2bfloat16_rn(a * inv);
+    for (int c = 32; c < n; ++c) {
+      const float wgt = exp2f(lp[(long long)c * U] - M);
+      if (in) {
+        const float4 v = *reinterpret_cast<const float4*>(op + (long long)c * U * d_v + ch);
+        a.x = fmaf(wgt, v.x, a.x); a.y = fmaf(wgt, v.y, a.y); a.z = fmaf(wgt, v.z, a.z); a.w = fmaf(wgt, v.w, a.w);
+      }
+    }
+    if (in) {
+      a.x *= inv; a.y *= inv; a.z *= inv; a.w *= inv;
+      if (out_is_f32) {
+        out4[(row * d_v + ch) >> 2] = a;
+      } else {
+        uint2 pk;
+        pk.x = pack_bf16(a.x, a.y);
+        pk.y = pack_bf16(a.z, a.w);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + row * d_v + ch) = pk;
+      }
+    }
   }
-  if (lse && lane == 0) lse[row] = nt > 0 ? (M + log2f(L)) * kLn2 : -INFINITY;
+  if (lse && lane == 0) lse[row] = (M + log2f(L)) * kLn2;
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -507,18 +588,19 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Tensor map over one cache pool: dims (channel, token slot, head, block), box 64 channels x box_tok tokens.
+// Tensor map over one cache pool: dims (64 channels, token slot, channel half, head, block); one box
+// brings box_tok tokens x all halves of one head, each half landing as 128-byte swizzled rows.
 bool make_pool_map(CUtensorMap* map, const void* base, int d, long long tok_extent, int heads, long long blocks,
                    long long st_tok, long long st_head, long long st_blk, int box_tok) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)tok_extent, (cuuint64_t)heads, (cuuint64_t)blocks};
-  const cuuint64_t strides[3] = {(cuuint64_t)st_tok * 2, (cuuint64_t)st_head * 2, (cuuint64_t)st_blk * 2};
-  const cuuint32_t box[4] = {64, (cuuint32_t)box_tok, 1, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  for (int i = 0; i < 3; ++i)
+  const cuuint64_t dims[5] = {64, (cuuint64_t)tok_extent, (cuuint64_t)(d / 64), (cuuint64_t)heads, (cuuint64_t)blocks};
+  const cuuint64_t strides[4] = {(cuuint64_t)st_tok * 2, 128, (cuuint64_t)st_head * 2, (cuuint64_t)st_blk * 2};
+  const cuuint32_t box[5] = {64, (cuuint32_t)box_tok, (cuuint32_t)(d / 64), 1, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  for (int i = 0; i < 4; ++i)
     if (strides[i] == 0 || strides[i] % 16 != 0 || strides[i] >= (1ull << 40)) return false;
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -549,7 +631,7 @@ struct Variant {
 
 template <int D_QK, int D_V, int KPU, int VPU>
 Variant variant() {
-  return Variant{decode_tma_kernel<D_QK, D_V, KPU, VPU>, (KPU * (D_QK / 64) + VPU * (D_V / 64)) * kSubTileBytes, D_V};
+  return Variant{decode_tma_kernel<D_QK, D_V, KPU, VPU>, kTT * 2 * (KPU * D_QK + VPU * D_V), D_V};
 }
 
 bool pick_variant(int d_qk, int d_v, int kpu, int vpu, Variant* v) {
@@ -646,8 +728,20 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
   if (err != cudaSuccess) return err;
   profile_after_split(stream);
   const long long rows = (long long)s.batch * s.n_q;
-  combine_segments_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, stream>>>(
-      p.o_partial, p.lse_partial, p.meta, s.batch, s.n_q, p.n_units, plan.U, s.d_v, plan.grid, out, lse, p.out_is_f32);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((rows + 3) / 4));
+  cfg.blockDim = dim3(128);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  err = cudaLaunchKernelEx(&cfg, combine_segments_kernel, (const float*)p.o_partial, (const float*)p.lse_partial,
+                           (const int*)p.meta, c.seqlens, c.max_seqlen, s.batch, s.n_q, p.n_units, plan.U, s.d_v,
+                           plan.grid, out, lse, p.out_is_f32);
+  if (err != cudaSuccess) return err;
   count_launch();
   return cudaGetLastError();
 }
