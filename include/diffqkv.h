@@ -183,14 +183,17 @@ diffqkv_status diffqkv_prefill(const void *q, const void *k_new, const void *v_n
  * act is read as SiLU, there are no biases, and weights use the nn.Linear layout [out, in]:
  *     x = h W_Q^T,   a = silu(x W_gate^T) * (x W_up^T),   q = a W_down^T
  *   h [T, d_model]   W_Q [d_q0, d_model]   W_gate, W_up [d_aug, d_q0]   W_down [d_out, d_aug]   all bf16
- *   workspace  diffqkv_augq_workspace_bytes(T, d_q0, d_aug) bytes for x and a (bf16)
+ *   workspace  diffqkv_augq_workspace_bytes(T, d_q0, d_aug) bytes, 256-byte aligned, for x and a
  *   q_out [T, d_out] bf16
- * All dimensions must be multiples of 128 except T.
+ *   dev_status as in diffqkv_decode, or NULL
+ * Products accumulate in fp32 on the tensor cores; x and a are rounded to bf16 once each (they are the next
+ * product's bf16 operands).  All dimensions must be multiples of 128 except T; T == 0 does nothing.
  */
 size_t diffqkv_augq_workspace_bytes(int64_t T, int32_t d_q0, int32_t d_aug);
 diffqkv_status diffqkv_augq(const void *h, const void *W_Q, const void *W_gate, const void *W_up,
                             const void *W_down, int64_t T, int32_t d_model, int32_t d_q0, int32_t d_aug,
-                            int32_t d_out, void *workspace, size_t workspace_bytes, void *q_out, void *stream);
+                            int32_t d_out, void *workspace, size_t workspace_bytes, void *q_out,
+                            int32_t *dev_status, void *stream);
 
 /* Static, never-null description of a status value. */
 const char *diffqkv_status_string(diffqkv_status status);

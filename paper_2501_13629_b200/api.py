@@ -74,7 +74,7 @@ _lib.diffqkv_augq_workspace_bytes.restype = C.c_size_t
 _lib.diffqkv_augq_workspace_bytes.argtypes = [C.c_int64, C.c_int32, C.c_int32]
 _lib.diffqkv_augq.restype = C.c_int
 _lib.diffqkv_augq.argtypes = [C.c_void_p] * 5 + [C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
-                                                 C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+                                                 C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.diffqkv_status_string.restype = C.c_char_p
 _lib.diffqkv_status_string.argtypes = [C.c_int]
 _lib.diffqkv_launch_count.restype = C.c_int64
@@ -277,7 +277,7 @@ def diffqkv_augq_workspace_bytes(T: int, d_q0: int, d_aug: int) -> int:
 
 def diffqkv_augq(h: torch.Tensor, W_Q: torch.Tensor, W_gate: torch.Tensor, W_up: torch.Tensor,
                  W_down: torch.Tensor, workspace: Optional[torch.Tensor] = None,
-                 q_out: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+                 q_out: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
     """h [T, d_model] bf16, weights in nn.Linear layout [out, in]; returns q [T, d_out] bf16."""
     T, d_model = h.shape
     d_q0, d_aug, d_out = W_Q.shape[0], W_gate.shape[0], W_down.shape[0]
@@ -287,7 +287,7 @@ def diffqkv_augq(h: torch.Tensor, W_Q: torch.Tensor, W_gate: torch.Tensor, W_up:
     if q_out is None:
         q_out = torch.empty((T, d_out), dtype=torch.bfloat16, device=h.device)
     st = _lib.diffqkv_augq(_p(h), _p(W_Q), _p(W_gate), _p(W_up), _p(W_down), T, d_model, d_q0, d_aug, d_out,
-                           _p(workspace), workspace.numel(), _p(q_out), _stream_ptr(stream))
+                           _p(workspace), workspace.numel(), _p(q_out), _p(dev_status), _stream_ptr(stream))
     if st != OK:
         raise DiffQKVError(st, "diffqkv_augq")
     return q_out

@@ -214,12 +214,26 @@ diffqkv_status diffqkv_prefill(const void*, const void*, const void*, int32_t, c
 
 size_t diffqkv_augq_workspace_bytes(int64_t T, int32_t d_q0, int32_t d_aug) {
   if (T < 0 || d_q0 <= 0 || d_aug <= 0) return 0;
-  return align_up((size_t)T * d_q0 * 2, 256) + align_up((size_t)T * d_aug * 2, 256);
+  return augq_workspace_bytes(T, d_q0, d_aug);
 }
 
-diffqkv_status diffqkv_augq(const void*, const void*, const void*, const void*, const void*, int64_t, int32_t,
-                            int32_t, int32_t, int32_t, void*, size_t, void*, void*) {
-  return DIFFQKV_ERR_UNSUPPORTED;
+diffqkv_status diffqkv_augq(const void* h, const void* W_Q, const void* W_gate, const void* W_up, const void* W_down,
+                            int64_t T, int32_t d_model, int32_t d_q0, int32_t d_aug, int32_t d_out, void* workspace,
+                            size_t workspace_bytes, void* q_out, int32_t* dev_status, void* stream) {
+  if (!h || !W_Q || !W_gate || !W_up || !W_down || !q_out) return DIFFQKV_ERR_INVALID_ARG;
+  if (T < 0 || d_model <= 0 || d_q0 <= 0 || d_aug <= 0 || d_out <= 0) return DIFFQKV_ERR_INVALID_ARG;
+  if (T > 0x7fffff00LL) return DIFFQKV_ERR_UNSUPPORTED;
+  if (d_model % 128 != 0 || d_q0 % 128 != 0 || d_aug % 128 != 0 || d_out % 128 != 0) return DIFFQKV_ERR_UNSUPPORTED;
+  const void* ptrs[6] = {h, W_Q, W_gate, W_up, W_down, q_out};
+  for (const void* ptr : ptrs)
+    if (!aligned16(ptr)) return DIFFQKV_ERR_ALIGNMENT;
+  if (T == 0) return DIFFQKV_OK;
+  if (!workspace || workspace_bytes < augq_workspace_bytes(T, d_q0, d_aug)) return DIFFQKV_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DIFFQKV_ERR_ALIGNMENT;
+  const cudaError_t err = launch_augq(h, W_Q, W_gate, W_up, W_down, T, d_model, d_q0, d_aug, d_out, workspace, q_out,
+                                      dev_status, static_cast<cudaStream_t>(stream));
+  if (err == cudaErrorNotSupported) return DIFFQKV_ERR_UNSUPPORTED;
+  return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
 
 const char* diffqkv_status_string(diffqkv_status status) {

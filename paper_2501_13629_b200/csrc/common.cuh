@@ -72,4 +72,10 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
                               void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream);
 void set_tma_max_blocks(int n);
 
+// Augmented-Q projection (augq.cu): three tcgen05 GEMMs, the gate/up pair fused with its silu-gate epilogue.
+size_t augq_workspace_bytes(long long T, int d_q0, int d_aug);
+cudaError_t launch_augq(const void* h, const void* W_Q, const void* W_gate, const void* W_up, const void* W_down,
+                        long long T, int d_model, int d_q0, int d_aug, int d_out, void* workspace, void* q_out,
+                        int* dev_status, cudaStream_t stream);
+
 }  // namespace diffqkv
