@@ -207,9 +207,23 @@ diffqkv_status diffqkv_combine(const float* o_partial, const float* lse_partial,
   return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
 
-diffqkv_status diffqkv_prefill(const void*, const void*, const void*, int32_t, const diffqkv_cache*,
-                               const diffqkv_shape*, void*, float*, int32_t*, void*) {
-  return DIFFQKV_ERR_UNSUPPORTED;
+diffqkv_status diffqkv_prefill(const void* q, const void* k_new, const void* v_new, int32_t q_len,
+                               const diffqkv_cache* cache, const diffqkv_shape* shape, void* out, float* lse,
+                               int32_t* dev_status, void* stream) {
+  diffqkv_status st = check_shape(shape);
+  if (st != DIFFQKV_OK) return st;
+  if (!q || !k_new || !v_new || !out || q_len < 0) return DIFFQKV_ERR_INVALID_ARG;
+  st = check_cache(cache, shape);
+  if (st != DIFFQKV_OK) return st;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return DIFFQKV_ERR_ALIGNMENT;
+  if (q_len > cache->max_seqlen) return DIFFQKV_ERR_INVALID_ARG;
+  int box_tok = 0;
+  if (!prefill_supported(*shape, *cache, &box_tok)) return DIFFQKV_ERR_UNSUPPORTED;
+  if (shape->batch == 0 || q_len == 0) return DIFFQKV_OK;
+  const cudaError_t err = launch_prefill(q, k_new, v_new, q_len, *cache, *shape, box_tok, out, lse, dev_status,
+                                         static_cast<cudaStream_t>(stream));
+  if (err == cudaErrorNotSupported) return DIFFQKV_ERR_UNSUPPORTED;
+  return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
 
 size_t diffqkv_augq_workspace_bytes(int64_t T, int32_t d_q0, int32_t d_aug) {

@@ -78,4 +78,11 @@ cudaError_t launch_augq(const void* h, const void* W_Q, const void* W_gate, cons
                         long long T, int d_model, int d_q0, int d_aug, int d_out, void* workspace, void* q_out,
                         int* dev_status, cudaStream_t stream);
 
+
+// Causal prefill (prefill.cu): cache update kernel, then tcgen05 attention over the cache.
+bool prefill_supported(const diffqkv_shape& s, const diffqkv_cache& c, int* box_tok);
+cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, int q_len, const diffqkv_cache& c,
+                           const diffqkv_shape& s, int box_tok, void* out, float* lse, int* dev_status,
+                           cudaStream_t stream);
+
 }  // namespace diffqkv
