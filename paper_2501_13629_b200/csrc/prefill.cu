@@ -12,7 +12,7 @@
 //     warps 2-5   softmax of M-tile 0, warps 6-9 of M-tile 1: one thread per query row (= TMEM lane) reads its 64
 //                 scores with tcgen05.ld, masks the diagonal tiles, keeps a running reference maximum that is only
 //                 raised when the row maximum exceeds it by 2^8 (then O is rescaled in TMEM), writes P as bf16 into
-//                 shared memory in the swizzled K-major layout the second product reads, and sums the rounded values
+//                 shared memory in the swizzled K-major layout the second product reads, and sums the fp32 values
 //   fp32 scores, softmax statistics and output accumulation; P is rounded to bf16 for the second product.
 // Every wait is bounded; on expiry the block reports DIFFQKV_ERR_TIMEOUT, drains and frees its TMEM.
 #include "common.cuh"
@@ -53,8 +53,17 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ float lo_f(uint32_t v) { return __uint_as_float(v << 16); }
-__device__ __forceinline__ float hi_f(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+// 2^x by the special-function unit alone (flushes denormal results to zero; -inf gives +0).
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 
 __device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity, abort_flag));
@@ -255,14 +264,17 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         tc::wait_ld();
         const int k0 = j * kKT;
         const bool diag = k0 + kKT - 1 > past + q0 + t * kQT;  // block-uniform: the tile reaches past some row's position
-        float mx = -INFINITY;
+        if (diag) {
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          float v = __uint_as_float(s[c]) * p.scale_log2;
-          if (diag && k0 + c > qpos) v = -INFINITY;
-          s[c] = __float_as_uint(v);
-          mx = fmaxf(mx, v);
+          for (int c = 0; c < 64; ++c)
+            if (k0 + c > qpos) s[c] = 0xff800000u;  // -inf: this token lies after the row's position
         }
+        // row maximum of the raw scores (scale > 0 keeps the order), three inputs per instruction
+        float mx_raw = __uint_as_float(s[0]);
+#pragma unroll
+        for (int c = 1; c < 63; c += 2) mx_raw = max3(mx_raw, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+        mx_raw = fmaxf(mx_raw, __uint_as_float(s[63]));
+        const float mx = mx_raw * p.scale_log2;
         float alpha = 1.f;
         const bool bump = mx > m_ref + kRescaleThreshold;  // true on the first tile (m_ref = -inf)
         if (bump) {
@@ -286,16 +298,17 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           }
         }
         l *= alpha;
+        const float neg_m = -m_ref;
         // P = 2^(S - m_ref), rounded to bf16; row r of the tile, 16-byte chunks XORed with the row index
 #pragma unroll
         for (int c8 = 0; c8 < 8; ++c8) {
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float p0 = exp2f(__uint_as_float(s[c8 * 8 + 2 * e]) - m_ref);
-            const float p1 = exp2f(__uint_as_float(s[c8 * 8 + 2 * e + 1]) - m_ref);
+            const float p0 = ex2(fmaf(__uint_as_float(s[c8 * 8 + 2 * e]), p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(s[c8 * 8 + 2 * e + 1]), p.scale_log2, neg_m));
             w[e] = pack2(p0, p1);
-            l += lo_f(w[e]) + hi_f(w[e]);
+            l += p0 + p1;
           }
           *reinterpret_cast<uint4*>(prow + ((c8 ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
