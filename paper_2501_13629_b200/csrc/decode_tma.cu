@@ -110,6 +110,7 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   uint64_t* bars = reinterpret_cast<uint64_t*>(lbuf + kConsumerWarps * kHeadsPerMma);  // full[s], empty[s]
   volatile int* abort_flag = reinterpret_cast<int*>(bars + 2 * p.stages);         // set when a wait ran out
   int* prefix = const_cast<int*>(abort_flag) + 2;                                 // [batch + 1]
+  int* lens_s = prefix + p.batch + 1;                                             // [batch] lengths, clamped
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t full0 = ptx::smem_u32(bars), empty0 = ptx::smem_u32(bars + p.stages);
@@ -124,12 +125,20 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     ptx::prefetch_tmap(&tmap_k);
     ptx::prefetch_tmap(&tmap_v);
   }
+  // Everything above touches only this block's shared memory and the kernel parameters; from here on the
+  // kernel reads what earlier work in the stream may still be producing (lengths, q, the cache).
+  ptx::grid_dependency_wait();
+  // One round of global loads for the lengths (a dependent round trip costs most of a microsecond here); the
+  // prefix below comes out of shared memory.  The per-sequence reads further down go to global memory again
+  // (by then first-level cache hits): measured, that streams config 5 about 4 % faster than reading lens_s.
+  for (int b = tid; b < p.batch; b += kThreads) lens_s[b] = min(max(p.seqlens[b], 0), p.max_seqlen);
+  __syncthreads();
   // exclusive prefix of tiles per sequence (warp 0: per-lane chunks, then a warp scan)
   if (warp == 0) {
     const int per = (p.batch + 31) / 32;
     const int lo = lane * per, hi = min(p.batch, lo + per);
     int sum = 0;
-    for (int b = lo; b < hi; ++b) sum += (min(max(p.seqlens[b], 0), p.max_seqlen) + kTT - 1) / kTT;
+    for (int b = lo; b < hi; ++b) sum += (lens_s[b] + kTT - 1) / kTT;
     int incl = sum;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -139,14 +148,11 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     int run = incl - sum;
     for (int b = lo; b < hi; ++b) {
       prefix[b] = run;
-      run += (min(max(p.seqlens[b], 0), p.max_seqlen) + kTT - 1) / kTT;
+      run += (lens_s[b] + kTT - 1) / kTT;
     }
     if (lane == 31) prefix[p.batch] = incl;
   }
   __syncthreads();
-  // Let the combine kernel (launched with programmatic stream serialisation) get resident early; it
-  // still waits for this whole grid to finish before it reads any partial.
-  ptx::grid_launch_dependents();
   if (blockIdx.x == 0)
     for (int b = tid; b <= p.batch; b += kThreads) p.meta[b] = prefix[b];
 
@@ -220,6 +226,10 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
       }
       if (w.g + 1 < g_end) blk = fetch_blk();
     }
+    // All loads of this block are on their way: let the combine kernel (launched with programmatic stream
+    // serialisation) become resident now rather than earlier -- blocks that wait for this grid take issue
+    // slots while they wait.  It still waits for this whole grid to finish before it reads any partial.
+    ptx::grid_launch_dependents();
     if (!ok) {
       // Give copies already in flight a bounded chance to land before the block's shared memory is released.
       for (int s = 0; s < min(issued, p.stages); ++s) {
@@ -465,7 +475,8 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   }
 }
 
-// Merge of the segment partials written above.  One warp per output row (sequence, query head).
+// Merge of the segment partials written above: one block per output row (sequence, query head), the
+// partials dealt round-robin to its four warps so that their loads are in flight together.
 // A row whose sequence fits inside one block was already written in final form by the decode kernel.
 // Launched with programmatic stream serialisation: everything before grid_dependency_wait() only
 // touches inputs of the call (seqlens), so it overlaps the decode kernel's tail.
@@ -475,10 +486,11 @@ combine_segments_kernel(const float* __restrict__ o_partial, const float* __rest
                         const int* __restrict__ meta, const int* __restrict__ seqlens, int max_seqlen, int batch,
                         int n_q, int n_units, int U, int d_v, int grid_decode, void* __restrict__ out,
                         float* __restrict__ lse, int out_is_f32) {
-  const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
-  const bool active = row < (long long)batch * n_q;
-  const int lane = threadIdx.x & 31;
-  const int b = active ? (int)(row / n_q) : 0, h = active ? (int)(row % n_q) : 0;
+  __shared__ float4 part[4][128];  // per-warp weighted sums, d_v <= 512
+  ptx::grid_launch_dependents();   // whatever follows in the stream may begin its own prologue
+  const long long row = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = (int)(row / n_q), h = (int)(row % n_q);
   const int u = h / U, col = h % U;
   int nt = 0;
   long long before = 0, all = 0;  // tiles of earlier sequences / of all sequences
@@ -498,7 +510,6 @@ combine_segments_kernel(const float* __restrict__ o_partial, const float* __rest
     }
   }
   ptx::grid_dependency_wait();
-  if (!active) return;
   if (!small) {
     nt = meta[b + 1] - meta[b];
     before = meta[b];
@@ -507,11 +518,11 @@ combine_segments_kernel(const float* __restrict__ o_partial, const float* __rest
   const long long total = (long long)n_units * all;
   float4* out4 = reinterpret_cast<float4*>(out);
   if (nt == 0) {  // empty sequence: the decode kernel never touched this row
-    for (int ch = lane * 4; ch < d_v; ch += 128) {
+    for (int ch = threadIdx.x * 4; ch < d_v; ch += 512) {
       if (out_is_f32) out4[(row * d_v + ch) >> 2] = make_float4(0.f, 0.f, 0.f, 0.f);
       else *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + row * d_v + ch) = make_uint2(0u, 0u);
     }
-    if (lse && lane == 0) lse[row] = -INFINITY;
+    if (lse && threadIdx.x == 0) lse[row] = -INFINITY;
     return;
   }
   const long long base = (long long)n_units * before + (long long)u * nt;
@@ -527,48 +538,45 @@ combine_segments_kernel(const float* __restrict__ o_partial, const float* __rest
   for (int c = lane; c < n; c += 32) M = fmaxf(M, lp[(long long)c * U]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-  float wreg = 0.f, L = 0.f;  // lane c keeps the weight of partial c (first 32 partials)
-  for (int c = lane; c < n; c += 32) {
-    const float e = exp2f(lp[(long long)c * U] - M);
-    if (c < 32) wreg = e;
-    L += e;
-  }
+  float L = 0.f;
+  for (int c = lane; c < n; c += 32) L += exp2f(lp[(long long)c * U] - M);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
-  const float inv = 1.f / L;
-  for (int ch0 = 0; ch0 < d_v; ch0 += 128) {  // uniform trip count: the shuffles need all lanes
+  for (int ch0 = 0; ch0 < d_v; ch0 += 128) {
     const int ch = ch0 + lane * 4;
     const bool in = ch < d_v;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-    const int n32 = min(n, 32);
 #pragma unroll 4
-    for (int c = 0; c < n32; ++c) {
-      const float wgt = __shfl_sync(0xffffffffu, wreg, c);
-      if (in) {
-        const float4 v = *reinterpret_cast<const float4*>(op + (long long)c * U * d_v + ch);
-        a.x = fmaf(wgt, v.x, a.x); a.y = fmaf(wgt, v.y, a.y); a.z = fmaf(wgt, v.z, a.z); a.w = fmaf(wgt, v.w, a.w);
-      }
-    }
-    for (int c = 32; c < n; ++c) {
+    for (int c = warp; c < n; c += 4) {
       const float wgt = exp2f(lp[(long long)c * U] - M);
       if (in) {
         const float4 v = *reinterpret_cast<const float4*>(op + (long long)c * U * d_v + ch);
         a.x = fmaf(wgt, v.x, a.x); a.y = fmaf(wgt, v.y, a.y); a.z = fmaf(wgt, v.z, a.z); a.w = fmaf(wgt, v.w, a.w);
       }
     }
-    if (in) {
-      a.x *= inv; a.y *= inv; a.z *= inv; a.w *= inv;
-      if (out_is_f32) {
-        out4[(row * d_v + ch) >> 2] = a;
-      } else {
-        uint2 pk;
-        pk.x = pack_bf16(a.x, a.y);
-        pk.y = pack_bf16(a.z, a.w);
-        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + row * d_v + ch) = pk;
-      }
+    part[warp][ch0 / 4 + lane] = a;
+  }
+  __syncthreads();
+  const float inv = 1.f / L;
+  for (int i = threadIdx.x; i < d_v / 4; i += 128) {
+    float4 a = part[0][i];
+#pragma unroll
+    for (int w = 1; w < 4; ++w) {
+      const float4 v = part[w][i];
+      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    }
+    a.x *= inv; a.y *= inv; a.z *= inv; a.w *= inv;
+    const int ch = i * 4;
+    if (out_is_f32) {
+      out4[(row * d_v + ch) >> 2] = a;
+    } else {
+      uint2 pk;
+      pk.x = pack_bf16(a.x, a.y);
+      pk.y = pack_bf16(a.z, a.w);
+      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + row * d_v + ch) = pk;
     }
   }
-  if (lse && lane == 0) lse[row] = (M + log2f(L)) * kLn2;
+  if (lse && threadIdx.x == 0) lse[row] = (M + log2f(L)) * kLn2;
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -664,7 +672,7 @@ bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPla
   }
   const DeviceInfo di = device_info();
   if (di.sms <= 0) return false;
-  const int fixed = 1024 + kConsumerWarps * kHeadsPerMma * (s.d_v + 4 + 2) * 4 + 2 * 16 * 8 + (s.batch + 1) * 4 + 64;
+  const int fixed = 1024 + kConsumerWarps * kHeadsPerMma * (s.d_v + 4 + 2) * 4 + 2 * 16 * 8 + (2 * s.batch + 1) * 4 + 64;
   int stages = (di.max_smem - fixed) / v.stage_bytes;
   if (stages > 8) stages = 8;
   if (stages < 2) return false;
@@ -722,22 +730,26 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
 
   cudaError_t err = cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem);
   if (err != cudaSuccess) return err;
-  v.fn<<<plan.grid, kThreads, plan.smem, stream>>>(mk, mv, p);
-  count_launch();
-  err = cudaGetLastError();
-  if (err != cudaSuccess) return err;
-  profile_after_split(stream);
-  const long long rows = (long long)s.batch * s.n_q;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)((rows + 3) / 4));
-  cfg.blockDim = dim3(128);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = stream;
+  // both kernels may start before their predecessor in the stream has finished; each waits on the device
+  // before it touches anything the predecessor may still be producing
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)plan.grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = (size_t)plan.smem;
+  err = cudaLaunchKernelEx(&cfg, v.fn, mk, mv, p);
+  if (err != cudaSuccess) return err;
+  count_launch();
+  profile_after_split(stream);
+  const long long rows = (long long)s.batch * s.n_q;
+  cfg.gridDim = dim3((unsigned)rows);
+  cfg.blockDim = dim3(128);
+  cfg.dynamicSmemBytes = 0;
   err = cudaLaunchKernelEx(&cfg, combine_segments_kernel, (const float*)p.o_partial, (const float*)p.lse_partial,
                            (const int*)p.meta, c.seqlens, c.max_seqlen, s.batch, s.n_q, p.n_units, plan.U, s.d_v,
                            plan.grid, out, lse, p.out_is_f32);
