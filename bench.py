@@ -304,6 +304,10 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=device)
         barrier = lambda: (dist.barrier(), torch.cuda.synchronize())  # noqa: E731
     peaks = measured_peaks()
+    if args.workload == "prefill":  # the config 4 leg alone (the command profilers wrap for the tensor-core kernels)
+        if rank == 0:
+            print(json.dumps({"workload": W.CFG4.name, **time_prefill(api, W, device, peaks, max(1, min(args.steps, 20)))}))
+        return
 
     cfg = W.CFG3
     host = W.make_decode_inputs(cfg)
@@ -461,6 +465,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="headline workload only")
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill"],
+                    help="decode = the headline line (default); prefill = only the config 4 timings")
     ap.add_argument("--profile", action="store_true",
                     help="only the timed loop of the headline workload (the command profilers wrap)")
     args = ap.parse_args()
