@@ -30,6 +30,9 @@ if ROOT not in sys.path:
 METRIC = "decode_kv_cache_bandwidth"
 UNIT = "GB/s"
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the split kernel on the headline workload, from the
+# ncu capture summarised in profiles/decode_tma_kernel_cfg3.md (set to None whenever the kernel changes after it).
+SPLIT_KERNEL_DRAM_BYTES = 407.8e6
 
 
 def measured_peaks():
@@ -349,7 +352,8 @@ def run_ours(args):
         k_ms = case.time_split_kernel(min(args.steps, 200))
         ach = case.bytes / (k_ms * 1e-3) / 1e9
         line["roofline"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                            "frac": ach / peaks["hbm_gbs"], "traffic": None, "kernel": "decode split kernel",
+                            "frac": ach / peaks["hbm_gbs"], "traffic": SPLIT_KERNEL_DRAM_BYTES,
+                            "kernel": "decode split kernel",
                             "kernel_ms": k_ms, "peak_source": peaks["source"] + " (burst copy)"}
         e2e_ms, h2d, d2h = case.time_e2e(min(args.steps, 500), min(args.warmup, 20))
         e2e_step = e2e_ms / min(args.steps, 500)
