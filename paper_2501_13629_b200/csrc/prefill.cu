@@ -5,10 +5,10 @@
 // Step 2, prefill_attn_kernel: one block per (sequence, query head, 256 query rows), longest blocks first.
 //   The 256 rows are two M-tiles of 128 that share every K/V tile the block stages (K head h*n_k/n_q, V head
 //   h*n_v/n_q, read from the cache, so a cached prefix is attended as well); KV tiles hold 64 tokens.
-//     warp 0      TMA producer: both Q tiles once, then (K tile, V tile) pairs into a 3-stage ring (128-byte swizzle)
+//     warp 0      TMA producer: both Q tiles once, then K tiles and V tiles into 4-slot rings with their own barriers
 //     warp 1      MMA issuer: S_t = Q_t K^T (tcgen05.mma 128x64x16, fp32 in TMEM), O_t += P_t V (128x128x16, V as an
-//                 N-major operand straight from the token-major tile); the two M-tiles alternate so that the tensor
-//                 core works on one while the softmax warps work on the other
+//                 N-major operand straight from the token-major tile); scores are double-buffered per M-tile, so
+//                 the next QK^T is issued before the softmax of the current tile ends, and the two M-tiles alternate
 //     warps 2-5   softmax of M-tile 0, warps 6-9 of M-tile 1: one thread per query row (= TMEM lane) reads its 64
 //                 scores with tcgen05.ld, masks the diagonal tiles, keeps a running reference maximum that is only
 //                 raised when the row maximum exceeds it by 2^8 (then O is rescaled in TMEM), writes P as bf16 into
@@ -26,13 +26,13 @@ namespace {
 constexpr int kQT = 128;  // query rows per M-tile
 constexpr int kKT = 64;   // cached tokens per KV tile
 constexpr int kD = 128;   // channels per head (Q/K and V)
-constexpr int kKVStages = 3;
+constexpr int kKVStages = 4;
 constexpr int kQBytes = kQT * kD * 2;   // 32 KB: [half][128 rows][128 B]
 constexpr int kKBytes = kKT * kD * 2;   // 16 KB: [half][64 rows][128 B]
 constexpr int kKVBytes = 2 * kKBytes;   // K tile then V tile
 constexpr int kPBytes = kQT * kKT * 2;  // 16 KB: [128 rows][128 B]
 constexpr int kPrefillThreads = 320;
-constexpr int kTmemCols = 512;          // S0 0..63, S1 64..127, O0 128..255, O1 256..383
+constexpr int kTmemCols = 512;          // S[t][buf] at (2 t + buf) * 64 (0..255), O[t] at 256 + 128 t
 constexpr int kPrefillSmem = 1024 + 2 * kQBytes + kKVStages * kKVBytes + 2 * kPBytes + 256;
 constexpr float kRescaleThreshold = 8.f;  // log2 domain
 
@@ -78,12 +78,13 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   unsigned char* kv_s = q_s + 2 * kQBytes;              // ring of (K, V)
   unsigned char* p_s = kv_s + kKVStages * kKVBytes;     // 2 M-tiles
   uint64_t* bars = reinterpret_cast<uint64_t*>(p_s + 2 * kPBytes);
-  // q_full, kv_full[S], kv_empty[S], s_full[2], p_full[2], o_done[2], drain
+  // q_full, k_full[S], k_empty[S], v_full[S], v_empty[S], s_full[2 tiles][2 buffers], p_full[2], o_done[2], drain
   const uint32_t q_full = ptx::smem_u32(bars);
-  const uint32_t kv_full0 = q_full + 8, kv_empty0 = kv_full0 + 8 * kKVStages;
-  const uint32_t s_full0 = kv_empty0 + 8 * kKVStages, p_full0 = s_full0 + 16, o_done0 = p_full0 + 16;
+  const uint32_t k_full0 = q_full + 8, k_empty0 = k_full0 + 8 * kKVStages;
+  const uint32_t v_full0 = k_empty0 + 8 * kKVStages, v_empty0 = v_full0 + 8 * kKVStages;
+  const uint32_t s_full0 = v_empty0 + 8 * kKVStages, p_full0 = s_full0 + 32, o_done0 = p_full0 + 16;
   const uint32_t drain = o_done0 + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 + 2 * kKVStages + 6);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 + 4 * kKVStages + 8);
   volatile int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -91,11 +92,14 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     *abort_flag = 0;
     ptx::mbar_init(q_full, 1);
     for (int s = 0; s < kKVStages; ++s) {
-      ptx::mbar_init(kv_full0 + 8 * s, 1);
-      ptx::mbar_init(kv_empty0 + 8 * s, 1);
+      ptx::mbar_init(k_full0 + 8 * s, 1);
+      ptx::mbar_init(k_empty0 + 8 * s, 1);
+      ptx::mbar_init(v_full0 + 8 * s, 1);
+      ptx::mbar_init(v_empty0 + 8 * s, 1);
     }
     for (int t = 0; t < 2; ++t) {
-      ptx::mbar_init(s_full0 + 8 * t, 1);
+      ptx::mbar_init(s_full0 + 16 * t, 1);
+      ptx::mbar_init(s_full0 + 16 * t + 8, 1);
       ptx::mbar_init(p_full0 + 8 * t, 4);
       ptx::mbar_init(o_done0 + 8 * t, 1);
     }
@@ -141,7 +145,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       for (int t = 0; t < 2; ++t)
         if (nkv[t] > 0) ptx::tma_load_5d(q_u32 + t * kQBytes, &tmap_q, q_full, 0, q0 + t * kQT, 0, h, b);
     }
-    // One box per (K or V, token part, channel half): lane x owns box x of every tile.
+    // One box per (K or V, token part, channel half): lane x owns box x of every tile.  K and V tiles have their
+    // own full/empty barriers: a K slot is free again as soon as its QK^T is done, two tiles before its V slot.
     const int parts = kKT / p.box_tok;
     const int boxes = 4 * parts;
     const int my_kv = lane / (2 * parts), my_part = (lane / 2) % parts, my_half = lane & 1;
@@ -149,96 +154,114 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     int stage = 0, issued = 0;
     uint32_t phase = 0;
     bool ok = true;
-    for (int j = 0; j < nkv_max; ++j) {
-      if (!wait_warp(kv_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+    for (int j = 0; j < nkv_max && ok; ++j) {
       const int tok0 = j * kKT;
       const int parts_valid = min(parts, (kv_len - tok0 + p.box_tok - 1) / p.box_tok);
-      const uint32_t bar = kv_full0 + 8 * stage;
-      if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)parts_valid * p.box_tok * 128u * 4u);
-      __syncwarp();
-      if (lane < boxes && my_part < parts_valid) {
-        const int tok = tok0 + my_part * p.box_tok;
-        int blk = b, slot = tok;
-        if (p.page_table) {
-          blk = p.page_table[(long long)b * p.max_pages_per_seq + tok / p.page_size];
-          slot = tok % p.page_size;
-          if (blk < 0 || blk >= p.num_blocks) {  // never read outside the pool: flag it, read block 0 instead
-            report(p.dev_status, DIFFQKV_ERR_INDEX);
-            blk = 0;
-          }
+      int blk = b, slot = tok0 + my_part * p.box_tok;
+      const bool mine = lane < boxes && my_part < parts_valid;
+      if (mine && p.page_table) {
+        const int tok = slot;
+        blk = p.page_table[(long long)b * p.max_pages_per_seq + tok / p.page_size];
+        slot = tok % p.page_size;
+        if (blk < 0 || blk >= p.num_blocks) {  // never read outside the pool: flag it, read block 0 instead
+          report(p.dev_status, DIFFQKV_ERR_INDEX);
+          blk = 0;
         }
-        const uint32_t dst = kv_u32 + stage * kKVBytes + my_off;
-        if (my_kv == 0) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, my_half, hk, blk);
-        else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, my_half, hv, blk);
       }
-      ++issued;
+      const uint32_t dst = kv_u32 + stage * kKVBytes + my_off;
+#pragma unroll
+      for (int kv = 0; kv < 2; ++kv) {
+        if (!wait_warp((kv ? v_empty0 : k_empty0) + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+        const uint32_t bar = (kv ? v_full0 : k_full0) + 8 * stage;
+        if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)parts_valid * p.box_tok * 128u * 2u);
+        __syncwarp();
+        if (mine && my_kv == kv) {
+          if (kv == 0) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, my_half, hk, blk);
+          else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, my_half, hv, blk);
+        }
+        if (kv) ++issued;
+      }
       if (++stage == kKVStages) { stage = 0; phase ^= 1; }
     }
     if (!ok) {
       report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+      // give copies in flight a bounded chance to land before the block's shared memory is released (a K copy
+      // whose V twin was never issued is covered by the wait on the next use of its barrier timing out)
       ptx::mbar_wait(q_full, 0, nullptr);
-      for (int s = 0; s < min(issued, kKVStages); ++s) {
-        const int uses = (issued - s + kKVStages - 1) / kKVStages;
-        ptx::mbar_wait(kv_full0 + 8 * s, (uint32_t)(uses - 1) & 1u, nullptr);
+      for (int s2 = 0; s2 < min(issued, kKVStages); ++s2) {
+        const int uses = (issued - s2 + kKVStages - 1) / kKVStages;
+        ptx::mbar_wait(k_full0 + 8 * s2, (uint32_t)(uses - 1) & 1u, nullptr);
+        ptx::mbar_wait(v_full0 + 8 * s2, (uint32_t)(uses - 1) & 1u, nullptr);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
+    // One thread runs the whole issue loop.  The products here are small (32 or 64 tensor-pipe cycles each), so the
+    // loop is kept lean: descriptor halves are precomputed and only their address field is stepped.
     constexpr uint32_t idesc_s = tc::idesc_bf16_f32(kQT, kKT, 0, 0);
     constexpr uint32_t idesc_pv = tc::idesc_bf16_f32(kQT, kD, 0, 1);
-    auto issue_s = [&](int t, int j) {  // S_t = Q_t . K_j^T
-      const uint32_t qa = q_u32 + t * kQBytes, ka = kv_u32 + (j % kKVStages) * kKVBytes;
+    constexpr uint32_t hi_k = tc::smem_desc_hi_sw128(1024);  // K-major operands (Q, K, P) and the N-major V alike:
+                                                             // 8-row groups are 1024 bytes apart
+    bool ok = true;
+    if (lane == 0) {
+      const uint32_t q_lo = tc::smem_desc_lo(q_u32, 16), k_lo = tc::smem_desc_lo(kv_u32, 16);
+      const uint32_t p_lo = tc::smem_desc_lo(p_u32, 16), v_lo = tc::smem_desc_lo(kv_u32 + kKBytes, kKT * 128);
+      auto issue_s = [&](int t, int j) {  // S_t = Q_t . K_j^T
+        const uint32_t qa = q_lo + t * (kQBytes >> 4), ka = k_lo + (j % kKVStages) * (kKVBytes >> 4);
+        const uint32_t d = tmem_base + (2 * t + (j & 1)) * kKT;
+        tc::mma_ss_halves<false>(d, qa, hi_k, ka, hi_k, idesc_s);
 #pragma unroll
-      for (int ks = 0; ks < kD / 16; ++ks) {
-        const uint64_t da = tc::smem_desc_sw128(qa + (ks / 4) * (kQT * 128) + (ks % 4) * 32, 16, 1024);
-        const uint64_t db = tc::smem_desc_sw128(ka + (ks / 4) * (kKT * 128) + (ks % 4) * 32, 16, 1024);
-        tc::mma_ss(tmem_base + t * kKT, da, db, idesc_s, ks > 0 ? 1u : 0u);
-      }
-      tc::commit(s_full0 + 8 * t);
-    };
-    auto issue_pv = [&](int t, int j) {  // O_t += P_t . V_j
-      const uint32_t pa = p_u32 + t * kPBytes, va = kv_u32 + (j % kKVStages) * kKVBytes + kKBytes;
+        for (int ks = 1; ks < kD / 16; ++ks)
+          tc::mma_ss_halves<true>(d, qa + (((ks / 4) * (kQT * 128) + (ks % 4) * 32) >> 4), hi_k,
+                                  ka + (((ks / 4) * (kKT * 128) + (ks % 4) * 32) >> 4), hi_k, idesc_s);
+        tc::commit(s_full0 + 16 * t + 8 * (j & 1));
+      };
+      auto issue_pv = [&](int t, int j) {  // O_t += P_t . V_j
+        const uint32_t pa = p_lo + t * (kPBytes >> 4), va = v_lo + (j % kKVStages) * (kKVBytes >> 4);
+        const uint32_t d = tmem_base + 256 + t * kD;
+        if (j == 0) tc::mma_ss_halves<false>(d, pa, hi_k, va, hi_k, idesc_pv);
+        else tc::mma_ss_halves<true>(d, pa, hi_k, va, hi_k, idesc_pv);
 #pragma unroll
-      for (int k = 0; k < kKT / 16; ++k) {
-        const uint64_t da = tc::smem_desc_sw128(pa + k * 32, 16, 1024);
-        const uint64_t db = tc::smem_desc_sw128(va + k * (16 * 128), kKT * 128, 1024);
-        tc::mma_ss(tmem_base + 128 + t * kD, da, db, idesc_pv, (j > 0 || k > 0) ? 1u : 0u);
+        for (int k = 1; k < kKT / 16; ++k)
+          tc::mma_ss_halves<true>(d, pa + ((k * 32) >> 4), hi_k, va + ((k * 16 * 128) >> 4), hi_k, idesc_pv);
+        tc::commit(o_done0 + 8 * t);
+      };
+      // The scores of a tile have two buffers per M-tile: S(t, j + 2) is issued as soon as the softmax warps have
+      // consumed S(t, j) (which p_full(t, j) implies), so S(t, j + 1) is ready long before they ask for it.
+      ok = ptx::mbar_wait(q_full, 0, abort_flag);
+      for (int j = 0; j < min(2, nkv_max) && ok; ++j) {
+        ok = ptx::mbar_wait(k_full0 + 8 * j, 0, abort_flag);
+        if (!ok) break;
+        tc::fence_after_sync();
+        if (j < nkv[0]) issue_s(0, j);
+        if (j < nkv[1]) issue_s(1, j);
+        tc::commit(k_empty0 + 8 * j);  // K tile j is free once these products are done
       }
-      tc::commit(o_done0 + 8 * t);
-    };
-    bool ok = wait_warp(q_full, 0, abort_flag);
-    if (ok && nkv_max > 0) ok = wait_warp(kv_full0, 0, abort_flag);
-    if (ok) {
-      tc::fence_after_sync();
-      if (lane == 0) {
-        if (nkv[0] > 0) issue_s(0, 0);
-        if (nkv[1] > 0) issue_s(1, 0);
+      for (int j = 0; j < nkv_max && ok; ++j) {
+        const int st = j % kKVStages, st2 = (j + 2) % kKVStages;
+        const uint32_t ph = (j / kKVStages) & 1, ph2 = ((j + 2) / kKVStages) & 1;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          if (j < nkv[t]) {
+            if (!ptx::mbar_wait(p_full0 + 8 * t, j & 1, abort_flag) || !ptx::mbar_wait(v_full0 + 8 * st, ph, abort_flag)) {
+              ok = false;
+              break;
+            }
+            tc::fence_after_sync();
+            issue_pv(t, j);
+          }
+          if (t == 1) tc::commit(v_empty0 + 8 * st);  // every MMA that reads V tile j has been issued
+          if (j + 2 < nkv[t]) {
+            if (!ptx::mbar_wait(k_full0 + 8 * st2, ph2, abort_flag)) { ok = false; break; }
+            tc::fence_after_sync();
+            issue_s(t, j + 2);
+          }
+          if (t == 1 && j + 2 < nkv_max) tc::commit(k_empty0 + 8 * st2);  // ... and every MMA that reads K tile j + 2
+        }
       }
-      __syncwarp();
+      if (!ok) report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+      tc::commit(drain);
     }
-    for (int j = 0; j < nkv_max && ok; ++j) {
-#pragma unroll
-      for (int t = 0; t < 2; ++t) {
-        if (j < nkv[t]) {
-          if (!wait_warp(p_full0 + 8 * t, j & 1, abort_flag)) { ok = false; break; }
-          tc::fence_after_sync();
-          if (lane == 0) issue_pv(t, j);
-          __syncwarp();
-        }
-        if (t == 1) {  // every MMA that reads stage j has been issued
-          if (lane == 0) tc::commit(kv_empty0 + 8 * (j % kKVStages));
-          __syncwarp();
-        }
-        if (j + 1 < nkv[t]) {
-          if (!wait_warp(kv_full0 + 8 * ((j + 1) % kKVStages), ((j + 1) / kKVStages) & 1, abort_flag)) { ok = false; break; }
-          tc::fence_after_sync();
-          if (lane == 0) issue_s(t, j + 1);
-          __syncwarp();
-        }
-      }
-    }
-    if (!ok) report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
-    if (lane == 0) tc::commit(drain);
     __syncwarp();
   } else {
     // ------------------------------------------------------------------ softmax warps
@@ -250,13 +273,13 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       const int qrow = q0 + t * kQT + r;
       const int qpos = past + qrow;
       const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-      const uint32_t s_taddr = lane_base + t * kKT;
-      const uint32_t o_taddr = lane_base + 128 + t * kD;
+      const uint32_t o_taddr = lane_base + 256 + t * kD;
       unsigned char* prow = p_s + t * kPBytes + r * 128;
       float m_ref = -INFINITY, l = 0.f;
       bool ok = true;
       for (int j = 0; j < n; ++j) {
-        if (!wait_warp(s_full0 + 8 * t, j & 1, abort_flag)) { ok = false; break; }
+        if (!wait_warp(s_full0 + 16 * t + 8 * (j & 1), (j >> 1) & 1, abort_flag)) { ok = false; break; }
+        const uint32_t s_taddr = lane_base + (2 * t + (j & 1)) * kKT;
         tc::fence_after_sync();
         uint32_t s[64];
         tc::ld_32x32b_x32(s_taddr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
@@ -315,7 +338,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         if (j == nkv_max - 1 && (kv_len & (kKT - 1)) != 0) {
           // ragged last tile: V rows past the sequence end hold whatever followed in memory; zero them
           // (0 * NaN would poison the product).  Both M-tiles may do this; they write the same zeros.
-          if (!wait_warp(kv_full0 + 8 * (j % kKVStages), (j / kKVStages) & 1, abort_flag)) { ok = false; break; }
+          if (!wait_warp(v_full0 + 8 * (j % kKVStages), (j / kKVStages) & 1, abort_flag)) { ok = false; break; }
           const int row = r & 63, half = r >> 6;
           if (row >= kv_len - k0) {
             uint4* dst = reinterpret_cast<uint4*>(kv_s + (j % kKVStages) * kKVBytes + kKBytes + half * (kKT * 128) + row * 128);
