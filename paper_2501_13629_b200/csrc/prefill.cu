@@ -4,15 +4,19 @@
 // Step 1, cache_append_kernel: the new K and V rows go to positions past_b .. past_b + q_len - 1 of the pools.
 // Step 2, prefill_attn_kernel: one block per (sequence, query head, 256 query rows), longest blocks first.
 //   The 256 rows are two M-tiles of 128 that share every K/V tile the block stages (K head h*n_k/n_q, V head
-//   h*n_v/n_q, read from the cache, so a cached prefix is attended as well); KV tiles hold 64 tokens.
-//     warp 0      TMA producer: both Q tiles once, then K tiles and V tiles into 4-slot rings with their own barriers
-//     warp 1      MMA issuer: S_t = Q_t K^T (tcgen05.mma 128x64x16, fp32 in TMEM), O_t += P_t V (128x128x16, V as an
-//                 N-major operand straight from the token-major tile); scores are double-buffered per M-tile, so
-//                 the next QK^T is issued before the softmax of the current tile ends, and the two M-tiles alternate
-//     warps 2-5   softmax of M-tile 0, warps 6-9 of M-tile 1: one thread per query row (= TMEM lane) reads its 64
-//                 scores with tcgen05.ld, masks the diagonal tiles, keeps a running reference maximum that is only
-//                 raised when the row maximum exceeds it by 2^8 (then O is rescaled in TMEM), writes P as bf16 into
-//                 shared memory in the swizzled K-major layout the second product reads, and sums the fp32 values
+//   h*n_v/n_q, read from the cache, so a cached prefix is attended as well); KV tiles hold 128 tokens.
+//     warp 0      TMA producer: both Q tiles once, then K tiles (ring of 3) and V tiles (ring of 2), 128-byte swizzle,
+//                 each ring with its own barriers: a K slot is free as soon as its QK^T is done
+//     warp 1      one thread issues the MMAs: S_t = Q_t K^T (tcgen05.mma 128x128x16 from shared memory, fp32 in
+//                 TMEM) and O_t += P_t V (128x128x16, P read from TMEM, V as an N-major operand straight from its
+//                 token-major tile); the two M-tiles alternate, so the tensor core works on one while the softmax
+//                 warps work on the other.  Operands are what bounds these products (about 100 bytes per cycle
+//                 reach the tensor core from shared memory), hence 128-wide tiles and P kept out of shared memory.
+//     warps 2-5   softmax of M-tile 0, warps 6-9 of M-tile 1: one thread per query row (= TMEM lane).  Pass 1 reads
+//                 the 128 scores (tcgen05.ld) for the row maximum; a running reference maximum is only raised when
+//                 exceeded by 2^8 (then O is rescaled in TMEM).  Pass 2 reads them again 32 at a time, computes
+//                 P = 2^(S scale - m), sums it in fp32 and writes it as packed bf16 over the scores it has already
+//                 consumed (tcgen05.st), where the second product reads it.
 //   fp32 scores, softmax statistics and output accumulation; P is rounded to bf16 for the second product.
 // Every wait is bounded; on expiry the block reports DIFFQKV_ERR_TIMEOUT, drains and frees its TMEM.
 #include "common.cuh"
@@ -24,16 +28,14 @@ namespace diffqkv {
 namespace {
 
 constexpr int kQT = 128;  // query rows per M-tile
-constexpr int kKT = 64;   // cached tokens per KV tile
+constexpr int kKT = 128;  // cached tokens per KV tile
 constexpr int kD = 128;   // channels per head (Q/K and V)
-constexpr int kKVStages = 4;
-constexpr int kQBytes = kQT * kD * 2;   // 32 KB: [half][128 rows][128 B]
-constexpr int kKBytes = kKT * kD * 2;   // 16 KB: [half][64 rows][128 B]
-constexpr int kKVBytes = 2 * kKBytes;   // K tile then V tile
-constexpr int kPBytes = kQT * kKT * 2;  // 16 KB: [128 rows][128 B]
+constexpr int kKSlots = 3, kVSlots = 2;
+constexpr int kQBytes = kQT * kD * 2;  // 32 KB: [half][128 rows][128 B]
+constexpr int kTBytes = kKT * kD * 2;  // 32 KB, a K tile or a V tile: [half][128 rows][128 B]
 constexpr int kPrefillThreads = 320;
-constexpr int kTmemCols = 512;          // S[t][buf] at (2 t + buf) * 64 (0..255), O[t] at 256 + 128 t
-constexpr int kPrefillSmem = 1024 + 2 * kQBytes + kKVStages * kKVBytes + 2 * kPBytes + 256;
+constexpr int kTmemCols = 512;         // S[t] (and P[t] over its first 64 columns) at 128 t, O[t] at 256 + 128 t
+constexpr int kPrefillSmem = 1024 + 2 * kQBytes + (kKSlots + kVSlots) * kTBytes + 256;
 constexpr float kRescaleThreshold = 8.f;  // log2 domain
 
 struct PrefillParams {
@@ -41,7 +43,7 @@ struct PrefillParams {
   const int* page_table;
   int page_size, max_pages_per_seq, num_blocks, max_seqlen;
   int batch, q_len, n_q, n_k, n_v, n_qpairs;
-  int box_tok;  // tokens per TMA box of the cache maps (64, or the page size when smaller)
+  int box_tok;  // tokens per TMA box of the cache maps (128, or the page size when smaller)
   float scale_log2;
   void* out;
   int out_is_f32;
@@ -74,32 +76,33 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                     const __grid_constant__ CUtensorMap tmap_v, const PrefillParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char* q_s = smem;                            // 2 M-tiles
-  unsigned char* kv_s = q_s + 2 * kQBytes;              // ring of (K, V)
-  unsigned char* p_s = kv_s + kKVStages * kKVBytes;     // 2 M-tiles
-  uint64_t* bars = reinterpret_cast<uint64_t*>(p_s + 2 * kPBytes);
-  // q_full, k_full[S], k_empty[S], v_full[S], v_empty[S], s_full[2 tiles][2 buffers], p_full[2], o_done[2], drain
+  unsigned char* q_s = smem;                      // 2 M-tiles
+  unsigned char* k_s = q_s + 2 * kQBytes;         // ring of K tiles
+  unsigned char* v_s = k_s + kKSlots * kTBytes;   // ring of V tiles
+  uint64_t* bars = reinterpret_cast<uint64_t*>(v_s + kVSlots * kTBytes);
+  // q_full, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2], drain
   const uint32_t q_full = ptx::smem_u32(bars);
-  const uint32_t k_full0 = q_full + 8, k_empty0 = k_full0 + 8 * kKVStages;
-  const uint32_t v_full0 = k_empty0 + 8 * kKVStages, v_empty0 = v_full0 + 8 * kKVStages;
-  const uint32_t s_full0 = v_empty0 + 8 * kKVStages, p_full0 = s_full0 + 32, o_done0 = p_full0 + 16;
+  const uint32_t k_full0 = q_full + 8, k_empty0 = k_full0 + 8 * kKSlots;
+  const uint32_t v_full0 = k_empty0 + 8 * kKSlots, v_empty0 = v_full0 + 8 * kVSlots;
+  const uint32_t s_full0 = v_empty0 + 8 * kVSlots, p_full0 = s_full0 + 16, o_done0 = p_full0 + 16;
   const uint32_t drain = o_done0 + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 + 4 * kKVStages + 8);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 + 2 * kKSlots + 2 * kVSlots + 6);
   volatile int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     *abort_flag = 0;
     ptx::mbar_init(q_full, 1);
-    for (int s = 0; s < kKVStages; ++s) {
+    for (int s = 0; s < kKSlots; ++s) {
       ptx::mbar_init(k_full0 + 8 * s, 1);
       ptx::mbar_init(k_empty0 + 8 * s, 1);
+    }
+    for (int s = 0; s < kVSlots; ++s) {
       ptx::mbar_init(v_full0 + 8 * s, 1);
       ptx::mbar_init(v_empty0 + 8 * s, 1);
     }
     for (int t = 0; t < 2; ++t) {
-      ptx::mbar_init(s_full0 + 16 * t, 1);
-      ptx::mbar_init(s_full0 + 16 * t + 8, 1);
+      ptx::mbar_init(s_full0 + 8 * t, 1);
       ptx::mbar_init(p_full0 + 8 * t, 4);
       ptx::mbar_init(o_done0 + 8 * t, 1);
     }
@@ -134,7 +137,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     nkv[t] = r0 < p.q_len ? (min(kv_len, past + r0 + kQT) + kKT - 1) / kKT : 0;
   }
   const int nkv_max = max(nkv[0], nkv[1]);
-  const uint32_t q_u32 = ptx::smem_u32(q_s), kv_u32 = ptx::smem_u32(kv_s), p_u32 = ptx::smem_u32(p_s);
+  const uint32_t q_u32 = ptx::smem_u32(q_s), k_u32 = ptx::smem_u32(k_s), v_u32 = ptx::smem_u32(v_s);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -145,14 +148,13 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       for (int t = 0; t < 2; ++t)
         if (nkv[t] > 0) ptx::tma_load_5d(q_u32 + t * kQBytes, &tmap_q, q_full, 0, q0 + t * kQT, 0, h, b);
     }
-    // One box per (K or V, token part, channel half): lane x owns box x of every tile.  K and V tiles have their
-    // own full/empty barriers: a K slot is free again as soon as its QK^T is done, two tiles before its V slot.
+    // One box per (token part, channel half) of a tile: lane x owns box x of every K tile and of every V tile.
     const int parts = kKT / p.box_tok;
-    const int boxes = 4 * parts;
-    const int my_kv = lane / (2 * parts), my_part = (lane / 2) % parts, my_half = lane & 1;
-    const uint32_t my_off = my_kv * kKBytes + my_half * (kKT * 128) + my_part * (p.box_tok * 128);
-    int stage = 0, issued = 0;
-    uint32_t phase = 0;
+    const int boxes = 2 * parts;
+    const int my_part = lane >> 1, my_half = lane & 1;
+    const uint32_t my_off = my_half * (kKT * 128) + my_part * (p.box_tok * 128);
+    int ks = 0, vs = 0, issued_k = 0, issued_v = 0;
+    uint32_t kph = 0, vph = 0;
     bool ok = true;
     for (int j = 0; j < nkv_max && ok; ++j) {
       const int tok0 = j * kKT;
@@ -168,96 +170,89 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           blk = 0;
         }
       }
-      const uint32_t dst = kv_u32 + stage * kKVBytes + my_off;
-#pragma unroll
-      for (int kv = 0; kv < 2; ++kv) {
-        if (!wait_warp((kv ? v_empty0 : k_empty0) + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-        const uint32_t bar = (kv ? v_full0 : k_full0) + 8 * stage;
-        if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)parts_valid * p.box_tok * 128u * 2u);
-        __syncwarp();
-        if (mine && my_kv == kv) {
-          if (kv == 0) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, my_half, hk, blk);
-          else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, my_half, hv, blk);
-        }
-        if (kv) ++issued;
-      }
-      if (++stage == kKVStages) { stage = 0; phase ^= 1; }
+      const uint32_t tx = (uint32_t)parts_valid * p.box_tok * 128u * 2u;
+      if (!wait_warp(k_empty0 + 8 * ks, kph ^ 1, abort_flag)) { ok = false; break; }
+      if (lane == 0) ptx::mbar_arrive_expect_tx(k_full0 + 8 * ks, tx);
+      __syncwarp();
+      if (mine) ptx::tma_load_5d(k_u32 + ks * kTBytes + my_off, &tmap_k, k_full0 + 8 * ks, 0, slot, my_half, hk, blk);
+      ++issued_k;
+      if (++ks == kKSlots) { ks = 0; kph ^= 1; }
+      if (!wait_warp(v_empty0 + 8 * vs, vph ^ 1, abort_flag)) { ok = false; break; }
+      if (lane == 0) ptx::mbar_arrive_expect_tx(v_full0 + 8 * vs, tx);
+      __syncwarp();
+      if (mine) ptx::tma_load_5d(v_u32 + vs * kTBytes + my_off, &tmap_v, v_full0 + 8 * vs, 0, slot, my_half, hv, blk);
+      ++issued_v;
+      if (++vs == kVSlots) { vs = 0; vph ^= 1; }
     }
     if (!ok) {
       report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
-      // give copies in flight a bounded chance to land before the block's shared memory is released (a K copy
-      // whose V twin was never issued is covered by the wait on the next use of its barrier timing out)
+      // give copies in flight a bounded chance to land before the block's shared memory is released
       ptx::mbar_wait(q_full, 0, nullptr);
-      for (int s2 = 0; s2 < min(issued, kKVStages); ++s2) {
-        const int uses = (issued - s2 + kKVStages - 1) / kKVStages;
-        ptx::mbar_wait(k_full0 + 8 * s2, (uint32_t)(uses - 1) & 1u, nullptr);
-        ptx::mbar_wait(v_full0 + 8 * s2, (uint32_t)(uses - 1) & 1u, nullptr);
-      }
+      for (int s2 = 0; s2 < min(issued_k, kKSlots); ++s2)
+        ptx::mbar_wait(k_full0 + 8 * s2, (uint32_t)((issued_k - s2 + kKSlots - 1) / kKSlots - 1) & 1u, nullptr);
+      for (int s2 = 0; s2 < min(issued_v, kVSlots); ++s2)
+        ptx::mbar_wait(v_full0 + 8 * s2, (uint32_t)((issued_v - s2 + kVSlots - 1) / kVSlots - 1) & 1u, nullptr);
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    // One thread runs the whole issue loop.  The products here are small (32 or 64 tensor-pipe cycles each), so the
-    // loop is kept lean: descriptor halves are precomputed and only their address field is stepped.
-    constexpr uint32_t idesc_s = tc::idesc_bf16_f32(kQT, kKT, 0, 0);
-    constexpr uint32_t idesc_pv = tc::idesc_bf16_f32(kQT, kD, 0, 1);
-    constexpr uint32_t hi_k = tc::smem_desc_hi_sw128(1024);  // K-major operands (Q, K, P) and the N-major V alike:
-                                                             // 8-row groups are 1024 bytes apart
+    // ------------------------------------------------------------------ MMA issuer (one thread)
+    constexpr uint32_t idesc = tc::idesc_bf16_f32(kQT, 128, 0, 0);     // S: Q and K both K-major, N = 128 tokens
+    constexpr uint32_t idesc_pv = tc::idesc_bf16_f32(kQT, kD, 0, 1);   // O: V is N-major, N = 128 channels
+    constexpr uint32_t hi = tc::smem_desc_hi_sw128(1024);              // 8-row groups are 1024 bytes apart everywhere
     bool ok = true;
     if (lane == 0) {
-      const uint32_t q_lo = tc::smem_desc_lo(q_u32, 16), k_lo = tc::smem_desc_lo(kv_u32, 16);
-      const uint32_t p_lo = tc::smem_desc_lo(p_u32, 16), v_lo = tc::smem_desc_lo(kv_u32 + kKBytes, kKT * 128);
-      auto issue_s = [&](int t, int j) {  // S_t = Q_t . K_j^T
-        const uint32_t qa = q_lo + t * (kQBytes >> 4), ka = k_lo + (j % kKVStages) * (kKVBytes >> 4);
-        const uint32_t d = tmem_base + (2 * t + (j & 1)) * kKT;
-        tc::mma_ss_halves<false>(d, qa, hi_k, ka, hi_k, idesc_s);
+      const uint32_t q_lo = tc::smem_desc_lo(q_u32, 16), k_lo = tc::smem_desc_lo(k_u32, 16);
+      const uint32_t v_lo = tc::smem_desc_lo(v_u32, kKT * 128);  // 64-channel chunks of V are one half tile apart
+      auto issue_s = [&](int t, int slot) {  // S_t = Q_t . K^T
+        const uint32_t qa = q_lo + t * (kQBytes >> 4), ka = k_lo + slot * (kTBytes >> 4);
+        const uint32_t d = tmem_base + t * 128;
+        tc::mma_ss_halves<false>(d, qa, hi, ka, hi, idesc);
 #pragma unroll
-        for (int ks = 1; ks < kD / 16; ++ks)
-          tc::mma_ss_halves<true>(d, qa + (((ks / 4) * (kQT * 128) + (ks % 4) * 32) >> 4), hi_k,
-                                  ka + (((ks / 4) * (kKT * 128) + (ks % 4) * 32) >> 4), hi_k, idesc_s);
-        tc::commit(s_full0 + 16 * t + 8 * (j & 1));
+        for (int ks = 1; ks < kD / 16; ++ks) {
+          const uint32_t step = ((ks / 4) * (128 * 128) + (ks % 4) * 32) >> 4;
+          tc::mma_ss_halves<true>(d, qa + step, hi, ka + step, hi, idesc);
+        }
+        tc::commit(s_full0 + 8 * t);
       };
-      auto issue_pv = [&](int t, int j) {  // O_t += P_t . V_j
-        const uint32_t pa = p_lo + t * (kPBytes >> 4), va = v_lo + (j % kKVStages) * (kKVBytes >> 4);
-        const uint32_t d = tmem_base + 256 + t * kD;
-        if (j == 0) tc::mma_ss_halves<false>(d, pa, hi_k, va, hi_k, idesc_pv);
-        else tc::mma_ss_halves<true>(d, pa, hi_k, va, hi_k, idesc_pv);
+      auto issue_pv = [&](int t, int slot, bool first) {  // O_t += P_t . V
+        const uint32_t va = v_lo + slot * (kTBytes >> 4);
+        const uint32_t d = tmem_base + 256 + t * kD, pa = tmem_base + t * 128;
+        if (first) tc::mma_ts_halves<false>(d, pa, va, hi, idesc_pv);
+        else tc::mma_ts_halves<true>(d, pa, va, hi, idesc_pv);
 #pragma unroll
-        for (int k = 1; k < kKT / 16; ++k)
-          tc::mma_ss_halves<true>(d, pa + ((k * 32) >> 4), hi_k, va + ((k * 16 * 128) >> 4), hi_k, idesc_pv);
+        for (int k = 1; k < kKT / 16; ++k) tc::mma_ts_halves<true>(d, pa + k * 8, va + ((k * 16 * 128) >> 4), hi, idesc_pv);
         tc::commit(o_done0 + 8 * t);
       };
-      // The scores of a tile have two buffers per M-tile: S(t, j + 2) is issued as soon as the softmax warps have
-      // consumed S(t, j) (which p_full(t, j) implies), so S(t, j + 1) is ready long before they ask for it.
       ok = ptx::mbar_wait(q_full, 0, abort_flag);
-      for (int j = 0; j < min(2, nkv_max) && ok; ++j) {
-        ok = ptx::mbar_wait(k_full0 + 8 * j, 0, abort_flag);
-        if (!ok) break;
+      if (ok && nkv_max > 0) ok = ptx::mbar_wait(k_full0, 0, abort_flag);
+      if (ok && nkv_max > 0) {
         tc::fence_after_sync();
-        if (j < nkv[0]) issue_s(0, j);
-        if (j < nkv[1]) issue_s(1, j);
-        tc::commit(k_empty0 + 8 * j);  // K tile j is free once these products are done
+        if (nkv[0] > 0) issue_s(0, 0);
+        if (nkv[1] > 0) issue_s(1, 0);
+        tc::commit(k_empty0);  // K tile 0 is free once these products are done
       }
+      int ks = 1 % kKSlots, vs = 0;  // slot of K tile j + 1, slot of V tile j
+      uint32_t kph = 0, vph = 0;
       for (int j = 0; j < nkv_max && ok; ++j) {
-        const int st = j % kKVStages, st2 = (j + 2) % kKVStages;
-        const uint32_t ph = (j / kKVStages) & 1, ph2 = ((j + 2) / kKVStages) & 1;
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
           if (j < nkv[t]) {
-            if (!ptx::mbar_wait(p_full0 + 8 * t, j & 1, abort_flag) || !ptx::mbar_wait(v_full0 + 8 * st, ph, abort_flag)) {
+            if (!ptx::mbar_wait(p_full0 + 8 * t, j & 1, abort_flag) || !ptx::mbar_wait(v_full0 + 8 * vs, vph, abort_flag)) {
               ok = false;
               break;
             }
             tc::fence_after_sync();
-            issue_pv(t, j);
+            issue_pv(t, vs, j == 0);
           }
-          if (t == 1) tc::commit(v_empty0 + 8 * st);  // every MMA that reads V tile j has been issued
-          if (j + 2 < nkv[t]) {
-            if (!ptx::mbar_wait(k_full0 + 8 * st2, ph2, abort_flag)) { ok = false; break; }
+          if (t == 1) tc::commit(v_empty0 + 8 * vs);  // every MMA that reads V tile j has been issued
+          if (j + 1 < nkv[t]) {  // P_t of tile j has been consumed by then (same pipe, in order): S_t may be overwritten
+            if (!ptx::mbar_wait(k_full0 + 8 * ks, kph, abort_flag)) { ok = false; break; }
             tc::fence_after_sync();
-            issue_s(t, j + 2);
+            issue_s(t, ks);
           }
-          if (t == 1 && j + 2 < nkv_max) tc::commit(k_empty0 + 8 * st2);  // ... and every MMA that reads K tile j + 2
+          if (t == 1 && j + 1 < nkv_max) tc::commit(k_empty0 + 8 * ks);  // ... and every MMA that reads K tile j + 1
         }
+        if (++ks == kKSlots) { ks = 0; kph ^= 1; }
+        if (++vs == kVSlots) { vs = 0; vph ^= 1; }
       }
       if (!ok) report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
       tc::commit(drain);
@@ -273,80 +268,99 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       const int qrow = q0 + t * kQT + r;
       const int qpos = past + qrow;
       const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      const uint32_t s_taddr = lane_base + t * 128;  // scores, and P over their first 64 columns
       const uint32_t o_taddr = lane_base + 256 + t * kD;
-      unsigned char* prow = p_s + t * kPBytes + r * 128;
       float m_ref = -INFINITY, l = 0.f;
       bool ok = true;
       for (int j = 0; j < n; ++j) {
-        if (!wait_warp(s_full0 + 16 * t + 8 * (j & 1), (j >> 1) & 1, abort_flag)) { ok = false; break; }
-        const uint32_t s_taddr = lane_base + (2 * t + (j & 1)) * kKT;
+        if (!wait_warp(s_full0 + 8 * t, j & 1, abort_flag)) { ok = false; break; }
         tc::fence_after_sync();
-        uint32_t s[64];
-        tc::ld_32x32b_x32(s_taddr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-        tc::ld_32x32b_x32(s_taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-        tc::wait_ld();
         const int k0 = j * kKT;
         const bool diag = k0 + kKT - 1 > past + q0 + t * kQT;  // block-uniform: the tile reaches past some row's position
-        if (diag) {
+        // ---- pass 1: row maximum of the raw scores (scale > 0 keeps the order)
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-          for (int c = 0; c < 64; ++c)
-            if (k0 + c > qpos) s[c] = 0xff800000u;  // -inf: this token lies after the row's position
+        for (int c = 0; c < 2; ++c) {
+          uint32_t s[64];
+          tc::ld_32x32b_x32(s_taddr + c * 64, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+          tc::ld_32x32b_x32(s_taddr + c * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+          tc::wait_ld();
+          if (diag) {
+#pragma unroll
+            for (int e = 0; e < 64; ++e)
+              if (k0 + c * 64 + e > qpos) s[e] = 0xff800000u;  // -inf: this token lies after the row's position
+          }
+#pragma unroll
+          for (int e = 0; e < 64; e += 8) {  // four independent chains, three inputs per instruction
+            mx0 = max3(mx0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
+            mx1 = max3(mx1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
+            mx2 = max3(mx2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
+            mx3 = max3(mx3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
+          }
         }
-        // row maximum of the raw scores (scale > 0 keeps the order), three inputs per instruction
-        float mx_raw = __uint_as_float(s[0]);
-#pragma unroll
-        for (int c = 1; c < 63; c += 2) mx_raw = max3(mx_raw, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-        mx_raw = fmaxf(mx_raw, __uint_as_float(s[63]));
-        const float mx = mx_raw * p.scale_log2;
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
         float alpha = 1.f;
         const bool bump = mx > m_ref + kRescaleThreshold;  // true on the first tile (m_ref = -inf)
         if (bump) {
           alpha = exp2f(m_ref - mx);
           m_ref = mx;
         }
-        if (j > 0) {
+        if (j > 0 && __any_sync(0xffffffffu, bump)) {  // rescale this warp's rows of O in tensor memory
           if (!wait_warp(o_done0 + 8 * t, (j - 1) & 1, abort_flag)) { ok = false; break; }
           tc::fence_after_sync();
-          if (__any_sync(0xffffffffu, bump)) {  // rescale this warp's rows of O in tensor memory
 #pragma unroll 1
-            for (int c = 0; c < kD / 32; ++c) {
-              uint32_t o[32];
-              tc::ld_32x32b_x32(o_taddr + c * 32, o);
-              tc::wait_ld();
+          for (int c = 0; c < kD / 32; ++c) {
+            uint32_t o[32];
+            tc::ld_32x32b_x32(o_taddr + c * 32, o);
+            tc::wait_ld();
 #pragma unroll
-              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-              tc::st_32x32b_x32(o_taddr + c * 32, o);
-            }
-            tc::wait_st();
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tc::st_32x32b_x32(o_taddr + c * 32, o);
           }
+          tc::wait_st();
         }
         l *= alpha;
         const float neg_m = -m_ref;
-        // P = 2^(S - m_ref), rounded to bf16; row r of the tile, 16-byte chunks XORed with the row index
+        // ---- pass 2: P = 2^(S scale - m_ref) as packed bf16 over the scores already consumed; fp32 row sum
+        float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8) {
-          uint32_t w[4];
+        for (int c = 0; c < 4; ++c) {
+          uint32_t s[32];
+          tc::ld_32x32b_x32(s_taddr + c * 32, s);
+          tc::wait_ld();
+          if (diag) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float p0 = ex2(fmaf(__uint_as_float(s[c8 * 8 + 2 * e]), p.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(s[c8 * 8 + 2 * e + 1]), p.scale_log2, neg_m));
-            w[e] = pack2(p0, p1);
-            l += p0 + p1;
+            for (int e = 0; e < 32; ++e)
+              if (k0 + c * 32 + e > qpos) s[e] = 0xff800000u;
           }
-          *reinterpret_cast<uint4*>(prow + ((c8 ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+          uint32_t w[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float p0 = ex2(fmaf(__uint_as_float(s[2 * e]), p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(s[2 * e + 1]), p.scale_log2, neg_m));
+            w[e] = pack2(p0, p1);
+            l0 += p0;
+            l1 += p1;
+          }
+          tc::st_32x32b_x16(s_taddr + c * 16, w);  // columns 16c .. 16c+15: scores 0 .. 32c+31 are consumed
         }
+        l += l0 + l1;
         if (j == nkv_max - 1 && (kv_len & (kKT - 1)) != 0) {
           // ragged last tile: V rows past the sequence end hold whatever followed in memory; zero them
           // (0 * NaN would poison the product).  Both M-tiles may do this; they write the same zeros.
-          if (!wait_warp(v_full0 + 8 * (j % kKVStages), (j / kKVStages) & 1, abort_flag)) { ok = false; break; }
-          const int row = r & 63, half = r >> 6;
-          if (row >= kv_len - k0) {
-            uint4* dst = reinterpret_cast<uint4*>(kv_s + (j % kKVStages) * kKVBytes + kKBytes + half * (kKT * 128) + row * 128);
+          const int vslot = j % kVSlots;
+          if (!wait_warp(v_full0 + 8 * vslot, (j / kVSlots) & 1, abort_flag)) { ok = false; break; }
+          if (r >= kv_len - k0) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) dst[e] = make_uint4(0, 0, 0, 0);
+            for (int half = 0; half < 2; ++half) {
+              uint4* dst = reinterpret_cast<uint4*>(v_s + vslot * kTBytes + half * (kKT * 128) + r * 128);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) dst[e] = make_uint4(0, 0, 0, 0);
+            }
           }
+          ptx::fence_proxy_async();
         }
-        ptx::fence_proxy_async();
+        tc::wait_st();
         tc::fence_before_sync();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(p_full0 + 8 * t);
