@@ -292,6 +292,17 @@ def time_prefill(api, W, device, peaks, steps):
     return res
 
 
+def max_over_ranks(value: float, device) -> float:
+    """The slowest rank's value (all-reduce MAX over the default process group; identity without one)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def run_ours(args):
     import torch
     from paper_2501_13629_b200 import api, workloads as W
@@ -320,11 +331,7 @@ def run_ours(args):
         ms = case.time_steps(args.steps, args.warmup, barrier)
     launches = api.launch_count() - launches0 - 0
     launches_timed = launches * args.steps // (args.steps + args.warmup)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, device)
     assert int(case.status.item()) == 0, "device status reported an error"
     ms_per_step = ms / args.steps
     value = world * case.bytes / (ms_per_step * 1e-3) / 1e9
@@ -434,7 +441,7 @@ def run_reference(args):
     host = W.make_decode_inputs(cfg)
     pairs = _all_pairs(cfg)
     t_row = _time_oracle_pairs(oracle, host, pairs[:cores]) / 1.0  # wall time of `cores` rows in parallel
-    budget = 150.0
+    budget = float(args.budget_s)
     total_steps = args.steps + args.warmup
     per_step_rows = int(max(1, min(len(pairs), (budget / total_steps / max(t_row, 1e-6)) * cores)))
     sample = pairs[:per_step_rows]
@@ -469,6 +476,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="headline workload only")
+    ap.add_argument("--budget-s", type=float, default=150.0,
+                    help="--impl reference: seconds of oracle time the whole run may take (sizes the per-step sample)")
     ap.add_argument("--workload", default="decode", choices=["decode", "prefill"],
                     help="decode = the headline line (default); prefill = only the config 4 timings")
     ap.add_argument("--profile", action="store_true",

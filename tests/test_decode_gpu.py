@@ -257,3 +257,34 @@ def test_dominant_and_uniform_softmax(api, oracle):
     ref2, _ = run_oracle(oracle, inp2)
     out2, _, _ = run_decode(api, inp2)
     check_bf16(out2, ref2, "dominant")
+
+
+def test_config5_full_size_sampled_rows(api, oracle):
+    """Config 5 at its full size (64 sequences, lengths uniform in [1024, 65536], 16-token pages, shuffled page
+    table, 6.4 GB of cache) in the launch configuration the benchmark times; the oracle recomputes a sample of
+    (sequence, query head) rows from the same bytes copied back to the host."""
+    import bench
+    cfg = W.CFG5
+    case = bench.DecodeCase(api, cfg, torch.device("cuda", 0))
+    lse = torch.full((cfg.batch, cfg.n_q), float("nan"), dtype=torch.float32, device="cuda")
+    out = torch.empty((cfg.batch, cfg.n_q, cfg.d_v), dtype=torch.float32, device="cuda")
+    cache = case.caches[0]
+    api.diffqkv_decode(case.q, cache, cfg.n_k, cfg.n_v, cfg.scale, workspace=case.workspace, out=out, lse=lse,
+                       dev_status=case.status)
+    torch.cuda.synchronize()
+    assert int(case.status.item()) == 0 and api.last_decode_kernel() == api.KERNEL_TMA
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    k_host = cache.k.view(torch.uint16).cpu().numpy()
+    v_host = cache.v.view(torch.uint16).cpu().numpy()
+    q_host = case.q.view(torch.uint16).cpu().numpy()
+    lens = case.seqlens_host
+    ks, vs = tuple(cache.k.stride()[:3]), tuple(cache.v.stride()[:3])
+    ocache = oracle.Cache(k_host, v_host, ks, vs, lens, cache.page_table.cpu().numpy(), cfg.page_size)
+    g = np.random.Generator(np.random.Philox(key=555))
+    seqs = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 0, cfg.batch - 1, *g.integers(0, cfg.batch, 4).tolist()})
+    pairs = np.array([(b, h) for b in seqs for h in g.choice(cfg.n_q, 4, replace=False)], dtype=np.int32)
+    ref, lse_ref = oracle.decode(q_host, ocache, cfg.n_q, cfg.n_k, cfg.n_v, cfg.d_qk, cfg.d_v, cfg.scale, pairs=pairs)
+    sel = (pairs[:, 0], pairs[:, 1])
+    check_bf16(got[sel], ref[sel], "cfg5 full size")
+    check_lse(lse.cpu().numpy().astype(np.float64)[sel], lse_ref[sel], 2e-2, "cfg5 full size")
