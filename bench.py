@@ -276,8 +276,10 @@ def time_prefill(api, W, device, peaks, steps):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / steps
 
-    augq_ms = timed(lambda: api.diffqkv_augq(h, w_q, w_g, w_u, w_d, workspace=ws, q_out=q, dev_status=status))
-    attn_ms = timed(lambda: api.diffqkv_prefill(q4, k_new, v_new, cache, cfg.scale, out=out, dev_status=status))
+    with ClockSampler(device.index or 0) as ck_a:
+        augq_ms = timed(lambda: api.diffqkv_augq(h, w_q, w_g, w_u, w_d, workspace=ws, q_out=q, dev_status=status))
+    with ClockSampler(device.index or 0) as ck_p:
+        attn_ms = timed(lambda: api.diffqkv_prefill(q4, k_new, v_new, cache, cfg.scale, out=out, dev_status=status))
     assert int(status.item()) == 0, "device status reported an error"
     augq_flops = 2.0 * T * (cfg.d_model * d_q0 + 2 * d_q0 * cfg.d_aug + cfg.d_aug * d_q0)
     attn_flops = 2.0 * cfg.batch * cfg.n_q * (cfg.seq * (cfg.seq + 1) / 2) * (cfg.d_qk + cfg.d_v)
@@ -287,6 +289,7 @@ def time_prefill(api, W, device, peaks, steps):
         res[name] = {"ms": ms, "TFLOP/s": tf, "flops": fl, "bound": "tensor",
                      "frac_of_measured_bf16_burst": tf / peaks["bf16_tflops"],
                      "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"]}
+    res["augq"]["clocks"], res["attention"]["clocks"] = ck_a.summary(), ck_p.summary()
     res["attention"]["note"] = "causal flops (lower triangle incl. diagonal); time includes the cache-update kernel"
     res["working_set"] = "weights 92 MB + activations 0.5 GB per step: larger than L2"
     return res
