@@ -295,6 +295,27 @@ def time_prefill(api, W, device, peaks, steps):
     return res
 
 
+def time_sigma_table(api, W, device, steps):
+    """The paper's own efficiency experiment in shape: SIGMA-1.5B attention heads (32 query, 4 K, 16 V heads, head
+    dimension 64) against the standard model's 16 K / 16 V heads at prefix lengths 2k, 4k, 16k and 32k (batch 8,
+    bf16 cache drawn on the device): time of one decode step and the share of it the split kernel takes."""
+    import dataclasses
+    rows = []
+    for prefix in (2048, 4096, 16384, 32768):
+        row = {"prefix": prefix}
+        for name, n_k, n_v in (("sigma", 4, 16), ("std", 16, 16)):
+            cfg = dataclasses.replace(W.SIGMA15B, name=f"{name}_{prefix}", batch=8, n_k=n_k, n_v=n_v, kv_len=prefix)
+            case = DecodeCase(api, cfg, device)
+            ms = case.time_steps(steps, 20) / steps
+            row[name] = {"us_per_step": ms * 1e3, "GB/s": case.bytes / ms / 1e6, "kv_bytes": case.bytes,
+                         "rotate": case.rotate}
+            del case
+        row["time_reduction_pct"] = 100.0 * (1.0 - row["sigma"]["us_per_step"] / row["std"]["us_per_step"])
+        row["bytes_reduction_pct"] = 100.0 * (1.0 - row["sigma"]["kv_bytes"] / row["std"]["kv_bytes"])
+        rows.append(row)
+    return rows
+
+
 def max_over_ranks(value: float, device) -> float:
     """The slowest rank's value (all-reduce MAX over the default process group; identity without one)."""
     import torch
@@ -392,6 +413,8 @@ def run_ours(args):
             del c5
             torch.cuda.empty_cache()
             others[W.CFG4.name] = time_prefill(api, W, device, peaks, max(5, min(args.steps, 20)))
+            torch.cuda.empty_cache()
+            others["sigma1p5b_vs_std_heads"] = time_sigma_table(api, W, device, max(20, min(args.steps, 300)))
         line["others"] = others
         line["cpu_baseline"] = cpu_baseline(host, budget_s=12.0)
         print(json.dumps(line))
