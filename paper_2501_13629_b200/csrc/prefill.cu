@@ -277,26 +277,23 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         tc::fence_after_sync();
         const int k0 = j * kKT;
         const bool diag = k0 + kKT - 1 > past + q0 + t * kQT;  // block-uniform: the tile reaches past some row's position
-        // ---- pass 1: row maximum of the raw scores (scale > 0 keeps the order)
+        // ---- all 128 scores of the row into registers; row maximum of the raw scores (scale > 0 keeps the order)
+        uint32_t s[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tc::ld_32x32b_x32(s_taddr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+        tc::wait_ld();
+        if (diag) {
+#pragma unroll
+          for (int e = 0; e < 128; ++e)
+            if (k0 + e > qpos) s[e] = 0xff800000u;  // -inf: this token lies after the row's position
+        }
         float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t s[64];
-          tc::ld_32x32b_x32(s_taddr + c * 64, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-          tc::ld_32x32b_x32(s_taddr + c * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-          tc::wait_ld();
-          if (diag) {
-#pragma unroll
-            for (int e = 0; e < 64; ++e)
-              if (k0 + c * 64 + e > qpos) s[e] = 0xff800000u;  // -inf: this token lies after the row's position
-          }
-#pragma unroll
-          for (int e = 0; e < 64; e += 8) {  // four independent chains, three inputs per instruction
-            mx0 = max3(mx0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
-            mx1 = max3(mx1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
-            mx2 = max3(mx2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
-            mx3 = max3(mx3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
-          }
+        for (int e = 0; e < 128; e += 8) {  // four independent chains, three inputs per instruction
+          mx0 = max3(mx0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
+          mx1 = max3(mx1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
+          mx2 = max3(mx2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
+          mx3 = max3(mx3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
         }
         const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
         float alpha = 1.f;
@@ -321,28 +318,20 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         }
         l *= alpha;
         const float neg_m = -m_ref;
-        // ---- pass 2: P = 2^(S scale - m_ref) as packed bf16 over the scores already consumed; fp32 row sum
+        // ---- P = 2^(S scale - m_ref) as packed bf16 over the first 64 score columns; fp32 row sum
         float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t s[32];
-          tc::ld_32x32b_x32(s_taddr + c * 32, s);
-          tc::wait_ld();
-          if (diag) {
+        for (int c = 0; c < 2; ++c) {
+          uint32_t w[32];
 #pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (k0 + c * 32 + e > qpos) s[e] = 0xff800000u;
-          }
-          uint32_t w[16];
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float p0 = ex2(fmaf(__uint_as_float(s[2 * e]), p.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(s[2 * e + 1]), p.scale_log2, neg_m));
+          for (int e = 0; e < 32; ++e) {
+            const float p0 = ex2(fmaf(__uint_as_float(s[c * 64 + 2 * e]), p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(s[c * 64 + 2 * e + 1]), p.scale_log2, neg_m));
             w[e] = pack2(p0, p1);
             l0 += p0;
             l1 += p1;
           }
-          tc::st_32x32b_x16(s_taddr + c * 16, w);  // columns 16c .. 16c+15: scores 0 .. 32c+31 are consumed
+          tc::st_32x32b_x32(s_taddr + c * 32, w);
         }
         l += l0 + l1;
         if (j == nkv_max - 1 && (kv_len & (kKT - 1)) != 0) {
