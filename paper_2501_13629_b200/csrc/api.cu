@@ -9,11 +9,13 @@ static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 DecodePlan plan_decode(const diffqkv_shape& shape, int max_seqlen, int num_splits) {
-  (void)shape;
   if (max_seqlen < 1) max_seqlen = 1;
   int want = num_splits;
-  if (want <= 0) {  // automatic: chunks of about 512 tokens, at most 32 splits
+  if (want <= 0) {  // automatic: chunks of about 512 tokens, shorter when that leaves most SMs idle; at most 32 splits
     want = (max_seqlen + 511) / 512;
+    const long long rows = (long long)shape.batch * shape.n_q;
+    const long long fill = rows > 0 ? (592 + rows - 1) / rows : 1;  // about four blocks per SM
+    if (want < fill) want = (int)fill;
     if (want > 32) want = 32;
   }
   if (want < 1) want = 1;
