@@ -316,6 +316,23 @@ def time_sigma_table(api, W, device, steps):
     return rows
 
 
+def time_context_sweep(api, W, device, steps):
+    """DiffQKV (32 query / 4 K / 8 V heads) against its GQA twin (8 K / 8 V heads) over the context length, batch 4,
+    d 128, bf16 cache drawn on the device: one decode step each; the bytes model predicts 25 % less time."""
+    import dataclasses
+    rows = []
+    for ctx in (4096, 8192, 16384, 32768, 65536, 131072):
+        row = {"context": ctx}
+        for name, cfg in (("diffqkv", W.CFG3), ("gqa", W.CFG3.gqa_twin())):
+            case = DecodeCase(api, dataclasses.replace(cfg, name=f"{name}_{ctx}", kv_len=ctx), device)
+            ms = case.time_steps(steps, 20) / steps
+            row[name] = {"us_per_step": ms * 1e3, "GB/s": case.bytes / ms / 1e6, "rotate": case.rotate}
+            del case
+        row["speedup"] = row["gqa"]["us_per_step"] / row["diffqkv"]["us_per_step"]
+        rows.append(row)
+    return rows
+
+
 def max_over_ranks(value: float, device) -> float:
     """The slowest rank's value (all-reduce MAX over the default process group; identity without one)."""
     import torch
@@ -415,6 +432,8 @@ def run_ours(args):
             others[W.CFG4.name] = time_prefill(api, W, device, peaks, max(5, min(args.steps, 20)))
             torch.cuda.empty_cache()
             others["sigma1p5b_vs_std_heads"] = time_sigma_table(api, W, device, max(20, min(args.steps, 300)))
+            torch.cuda.empty_cache()
+            others["diffqkv_vs_gqa_over_context"] = time_context_sweep(api, W, device, max(20, min(args.steps, 200)))
         line["others"] = others
         line["cpu_baseline"] = cpu_baseline(host, budget_s=12.0)
         print(json.dumps(line))
