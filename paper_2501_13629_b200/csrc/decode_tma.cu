@@ -4,7 +4,8 @@
 // Work decomposition.  Query heads are handled in "units": U = n_q / min(n_k, n_v) consecutive query
 // heads that share K heads and V heads among themselves only (Eq. (idx) of the paper makes the head
 // maps contiguous blocks).  A unit holds KPU = n_k / min K heads and VPU = n_v / min V heads, one of
-// the two being 1.  The sequence axis is cut into tiles of 64 tokens.  All (sequence, unit, tile)
+// the two being 1; where that makes tiles smaller than 32 KB, up to four neighbouring units are taken
+// together as one.  The sequence axis is cut into tiles of 64 tokens.  All (sequence, unit, tile)
 // triples, in that order, form one flat list that is divided evenly over the persistent blocks of
 // the grid; a maximal run of one block's tiles inside one (sequence, unit) is a segment and yields
 // one partial result (or the final result when the segment covers the whole sequence).
@@ -650,6 +651,7 @@ bool pick_variant(int d_qk, int d_v, int kpu, int vpu, Variant* v) {
   DIFFQKV_CASE(64, 64, 1, 1) DIFFQKV_CASE(64, 64, 1, 2) DIFFQKV_CASE(64, 64, 1, 4)
   DIFFQKV_CASE(64, 64, 2, 1) DIFFQKV_CASE(64, 64, 4, 1)
   DIFFQKV_CASE(64, 128, 1, 1) DIFFQKV_CASE(64, 128, 1, 2)
+  DIFFQKV_CASE(64, 64, 2, 2) DIFFQKV_CASE(64, 64, 4, 4) DIFFQKV_CASE(64, 64, 2, 4) DIFFQKV_CASE(64, 64, 4, 2)
 #undef DIFFQKV_CASE
   return false;
 }
@@ -660,10 +662,23 @@ bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPla
   if (s.dtype != DIFFQKV_BF16) return false;
   const int mn = s.n_k < s.n_v ? s.n_k : s.n_v;
   if (s.n_k % mn != 0 || s.n_v % mn != 0) return false;
-  const int U = s.n_q / mn, kpu = s.n_k / mn, vpu = s.n_v / mn;
+  int U = s.n_q / mn, kpu = s.n_k / mn, vpu = s.n_v / mn;
   if (U > kHeadsPerMma || s.batch > kMaxBatchTma || s.batch < 1) return false;
   Variant v;
   if (!pick_variant(s.d_qk, s.d_v, kpu, vpu, &v)) return false;
+  // Small units make small tiles (16-24 KB per 64 tokens at d = 64), and the fixed cost per tile then shows.  Several
+  // neighbouring units can share a tile: m units are one unit of m*U query heads with m*KPU K heads and m*VPU V
+  // heads (the head maps are contiguous blocks, so nothing else changes).  Merge while the tile stays within 64 KB.
+  if (v.stage_bytes < 32768) {
+    for (int m = 4; m >= 2; m >>= 1) {
+      Variant vm;
+      if (U * m <= kHeadsPerMma && mn % m == 0 && pick_variant(s.d_qk, s.d_v, kpu * m, vpu * m, &vm) &&
+          vm.stage_bytes <= 65536) {
+        U *= m; kpu *= m; vpu *= m; v = vm;
+        break;
+      }
+    }
+  }
   int box_tok = kTT;
   if (c.page_table) {
     if (c.page_size % 16 != 0) return false;
