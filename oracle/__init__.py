@@ -220,6 +220,37 @@ def augq(h: np.ndarray, W_Q: np.ndarray, W_gate: np.ndarray, W_up: np.ndarray, W
     return out
 
 
+def linear(x: np.ndarray, W: np.ndarray) -> np.ndarray:
+    """y = x W^T (W is [out, in], no bias) in float64 from the stored values."""
+    dt = _dtype_code(x)
+    assert _dtype_code(W) == dt
+    x, W = np.ascontiguousarray(x), np.ascontiguousarray(W)
+    T, d_in = x.shape
+    d_out = W.shape[0]
+    assert W.shape == (d_out, d_in)
+    y = np.zeros((T, d_out), dtype=np.float64)
+    lib().oracle_linear(_ptr(x), _ptr(W), C.c_int64(T), d_in, d_out, dt, _ptr(y))
+    return y
+
+
+def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
+    """Rotary embedding (rotate-half pairing) of x [T, n_heads, d] float64 at positions pos [T]; returns a copy."""
+    y = np.array(x, dtype=np.float64, order="C", copy=True)
+    T, n_heads, d = y.shape
+    assert d % 2 == 0
+    pos = np.ascontiguousarray(pos, dtype=np.int64)
+    assert pos.shape == (T,)
+    lib().oracle_rope(_ptr(y), _ptr(pos), C.c_int64(T), n_heads, d, C.c_double(theta))
+    return y
+
+
+def rope_tables(pos: np.ndarray, d: int, theta: float):
+    """cos and sin of the rotary angles, float64 [T, d/2]: the tables a caller hands to the GPU entry points."""
+    i = np.arange(d // 2, dtype=np.float64)
+    ang = np.asarray(pos, dtype=np.float64)[:, None] * np.power(float(theta), -2.0 * i / d)[None, :]
+    return np.cos(ang), np.sin(ang)
+
+
 def kv_bytes(seqlens: np.ndarray, n_k: int, n_v: int, d_qk: int, d_v: int, elt_bytes: int) -> float:
     """Bytes of K and V cache the method must stream once (the paper's cache cost model, alpha = element size)."""
     seqlens = np.ascontiguousarray(seqlens, dtype=np.int32)

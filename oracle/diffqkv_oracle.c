@@ -33,6 +33,9 @@
  * key returns its V row within (len-1)e^-gap, a pure-Python brute force on tiny
  * shapes, split/combine invariance, page-table invariance, prefill row i equals
  * decode at length i+1, and hand-worked tiny cases for the augmented Q.
+ * oracle_linear and oracle_rope (the projections and the rotary embedding around the cache update) are pinned
+ * by a library matmul, by closed forms and by the relative-position identity; that the rotary embedding uses the
+ * rotate-half pairing is a reading (the listing only names the call): "parity unpinned" for that choice.
  * The choice of SiLU as act_fn is a reading of the paper, not pinned by it:
  * for oracle_augq the activation choice is "parity unpinned" (the rest of the
  * chain is pinned by closed forms).
@@ -289,6 +292,41 @@ void oracle_augq(const void *h, const void *W_Q, const void *W_gate, const void 
     free(x);
     free(a);
   }
+}
+
+/* Plain projection (attention listing: k_proj, v_proj, q_proj): y = x W^T with W in the nn.Linear layout
+ * [out_features, in_features], no bias.  x [T, d_in] in the storage dtype, y [T, d_out] double. */
+void oracle_linear(const void *x, const void *W, int64_t T, int d_in, int d_out, int dtype, double *y) {
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < T; ++t)
+    for (int o = 0; o < d_out; ++o) {
+      double acc = 0.0;
+      for (int i = 0; i < d_in; ++i) acc += load_elt(x, t * d_in + i, dtype) * load_elt(W, (int64_t)o * d_in + i, dtype);
+      y[t * d_out + o] = acc;
+    }
+}
+
+/* Rotary position embedding of the attention listing (apply_rotary_pos_emb(q, k, cos, sin)), read as the
+ * rotate-half convention of the model family the listing derives from: within a head of width d, channel i < d/2
+ * pairs with channel i + d/2,
+ *     y_i       = x_i cos_i - x_{i+d/2} sin_i
+ *     y_{i+d/2} = x_{i+d/2} cos_i + x_i sin_i,
+ * with the angle of pair i at position pos being pos * theta^(-2 i / d) (the paper's model table gives
+ * theta = 50 000 and 500 000).  x is [T, n_heads, d] double, rotated in place; pos is [T]. */
+void oracle_rope(double *x, const int64_t *pos, int64_t T, int n_heads, int d, double theta) {
+  int half = d / 2;
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < T; ++t)
+    for (int h = 0; h < n_heads; ++h) {
+      double *v = x + (t * n_heads + h) * d;
+      for (int i = 0; i < half; ++i) {
+        double ang = (double)pos[t] * pow(theta, -2.0 * i / d);
+        double c = cos(ang), s = sin(ang);
+        double a = v[i], b = v[i + half];
+        v[i] = a * c - b * s;
+        v[i + half] = b * c + a * s;
+      }
+    }
 }
 
 /* KV-cache cost model, Eq. (cache_0) with alpha = element size, beta = 0:

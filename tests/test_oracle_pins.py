@@ -364,6 +364,64 @@ def test_augq_matches_library_matmul(oracle, dtype):
     assert np.array_equal(oracle.augq(h, wq, wg, wu, wd, rows=rows), out[rows])
 
 
+# --------------------------------------------------------------------------- projections and rotary embedding
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_linear_matches_library_matmul(oracle, dtype):
+    x, w = _rand(1, (7, 12), dtype), _rand(2, (5, 12), dtype)
+    ref = torch.from_numpy(W.as_f64(x)) @ torch.from_numpy(W.as_f64(w)).T
+    assert np.allclose(oracle.linear(x, w), ref.numpy(), rtol=1e-13, atol=1e-13)
+    # one-hot input picks a column of W^T
+    e = np.zeros((1, 12), np.float32)
+    e[0, 3] = 1.0
+    assert np.array_equal(oracle.linear(e, _rand(2, (5, 12))), W.as_f64(_rand(2, (5, 12)))[:, 3][None])
+
+
+def test_rope_closed_forms(oracle):
+    d, theta = 8, 50000.0
+    x = np.random.default_rng(3).standard_normal((6, 3, d))
+    pos = np.array([0, 1, 2, 7, 100, 4095])
+    y = oracle.rope(x, pos, theta)
+    assert np.array_equal(y[0], x[0])  # position 0 rotates by nothing
+    assert np.allclose(np.linalg.norm(y, axis=-1), np.linalg.norm(x, axis=-1), rtol=1e-13)  # a rotation
+    # pair 0 turns by exactly `pos` radians (theta^0 = 1): check one element by hand
+    t, h = 3, 1
+    a, b = x[t, h, 0], x[t, h, d // 2]
+    assert abs(y[t, h, 0] - (a * math.cos(7.0) - b * math.sin(7.0))) < 1e-14
+    assert abs(y[t, h, d // 2] - (b * math.cos(7.0) + a * math.sin(7.0))) < 1e-14
+    # the last pair turns by pos * theta^(-2 (d/2 - 1) / d)
+    ang = 100.0 * theta ** (-2.0 * (d // 2 - 1) / d)
+    a, b = x[4, 0, d // 2 - 1], x[4, 0, d - 1]
+    assert abs(y[4, 0, d // 2 - 1] - (a * math.cos(ang) - b * math.sin(ang))) < 1e-13
+    # tables are the same angles
+    c, s_ = oracle.rope_tables(pos, d, theta)
+    assert abs(c[4, d // 2 - 1] - math.cos(ang)) < 1e-15 and abs(s_[3, 0] - math.sin(7.0)) < 1e-15
+
+
+def test_rope_scores_depend_on_relative_position_only(oracle):
+    d, theta = 16, 500000.0
+    rng = np.random.default_rng(5)
+    q, k = rng.standard_normal((1, 1, d)), rng.standard_normal((1, 1, d))
+    dots = []
+    for m, n in ((10, 3), (107, 100), (5007, 5000)):
+        dots.append(float(np.sum(oracle.rope(q, np.array([m]), theta) * oracle.rope(k, np.array([n]), theta))))
+    assert max(dots) - min(dots) < 1e-9
+    other = float(np.sum(oracle.rope(q, np.array([10]), theta) * oracle.rope(k, np.array([4]), theta)))
+    assert abs(other - dots[0]) > 1e-6  # and they do depend on it
+
+
+def test_rope_is_the_complex_rotation(oracle):
+    """Pair (x_i, x_{i+d/2}) as a complex number is multiplied by e^{i angle}: numpy's complex arithmetic."""
+    d, theta = 32, 50000.0
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal((5, 2, d))
+    pos = np.array([1, 17, 300, 9999, 65535])
+    z = x[..., : d // 2] + 1j * x[..., d // 2:]
+    ang = pos[:, None] * theta ** (-2.0 * np.arange(d // 2) / d)[None, :]
+    zr = z * np.exp(1j * ang)[:, None, :]
+    ref = np.concatenate([zr.real, zr.imag], axis=-1)
+    assert np.allclose(oracle.rope(x, pos, theta), ref, rtol=0, atol=1e-12)
+
+
 # --------------------------------------------------------------------------- cost model
 def test_cache_cost_model_matches_paper(oracle):
     """Eq. (imp_t): SIGMA-1.5B against the 16/16 GQA model saves (32-20)/32 of the cache traffic."""
