@@ -281,6 +281,24 @@ def time_prefill(api, W, device, peaks, steps):
     with ClockSampler(device.index or 0) as ck_p:
         attn_ms = timed(lambda: api.diffqkv_prefill(q4, k_new, v_new, cache, cfg.scale, out=out, dev_status=status))
     assert int(status.item()) == 0, "device status reported an error"
+    # the projections around it in the listing: k = rope(h W_K^T), v = h W_V^T (rotary tables for positions 0 .. seq - 1)
+    w_k = rn(cfg.n_k * cfg.d_qk, cfg.d_model, std=cfg.d_model ** -0.5)
+    w_v = rn(cfg.n_v * cfg.d_v, cfg.d_model, std=cfg.d_model ** -0.5)
+    pos = torch.arange(cfg.seq, device=device, dtype=torch.float64).repeat(cfg.batch)
+    inv = torch.pow(torch.tensor(50000.0, dtype=torch.float64, device=device),
+                    -2.0 * torch.arange(cfg.d_qk // 2, device=device, dtype=torch.float64) / cfg.d_qk)
+    ang = pos[:, None] * inv[None, :]
+    cos, sin = torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()
+    k_out = torch.empty(T, cfg.n_k * cfg.d_qk, dtype=torch.bfloat16, device=device)
+    v_out = torch.empty(T, cfg.n_v * cfg.d_v, dtype=torch.bfloat16, device=device)
+
+    def kv_proj():
+        api.diffqkv_project(h, w_k, cfg.d_qk, cos, sin, out=k_out, dev_status=status)
+        api.diffqkv_project(h, w_v, out=v_out, dev_status=status)
+
+    kv_ms = timed(kv_proj)
+    augq_rope_ms = timed(lambda: api.diffqkv_augq_rope(h, w_q, w_g, w_u, w_d, cfg.d_qk, cos, sin, workspace=ws, q_out=q,
+                                                       dev_status=status))
     augq_flops = 2.0 * T * (cfg.d_model * d_q0 + 2 * d_q0 * cfg.d_aug + cfg.d_aug * d_q0)
     attn_flops = 2.0 * cfg.batch * cfg.n_q * (cfg.seq * (cfg.seq + 1) / 2) * (cfg.d_qk + cfg.d_v)
     res = {}
@@ -290,6 +308,10 @@ def time_prefill(api, W, device, peaks, steps):
                      "frac_of_measured_bf16_burst": tf / peaks["bf16_tflops"],
                      "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"]}
     res["augq"]["clocks"], res["attention"]["clocks"] = ck_a.summary(), ck_p.summary()
+    kv_flops = 2.0 * T * cfg.d_model * (cfg.n_k * cfg.d_qk + cfg.n_v * cfg.d_v)
+    res["kv_projection_rope"] = {"ms": kv_ms, "TFLOP/s": kv_flops / kv_ms / 1e9, "flops": kv_flops,
+                                 "note": "k = rope(h W_K^T) and v = h W_V^T, two launches"}
+    res["augq_rope"] = {"ms": augq_rope_ms, "TFLOP/s": augq_flops / augq_rope_ms / 1e9}
     res["attention"]["note"] = "causal flops (lower triangle incl. diagonal); time includes the cache-update kernel"
     res["working_set"] = "weights 92 MB + activations 0.5 GB per step: larger than L2"
     return res

@@ -195,6 +195,44 @@ diffqkv_status diffqkv_augq(const void *h, const void *W_Q, const void *W_gate, 
                             int32_t d_out, void *workspace, size_t workspace_bytes, void *q_out,
                             int32_t *dev_status, void *stream);
 
+/*
+ * diffqkv_augq_rope -- diffqkv_augq followed by the rotary position embedding of the appendix attention listing
+ * (apply_rotary_pos_emb on the query), fused into the last product's epilogue: the rotation acts on the fp32
+ * result before it is rounded to bf16.  The listing only names the call; it is read as the rotate-half pairing:
+ * within a head of width head_dim, channel i < head_dim/2 pairs with channel i + head_dim/2,
+ *     y_i = x_i cos[t, i] - x_{i+head_dim/2} sin[t, i],   y_{i+head_dim/2} = x_{i+head_dim/2} cos[t, i] + x_i sin[t, i].
+ *   cos, sin  [T, head_dim / 2] fp32 tables of the caller (angle of pair i at position pos: pos * theta^(-2 i / head_dim));
+ *             both NULL = no rotation
+ *   head_dim  64 or 128; d_out must be a multiple of it
+ * Everything else as diffqkv_augq.
+ */
+diffqkv_status diffqkv_augq_rope(const void *h, const void *W_Q, const void *W_gate, const void *W_up,
+                                 const void *W_down, int64_t T, int32_t d_model, int32_t d_q0, int32_t d_aug,
+                                 int32_t d_out, int32_t head_dim, const float *cos, const float *sin, void *workspace,
+                                 size_t workspace_bytes, void *q_out, int32_t *dev_status, void *stream);
+
+/*
+ * diffqkv_project -- a plain projection of the attention listing (k_proj, v_proj): y = x W^T with W in the
+ * nn.Linear layout [d_out, d_in], no bias, on the tensor cores with fp32 accumulation; with cos / sin given, the
+ * rotary embedding above is applied per head before rounding (the key projection), without them it is a plain
+ * product (the value projection).
+ *   x [T, d_in] bf16   W [d_out, d_in] bf16   y [T, d_out] bf16   d_in and d_out multiples of 128
+ * The result [T, n_heads, head_dim] is the k_new / v_new layout of diffqkv_prefill and diffqkv_cache_append.
+ */
+diffqkv_status diffqkv_project(const void *x, const void *W, int64_t T, int32_t d_in, int32_t d_out, int32_t head_dim,
+                               const float *cos, const float *sin, void *y, int32_t *dev_status, void *stream);
+
+/*
+ * diffqkv_cache_append -- the cache update of the attention listing on its own (diffqkv_prefill does the same
+ * before it attends): k_new [batch, q_len, n_k, d_qk] and v_new [batch, q_len, n_v, d_v] are written to token
+ * positions seqlens[b] .. seqlens[b] + q_len - 1 of the pools (any strides, paged or contiguous, bf16 or fp32).
+ * seqlens itself is not modified.  Positions at or past max_seqlen, and page ids outside the pool, are skipped
+ * and reported as DIFFQKV_ERR_INDEX in *dev_status.  A decode step is: append the new token's rows, add 1 to
+ * seqlens, call diffqkv_decode.
+ */
+diffqkv_status diffqkv_cache_append(const void *k_new, const void *v_new, int32_t q_len, const diffqkv_cache *cache,
+                                    const diffqkv_shape *shape, int32_t *dev_status, void *stream);
+
 /* Static, never-null description of a status value. */
 const char *diffqkv_status_string(diffqkv_status status);
 

@@ -29,7 +29,8 @@ EXPORTS = (
     "diffqkv_decode_num_splits", "diffqkv_decode_workspace_bytes", "diffqkv_decode", "gqa_decode",
     "diffqkv_combine", "diffqkv_prefill", "diffqkv_augq_workspace_bytes", "diffqkv_augq",
     "diffqkv_status_string", "diffqkv_launch_count", "diffqkv_profile_split_events", "diffqkv_decode_static",
-    "diffqkv_set_max_blocks", "diffqkv_last_decode_kernel",
+    "diffqkv_set_max_blocks", "diffqkv_last_decode_kernel", "diffqkv_augq_rope", "diffqkv_project",
+    "diffqkv_cache_append",
 )
 
 
@@ -75,6 +76,16 @@ _lib.diffqkv_augq_workspace_bytes.argtypes = [C.c_int64, C.c_int32, C.c_int32]
 _lib.diffqkv_augq.restype = C.c_int
 _lib.diffqkv_augq.argtypes = [C.c_void_p] * 5 + [C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                  C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.diffqkv_augq_rope.restype = C.c_int
+_lib.diffqkv_augq_rope.argtypes = [C.c_void_p] * 5 + [C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p,
+                                                      C.c_void_p, C.c_void_p]
+_lib.diffqkv_project.restype = C.c_int
+_lib.diffqkv_project.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.diffqkv_cache_append.restype = C.c_int
+_lib.diffqkv_cache_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(CacheStruct), C.POINTER(ShapeStruct),
+                                      C.c_void_p, C.c_void_p]
 _lib.diffqkv_status_string.restype = C.c_char_p
 _lib.diffqkv_status_string.argtypes = [C.c_int]
 _lib.diffqkv_launch_count.restype = C.c_int64
@@ -291,3 +302,57 @@ def diffqkv_augq(h: torch.Tensor, W_Q: torch.Tensor, W_gate: torch.Tensor, W_up:
     if st != OK:
         raise DiffQKVError(st, "diffqkv_augq")
     return q_out
+
+
+def diffqkv_augq_rope(h: torch.Tensor, W_Q: torch.Tensor, W_gate: torch.Tensor, W_up: torch.Tensor,
+                      W_down: torch.Tensor, head_dim: int, cos: torch.Tensor, sin: torch.Tensor,
+                      workspace: Optional[torch.Tensor] = None, q_out: Optional[torch.Tensor] = None,
+                      dev_status: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """diffqkv_augq with the rotary embedding fused into the last product; cos / sin [T, head_dim / 2] fp32."""
+    T, d_model = h.shape
+    d_q0, d_aug, d_out = W_Q.shape[0], W_gate.shape[0], W_down.shape[0]
+    assert cos.dtype == torch.float32 and sin.dtype == torch.float32 and cos.is_contiguous() and sin.is_contiguous()
+    assert tuple(cos.shape) == (T, head_dim // 2) and tuple(sin.shape) == (T, head_dim // 2)
+    if workspace is None:
+        workspace = torch.empty(max(diffqkv_augq_workspace_bytes(T, d_q0, d_aug), 256), dtype=torch.uint8,
+                                device=h.device)
+    if q_out is None:
+        q_out = torch.empty((T, d_out), dtype=torch.bfloat16, device=h.device)
+    st = _lib.diffqkv_augq_rope(_p(h), _p(W_Q), _p(W_gate), _p(W_up), _p(W_down), T, d_model, d_q0, d_aug, d_out,
+                                int(head_dim), _p(cos), _p(sin), _p(workspace), workspace.numel(), _p(q_out),
+                                _p(dev_status), _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_augq_rope")
+    return q_out
+
+
+def diffqkv_project(x: torch.Tensor, W: torch.Tensor, head_dim: int = 0, cos: Optional[torch.Tensor] = None,
+                    sin: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                    dev_status: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """y = x W^T (W [d_out, d_in], bf16), rotated per head when cos / sin [T, head_dim / 2] fp32 are given."""
+    T, d_in = x.shape
+    d_out = W.shape[0]
+    if cos is not None:
+        assert cos.dtype == torch.float32 and sin.dtype == torch.float32 and cos.is_contiguous() and sin.is_contiguous()
+        assert tuple(cos.shape) == (T, head_dim // 2) and tuple(sin.shape) == (T, head_dim // 2)
+    if out is None:
+        out = torch.empty((T, d_out), dtype=torch.bfloat16, device=x.device)
+    st = _lib.diffqkv_project(_p(x), _p(W), T, d_in, d_out, int(head_dim), _p(cos), _p(sin), _p(out), _p(dev_status),
+                              _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_project")
+    return out
+
+
+def diffqkv_cache_append(k_new: torch.Tensor, v_new: torch.Tensor, cache: KVCache,
+                         dev_status: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Write k_new [batch, q_len, n_k, d_qk] / v_new [batch, q_len, n_v, d_v] at positions seqlens[b] + i."""
+    batch, q_len, n_k, d_qk = k_new.shape
+    n_v, d_v = v_new.shape[2], v_new.shape[3]
+    # the append does not involve query heads; any count both head counts divide satisfies the shape check
+    shape = make_shape(batch, n_k * n_v, n_k, n_v, d_qk, d_v, k_new.dtype, k_new.dtype, 1.0)
+    cs = cache.c_struct()
+    st = _lib.diffqkv_cache_append(_p(k_new), _p(v_new), q_len, C.byref(cs), C.byref(shape), _p(dev_status),
+                                   _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_cache_append")

@@ -233,13 +233,25 @@ size_t diffqkv_augq_workspace_bytes(int64_t T, int32_t d_q0, int32_t d_aug) {
   return augq_workspace_bytes(T, d_q0, d_aug);
 }
 
-diffqkv_status diffqkv_augq(const void* h, const void* W_Q, const void* W_gate, const void* W_up, const void* W_down,
-                            int64_t T, int32_t d_model, int32_t d_q0, int32_t d_aug, int32_t d_out, void* workspace,
-                            size_t workspace_bytes, void* q_out, int32_t* dev_status, void* stream) {
+static diffqkv_status check_rope(const float* cos, const float* sin, int32_t head_dim, int32_t d_out) {
+  if (!cos && !sin) return DIFFQKV_OK;
+  if (!cos || !sin) return DIFFQKV_ERR_INVALID_ARG;
+  if (head_dim != 64 && head_dim != 128) return DIFFQKV_ERR_UNSUPPORTED;
+  if (d_out % head_dim != 0) return DIFFQKV_ERR_INVALID_ARG;
+  if (!aligned16(cos) || !aligned16(sin)) return DIFFQKV_ERR_ALIGNMENT;
+  return DIFFQKV_OK;
+}
+
+diffqkv_status diffqkv_augq_rope(const void* h, const void* W_Q, const void* W_gate, const void* W_up,
+                                 const void* W_down, int64_t T, int32_t d_model, int32_t d_q0, int32_t d_aug,
+                                 int32_t d_out, int32_t head_dim, const float* cos, const float* sin, void* workspace,
+                                 size_t workspace_bytes, void* q_out, int32_t* dev_status, void* stream) {
   if (!h || !W_Q || !W_gate || !W_up || !W_down || !q_out) return DIFFQKV_ERR_INVALID_ARG;
   if (T < 0 || d_model <= 0 || d_q0 <= 0 || d_aug <= 0 || d_out <= 0) return DIFFQKV_ERR_INVALID_ARG;
   if (T > 0x7fffff00LL) return DIFFQKV_ERR_UNSUPPORTED;
   if (d_model % 128 != 0 || d_q0 % 128 != 0 || d_aug % 128 != 0 || d_out % 128 != 0) return DIFFQKV_ERR_UNSUPPORTED;
+  const diffqkv_status rs = check_rope(cos, sin, head_dim, d_out);
+  if (rs != DIFFQKV_OK) return rs;
   const void* ptrs[6] = {h, W_Q, W_gate, W_up, W_down, q_out};
   for (const void* ptr : ptrs)
     if (!aligned16(ptr)) return DIFFQKV_ERR_ALIGNMENT;
@@ -247,8 +259,46 @@ diffqkv_status diffqkv_augq(const void* h, const void* W_Q, const void* W_gate, 
   if (!workspace || workspace_bytes < augq_workspace_bytes(T, d_q0, d_aug)) return DIFFQKV_ERR_WORKSPACE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DIFFQKV_ERR_ALIGNMENT;
   const cudaError_t err = launch_augq(h, W_Q, W_gate, W_up, W_down, T, d_model, d_q0, d_aug, d_out, workspace, q_out,
-                                      dev_status, static_cast<cudaStream_t>(stream));
+                                      dev_status, static_cast<cudaStream_t>(stream), cos, sin, head_dim);
   if (err == cudaErrorNotSupported) return DIFFQKV_ERR_UNSUPPORTED;
+  return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
+}
+
+diffqkv_status diffqkv_augq(const void* h, const void* W_Q, const void* W_gate, const void* W_up, const void* W_down,
+                            int64_t T, int32_t d_model, int32_t d_q0, int32_t d_aug, int32_t d_out, void* workspace,
+                            size_t workspace_bytes, void* q_out, int32_t* dev_status, void* stream) {
+  return diffqkv_augq_rope(h, W_Q, W_gate, W_up, W_down, T, d_model, d_q0, d_aug, d_out, 0, nullptr, nullptr,
+                           workspace, workspace_bytes, q_out, dev_status, stream);
+}
+
+diffqkv_status diffqkv_project(const void* x, const void* W, int64_t T, int32_t d_in, int32_t d_out, int32_t head_dim,
+                               const float* cos, const float* sin, void* y, int32_t* dev_status, void* stream) {
+  if (!x || !W || !y) return DIFFQKV_ERR_INVALID_ARG;
+  if (T < 0 || d_in <= 0 || d_out <= 0) return DIFFQKV_ERR_INVALID_ARG;
+  if (T > 0x7fffff00LL) return DIFFQKV_ERR_UNSUPPORTED;
+  if (d_in % 128 != 0 || d_out % 128 != 0) return DIFFQKV_ERR_UNSUPPORTED;
+  const diffqkv_status rs = check_rope(cos, sin, head_dim, d_out);
+  if (rs != DIFFQKV_OK) return rs;
+  if (!aligned16(x) || !aligned16(W) || !aligned16(y)) return DIFFQKV_ERR_ALIGNMENT;
+  if (T == 0) return DIFFQKV_OK;
+  const cudaError_t err = launch_project(x, W, T, d_in, d_out, y, dev_status, static_cast<cudaStream_t>(stream), cos,
+                                         sin, head_dim);
+  if (err == cudaErrorNotSupported) return DIFFQKV_ERR_UNSUPPORTED;
+  return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
+}
+
+diffqkv_status diffqkv_cache_append(const void* k_new, const void* v_new, int32_t q_len, const diffqkv_cache* cache,
+                                    const diffqkv_shape* shape, int32_t* dev_status, void* stream) {
+  diffqkv_status st = check_shape(shape);
+  if (st != DIFFQKV_OK) return st;
+  if (!k_new || !v_new || q_len < 0) return DIFFQKV_ERR_INVALID_ARG;
+  st = check_cache(cache, shape);
+  if (st != DIFFQKV_OK) return st;
+  if (!aligned16(k_new) || !aligned16(v_new)) return DIFFQKV_ERR_ALIGNMENT;
+  if (q_len > cache->max_seqlen) return DIFFQKV_ERR_INVALID_ARG;
+  if (shape->batch == 0 || q_len == 0) return DIFFQKV_OK;
+  const cudaError_t err = launch_cache_append(k_new, v_new, q_len, *cache, *shape, dev_status,
+                                              static_cast<cudaStream_t>(stream));
   return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
 

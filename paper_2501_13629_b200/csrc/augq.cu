@@ -34,6 +34,11 @@ struct GemmParams {
   int M, N;
   int m_tiles, n_tiles, k_blocks;
   int dual;  // 0: C tile 128x256 = A.B0^T;  1: C tile 128x128 = silu(A.B0^T) * (A.B1^T)
+  // rotary embedding applied to the fp32 result before it is rounded (plain mode only): tables [M, head_dim / 2],
+  // channel i < head_dim / 2 of a head pairs with channel i + head_dim / 2; NULL = none
+  const float* rope_cos;
+  const float* rope_sin;
+  int head_dim;
   int* dev_status;
 };
 
@@ -189,6 +194,44 @@ gemm_nt_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               *reinterpret_cast<uint4*>(crow + c * 32 + v * 8) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
           }
         }
+      } else if (p.rope_cos) {
+        __nv_bfloat16* crow = p.C + (long long)row * p.ldc + (long long)nt * kBN;
+        const int half = p.head_dim >> 1;
+        const long long trow = (long long)(row < p.M ? row : 0) * half;
+#pragma unroll 1
+        for (int hd = 0; hd < kBN; hd += p.head_dim) {  // heads of this column tile
+          if (nt * kBN + hd >= p.N) break;              // warp-uniform: partial last column tile
+#pragma unroll 1
+          for (int c = 0; c < half; c += 32) {
+            uint32_t x1[32], x2[32];
+            tc::ld_32x32b_x32(taddr + hd + c, x1);
+            tc::ld_32x32b_x32(taddr + hd + half + c, x2);
+            tc::wait_ld();
+            if (row < p.M) {
+              uint32_t o1[16], o2[16];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const float4 cs = *reinterpret_cast<const float4*>(p.rope_cos + trow + c + 4 * e);
+                const float4 sn = *reinterpret_cast<const float4*>(p.rope_sin + trow + c + 4 * e);
+                const float cv[4] = {cs.x, cs.y, cs.z, cs.w}, sv[4] = {sn.x, sn.y, sn.z, sn.w};
+                float y1[4], y2[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const float a = __uint_as_float(x1[4 * e + i]), b = __uint_as_float(x2[4 * e + i]);
+                  y1[i] = a * cv[i] - b * sv[i];
+                  y2[i] = b * cv[i] + a * sv[i];
+                }
+                o1[2 * e] = pack2(y1[0], y1[1]); o1[2 * e + 1] = pack2(y1[2], y1[3]);
+                o2[2 * e] = pack2(y2[0], y2[1]); o2[2 * e + 1] = pack2(y2[2], y2[3]);
+              }
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                *reinterpret_cast<uint4*>(crow + hd + c + v * 8) = make_uint4(o1[4 * v], o1[4 * v + 1], o1[4 * v + 2], o1[4 * v + 3]);
+                *reinterpret_cast<uint4*>(crow + hd + half + c + v * 8) = make_uint4(o2[4 * v], o2[4 * v + 1], o2[4 * v + 2], o2[4 * v + 3]);
+              }
+            }
+          }
+        }
       } else {
         __nv_bfloat16* crow = p.C + (long long)row * p.ldc + (long long)nt * kBN;
 #pragma unroll 1
@@ -240,7 +283,8 @@ int sm_count() {
 
 // C[M, N] = A[M, K] . B0[N, K]^T, or with B1: C[M, N] = silu(A.B0^T) * (A.B1^T).
 cudaError_t launch_gemm(const void* A, const void* B0, const void* B1, void* C, long long M, int N, int K,
-                        int* dev_status, cudaStream_t stream) {
+                        int* dev_status, cudaStream_t stream, const float* rope_cos = nullptr,
+                        const float* rope_sin = nullptr, int head_dim = 0) {
   CUtensorMap ma, mb0, mb1;
   if (!make_operand_map(&ma, A, M, K) || !make_operand_map(&mb0, B0, N, K) ||
       !make_operand_map(&mb1, B1 ? B1 : B0, N, K))
@@ -255,6 +299,9 @@ cudaError_t launch_gemm(const void* A, const void* B0, const void* B1, void* C, 
   p.n_tiles = p.dual ? N / 128 : (N + kBN - 1) / kBN;
   p.k_blocks = K / kBK;
   p.dev_status = dev_status;
+  p.rope_cos = p.dual ? nullptr : rope_cos;
+  p.rope_sin = rope_sin;
+  p.head_dim = head_dim;
   const int sms = sm_count();
   if (sms <= 0) return cudaErrorUnknown;
   const long long tiles = (long long)p.m_tiles * p.n_tiles;
@@ -275,7 +322,8 @@ size_t augq_workspace_bytes(long long T, int d_q0, int d_aug) {
 
 cudaError_t launch_augq(const void* h, const void* W_Q, const void* W_gate, const void* W_up, const void* W_down,
                         long long T, int d_model, int d_q0, int d_aug, int d_out, void* workspace, void* q_out,
-                        int* dev_status, cudaStream_t stream) {
+                        int* dev_status, cudaStream_t stream, const float* rope_cos, const float* rope_sin,
+                        int head_dim) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
   char* ws = reinterpret_cast<char*>(workspace);
   void* x = ws;
@@ -284,7 +332,13 @@ cudaError_t launch_augq(const void* h, const void* W_Q, const void* W_gate, cons
   if (err != cudaSuccess) return err;
   err = launch_gemm(x, W_gate, W_up, a, T, d_aug, d_q0, dev_status, stream);
   if (err != cudaSuccess) return err;
-  return launch_gemm(a, W_down, nullptr, q_out, T, d_out, d_aug, dev_status, stream);
+  return launch_gemm(a, W_down, nullptr, q_out, T, d_out, d_aug, dev_status, stream, rope_cos, rope_sin, head_dim);
+}
+
+// y[T, d_out] = x[T, d_in] . W[d_out, d_in]^T, optionally rotated per head (the K and V projections).
+cudaError_t launch_project(const void* x, const void* W, long long T, int d_in, int d_out, void* y, int* dev_status,
+                           cudaStream_t stream, const float* rope_cos, const float* rope_sin, int head_dim) {
+  return launch_gemm(x, W, nullptr, y, T, d_out, d_in, dev_status, stream, rope_cos, rope_sin, head_dim);
 }
 
 }  // namespace diffqkv

@@ -76,11 +76,16 @@ void set_tma_max_blocks(int n);
 size_t augq_workspace_bytes(long long T, int d_q0, int d_aug);
 cudaError_t launch_augq(const void* h, const void* W_Q, const void* W_gate, const void* W_up, const void* W_down,
                         long long T, int d_model, int d_q0, int d_aug, int d_out, void* workspace, void* q_out,
-                        int* dev_status, cudaStream_t stream);
+                        int* dev_status, cudaStream_t stream, const float* rope_cos = nullptr,
+                        const float* rope_sin = nullptr, int head_dim = 0);
+cudaError_t launch_project(const void* x, const void* W, long long T, int d_in, int d_out, void* y, int* dev_status,
+                           cudaStream_t stream, const float* rope_cos, const float* rope_sin, int head_dim);
 
 
 // Causal prefill (prefill.cu): cache update kernel, then tcgen05 attention over the cache.
 bool prefill_supported(const diffqkv_shape& s, const diffqkv_cache& c, int* box_tok);
+cudaError_t launch_cache_append(const void* k_new, const void* v_new, int q_len, const diffqkv_cache& c,
+                                const diffqkv_shape& s, int* dev_status, cudaStream_t stream);
 cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, int q_len, const diffqkv_cache& c,
                            const diffqkv_shape& s, int box_tok, void* out, float* lse, int* dev_status,
                            cudaStream_t stream);

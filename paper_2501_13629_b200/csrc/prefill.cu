@@ -475,29 +475,37 @@ bool prefill_supported(const diffqkv_shape& s, const diffqkv_cache& c, int* box_
   return true;
 }
 
-cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, int q_len, const diffqkv_cache& c,
-                           const diffqkv_shape& s, int box_tok, void* out, float* lse, int* dev_status,
-                           cudaStream_t stream) {
-  // ---- step 1: cache update
+// The cache update alone: rows past_b .. past_b + q_len - 1 of both pools (any strides, paged or contiguous, bf16 or fp32).
+cudaError_t launch_cache_append(const void* k_new, const void* v_new, int q_len, const diffqkv_cache& c,
+                                const diffqkv_shape& s, int* dev_status, cudaStream_t stream) {
+  const int epv = s.dtype == DIFFQKV_BF16 ? 8 : 4;  // elements per 16-byte vector
   AppendParams a;
   a.k_new = reinterpret_cast<const uint4*>(k_new);
   a.v_new = reinterpret_cast<const uint4*>(v_new);
   a.k_cache = reinterpret_cast<uint4*>(c.k_cache);
   a.v_cache = reinterpret_cast<uint4*>(c.v_cache);
-  a.k_sb = c.k_stride_blk / 8; a.k_sh = c.k_stride_head / 8; a.k_st = c.k_stride_tok / 8;
-  a.v_sb = c.v_stride_blk / 8; a.v_sh = c.v_stride_head / 8; a.v_st = c.v_stride_tok / 8;
+  a.k_sb = c.k_stride_blk / epv; a.k_sh = c.k_stride_head / epv; a.k_st = c.k_stride_tok / epv;
+  a.v_sb = c.v_stride_blk / epv; a.v_sh = c.v_stride_head / epv; a.v_st = c.v_stride_tok / epv;
   a.seqlens = c.seqlens; a.page_table = c.page_table;
   a.page_size = c.page_size; a.max_pages_per_seq = c.max_pages_per_seq;
   a.num_blocks = c.num_blocks; a.max_seqlen = c.max_seqlen;
   a.batch = s.batch; a.q_len = q_len; a.n_k = s.n_k; a.n_v = s.n_v;
-  a.vec_k = s.d_qk / 8; a.vec_v = s.d_v / 8;
+  a.vec_k = s.d_qk / epv; a.vec_v = s.d_v / epv;
   a.dev_status = dev_status;
   const long long vecs = (long long)s.batch * q_len * ((long long)s.n_k * a.vec_k + (long long)s.n_v * a.vec_v);
+  if (vecs == 0) return cudaSuccess;
   long long blocks = (vecs + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   cache_append_kernel<<<(unsigned)blocks, 256, 0, stream>>>(a);
   count_launch();
-  cudaError_t err = cudaGetLastError();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, int q_len, const diffqkv_cache& c,
+                           const diffqkv_shape& s, int box_tok, void* out, float* lse, int* dev_status,
+                           cudaStream_t stream) {
+  // ---- step 1: cache update
+  cudaError_t err = launch_cache_append(k_new, v_new, q_len, c, s, dev_status, stream);
   if (err != cudaSuccess) return err;
 
   // ---- step 2: attention over the cache
