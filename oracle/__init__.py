@@ -127,6 +127,28 @@ def decode(q: np.ndarray, cache: Cache, n_q: int, n_k: int, n_v: int, d_qk: int,
     return out, lse
 
 
+def decode_topk(q: np.ndarray, cache: Cache, n_q: int, n_k: int, n_v: int, d_qk: int, d_v: int, scale: float,
+                topk: int):
+    """Selective V fetching: attention over the `topk` highest-scoring cached tokens of every query head only.
+
+    Returns (out [batch,n_q,d_v], lse [batch,n_q], selected [batch,n_q,topk] int32 (-1 padded, best first),
+    margin [batch,n_q] = gap between the last kept and the first dropped score)."""
+    dt = _dtype_code(q)
+    q = np.ascontiguousarray(q)
+    batch = q.shape[0]
+    out = np.zeros((batch, n_q, d_v), dtype=np.float64)
+    lse = np.zeros((batch, n_q), dtype=np.float64)
+    sel = np.zeros((batch, n_q, topk), dtype=np.int32)
+    margin = np.zeros((batch, n_q), dtype=np.float64)
+    cs = cache.c_struct()
+    lib().oracle_decode_topk.restype = C.c_int
+    rc = lib().oracle_decode_topk(_ptr(q), C.byref(cs), batch, n_q, n_k, n_v, d_qk, d_v, dt, C.c_double(scale),
+                                  int(topk), _ptr(out), _ptr(lse), _ptr(sel), _ptr(margin))
+    if rc != 0:
+        raise ValueError("n_k and n_v must divide n_q and topk must be positive")
+    return out, lse, sel, margin
+
+
 def decode_splits(q: np.ndarray, cache: Cache, n_q: int, n_k: int, n_v: int, d_qk: int, d_v: int,
                   scale: float, cuts: Sequence[int]):
     """Per-split normalised outputs and lse for token ranges [cuts[s], cuts[s+1])."""

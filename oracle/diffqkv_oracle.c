@@ -152,6 +152,63 @@ int oracle_decode(const void *q, const oracle_cache *c, int batch, int n_q, int 
   return 0;
 }
 
+/* Selective V cache fetching (Section "Selective V Cache Fetching"; Table topkV uses the 100 highest scores):
+ * only the V vectors of the `topk` highest attention scores enter the output.  The steps, in the paper's order:
+ *   1. scores s_j = scale * <q_h, K[j, hk]> for every cached token j;
+ *   2. T = the topk tokens with the highest scores (equal scores: the earlier token first); all tokens if the
+ *      sequence has no more than topk;
+ *   3. softmax over T only (the paper does not say whether the weights are renormalised over the kept tokens;
+ *      read as renormalised, as in the top-k attention it cites), o = sum_{j in T} p_j V[j, hv].
+ * out [batch, n_q, d_v], lse [batch, n_q] = log sum_{j in T} exp(s_j); selected (optional) [batch, n_q, topk] int32
+ * token ids in descending score order, -1 padded; margin (optional) [batch, n_q] = s_(topk) - s_(topk+1), the gap
+ * that decides the selection (+inf when nothing is dropped). */
+typedef struct { double s; int32_t j; } scored_token;
+static int scored_cmp(const void *a, const void *b) {
+  const scored_token *x = (const scored_token *)a, *y = (const scored_token *)b;
+  if (x->s > y->s) return -1;
+  if (x->s < y->s) return 1;
+  return (x->j > y->j) - (x->j < y->j);
+}
+int oracle_decode_topk(const void *q, const oracle_cache *c, int batch, int n_q, int n_k, int n_v, int d_qk, int d_v,
+                       int dtype, double scale, int topk, double *out, double *lse, int32_t *selected, double *margin) {
+  if (n_k <= 0 || n_v <= 0 || n_q % n_k || n_q % n_v || topk <= 0) return -1;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t w = 0; w < (int64_t)batch * n_q; ++w) {
+    int b = (int)(w / n_q), h = (int)(w % n_q);
+    int hk = (int)(((int64_t)h * n_k) / n_q);
+    int hv = (int)(((int64_t)h * n_v) / n_q);
+    int64_t len = c->seqlens[b];
+    double *o = out + w * d_v;
+    for (int ch = 0; ch < d_v; ++ch) o[ch] = 0.0;
+    if (selected) for (int i = 0; i < topk; ++i) selected[w * topk + i] = -1;
+    if (margin) margin[w] = INFINITY;
+    if (len <= 0) { lse[w] = -INFINITY; continue; }
+    scored_token *st = (scored_token *)malloc(sizeof(scored_token) * (size_t)len);
+    for (int64_t j = 0; j < len; ++j) {
+      int64_t row = cache_row(c, 0, b, j, hk);
+      double acc = 0.0;
+      for (int ch = 0; ch < d_qk; ++ch)
+        acc += load_elt(q, ((int64_t)b * n_q + h) * d_qk + ch, dtype) * load_elt(c->k_cache, row + ch, dtype);
+      st[j].s = acc * scale;
+      st[j].j = (int32_t)j;
+    }
+    qsort(st, (size_t)len, sizeof(scored_token), scored_cmp);
+    int64_t kept = len < topk ? len : topk;
+    if (margin && kept < len) margin[w] = st[kept - 1].s - st[kept].s;
+    double m = st[0].s, l = 0.0;
+    for (int64_t i = 0; i < kept; ++i) l += exp(st[i].s - m);
+    for (int64_t i = 0; i < kept; ++i) {
+      double p = exp(st[i].s - m) / l;
+      int64_t row = cache_row(c, 1, b, st[i].j, hv);
+      for (int ch = 0; ch < d_v; ++ch) o[ch] += p * load_elt(c->v_cache, row + ch, dtype);
+      if (selected) selected[w * topk + i] = st[i].j;
+    }
+    lse[w] = m + log(l);
+    free(st);
+  }
+  return 0;
+}
+
 /* Decode restricted to an explicit token range per split: cuts [n_splits + 1]
  * ascending token positions shared by all sequences (clamped to each length).
  * o_partial [batch, n_q, n_splits, d_v], lse_partial [batch, n_q, n_splits]:

@@ -364,6 +364,62 @@ def test_augq_matches_library_matmul(oracle, dtype):
     assert np.array_equal(oracle.augq(h, wq, wg, wu, wd, rows=rows), out[rows])
 
 
+# --------------------------------------------------------------------------- selective V fetching
+def test_topk_keeps_everything_when_k_covers_the_sequence(oracle):
+    n_q, n_k, n_v, d, S = 8, 2, 4, 16, 40
+    q, k, v = _rand(201, (2, n_q, d)), _rand(202, (2, n_k, S, d)), _rand(203, (2, n_v, S, d))
+    cache = _contig_cache(oracle, k, v, [40, 13])
+    full, lse_full = oracle.decode(q, cache, n_q, n_k, n_v, d, d, 0.3)
+    for topk in (40, 64):
+        out, lse, sel, margin = oracle.decode_topk(q, cache, n_q, n_k, n_v, d, d, 0.3, topk)
+        assert np.allclose(out, full, rtol=0, atol=1e-13) and np.allclose(lse, lse_full, rtol=0, atol=1e-13)
+        assert np.all(np.isinf(margin)) and np.all(np.sort(sel[0, 0][sel[0, 0] >= 0]) == np.arange(40))
+        assert np.all(sel[1, :, 13:] == -1)
+
+
+def test_top1_returns_the_v_row_of_the_best_key(oracle):
+    n_q, n_k, n_v, d, S = 4, 2, 4, 8, 30
+    q, k, v = _rand(211, (1, n_q, d)), _rand(212, (1, n_k, S, d)), _rand(213, (1, n_v, S, d))
+    cache = _contig_cache(oracle, k, v, [S])
+    out, lse, sel, _ = oracle.decode_topk(q, cache, n_q, n_k, n_v, d, d, 1.0, 1)
+    for h in range(n_q):
+        s = W.as_f64(k[0, h // 2]) @ W.as_f64(q[0, h])
+        j = int(np.argmax(s))
+        assert sel[0, h, 0] == j and np.array_equal(out[0, h], W.as_f64(v[0, h, j])) and abs(lse[0, h] - s[j]) < 1e-13
+
+
+def test_topk_matches_numpy_selection_and_error_bound(oracle):
+    """Independent restatement with numpy's sort; and the distance to full attention is bounded by twice the
+    probability mass that was dropped times the largest |V|."""
+    n_q, n_k, n_v, d, S, topk = 8, 2, 4, 16, 200, 20
+    q, k, v = _rand(221, (1, n_q, d)), _rand(222, (1, n_k, S, d)), _rand(223, (1, n_v, S, d))
+    cache = _contig_cache(oracle, k, v, [S])
+    out, lse, sel, margin = oracle.decode_topk(q, cache, n_q, n_k, n_v, d, d, 0.5, topk)
+    full, _ = oracle.decode(q, cache, n_q, n_k, n_v, d, d, 0.5)
+    for h in range(n_q):
+        s = 0.5 * (W.as_f64(k[0, h // 4]) @ W.as_f64(q[0, h]))
+        order = np.argsort(-s, kind="stable")
+        keep = order[:topk]
+        assert np.array_equal(sel[0, h], keep)
+        p = np.exp(s[keep] - s[keep].max())
+        ref = (p / p.sum()) @ W.as_f64(v[0, h // 2])[keep]
+        assert np.allclose(out[0, h], ref, rtol=0, atol=1e-13)
+        assert abs(margin[0, h] - (s[order[topk - 1]] - s[order[topk]])) < 1e-13
+        pf = np.exp(s - s.max())
+        dropped = 1.0 - pf[keep].sum() / pf.sum()
+        assert np.abs(out[0, h] - full[0, h]).max() <= 2.0 * dropped * np.abs(W.as_f64(v[0, h // 2])).max() + 1e-12
+
+
+def test_topk_ties_take_the_earlier_token(oracle):
+    d = 4
+    q = np.ones((1, 1, d), np.float32)
+    k = np.ones((1, 1, 6, d), np.float32)  # every score equal
+    v = np.arange(6 * d, dtype=np.float32).reshape(1, 1, 6, d)
+    out, _, sel, margin = oracle.decode_topk(q, _contig_cache(oracle, k, v, [6]), 1, 1, 1, d, d, 1.0, 3)
+    assert np.array_equal(sel[0, 0], [0, 1, 2]) and margin[0, 0] == 0.0
+    assert np.allclose(out[0, 0], v[0, 0, :3].mean(axis=0))
+
+
 # --------------------------------------------------------------------------- projections and rotary embedding
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_linear_matches_library_matmul(oracle, dtype):
