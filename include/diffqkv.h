@@ -233,6 +233,23 @@ diffqkv_status diffqkv_project(const void *x, const void *W, int64_t T, int32_t 
 diffqkv_status diffqkv_cache_append(const void *k_new, const void *v_new, int32_t q_len, const diffqkv_cache *cache,
                                     const diffqkv_shape *shape, int32_t *dev_status, void *stream);
 
+/*
+ * diffqkv_decode_topk -- decode with selective V cache fetching (paper Section "Selective V Cache Fetching"; its
+ * table uses the 100 highest scores): every query head scores all cached tokens of its K head, keeps the `topk`
+ * highest scores (equal scores: the earlier token), takes the softmax over the kept scores only (the paper does
+ * not say whether the weights are renormalised; read as renormalised) and sums the kept V rows.  The K cache is
+ * streamed once, of the V cache only topk rows per query head are read.  A sequence with at most topk tokens gives
+ * exactly the full attention of diffqkv_decode.
+ *   q, cache, out, lse, dev_status as in diffqkv_decode; bf16 only, d_qk 64 or 128, at most 32 query heads per
+ *   K head, 1 <= topk <= 1024, pages of 16, 32, 64 or a multiple of 128 tokens
+ *   workspace  diffqkv_decode_topk_workspace_bytes(shape, cache->max_seqlen) bytes, 256-byte aligned: the fp32
+ *              scores [batch, n_q, max_seqlen rounded up to 128]
+ */
+size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape *shape, int32_t max_seqlen);
+diffqkv_status diffqkv_decode_topk(const void *q, const diffqkv_cache *cache, const diffqkv_shape *shape, int32_t topk,
+                                   void *workspace, size_t workspace_bytes, void *out, float *lse,
+                                   int32_t *dev_status, void *stream);
+
 /* Static, never-null description of a status value. */
 const char *diffqkv_status_string(diffqkv_status status);
 

@@ -30,7 +30,7 @@ EXPORTS = (
     "diffqkv_combine", "diffqkv_prefill", "diffqkv_augq_workspace_bytes", "diffqkv_augq",
     "diffqkv_status_string", "diffqkv_launch_count", "diffqkv_profile_split_events", "diffqkv_decode_static",
     "diffqkv_set_max_blocks", "diffqkv_last_decode_kernel", "diffqkv_augq_rope", "diffqkv_project",
-    "diffqkv_cache_append",
+    "diffqkv_cache_append", "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes",
 )
 
 
@@ -86,6 +86,11 @@ _lib.diffqkv_project.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C
 _lib.diffqkv_cache_append.restype = C.c_int
 _lib.diffqkv_cache_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(CacheStruct), C.POINTER(ShapeStruct),
                                       C.c_void_p, C.c_void_p]
+_lib.diffqkv_decode_topk_workspace_bytes.restype = C.c_size_t
+_lib.diffqkv_decode_topk_workspace_bytes.argtypes = [C.POINTER(ShapeStruct), C.c_int32]
+_lib.diffqkv_decode_topk.restype = C.c_int
+_lib.diffqkv_decode_topk.argtypes = [C.c_void_p, C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_int32, C.c_void_p,
+                                     C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.diffqkv_status_string.restype = C.c_char_p
 _lib.diffqkv_status_string.argtypes = [C.c_int]
 _lib.diffqkv_launch_count.restype = C.c_int64
@@ -356,3 +361,25 @@ def diffqkv_cache_append(k_new: torch.Tensor, v_new: torch.Tensor, cache: KVCach
                                    _stream_ptr(stream))
     if st != OK:
         raise DiffQKVError(st, "diffqkv_cache_append")
+
+
+def diffqkv_decode_topk(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: float, topk: int,
+                        workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                        lse: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                        out_dtype: Optional[torch.dtype] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Decode that reads only the V rows of the `topk` highest scores of every query head."""
+    batch, n_q, d_qk = q.shape
+    d_v = cache.v.shape[-1]
+    out_dtype = out_dtype or (out.dtype if out is not None else q.dtype)
+    shape = make_shape(batch, n_q, n_k, n_v, d_qk, d_v, q.dtype, out_dtype, scale)
+    if workspace is None:
+        nbytes = int(_lib.diffqkv_decode_topk_workspace_bytes(C.byref(shape), cache.max_seqlen))
+        workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
+    if out is None:
+        out = torch.empty((batch, n_q, d_v), dtype=out_dtype, device=q.device)
+    cs = cache.c_struct()
+    st = _lib.diffqkv_decode_topk(_p(q), C.byref(cs), C.byref(shape), int(topk), _p(workspace), workspace.numel(),
+                                  _p(out), _p(lse), _p(dev_status), _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_decode_topk")
+    return out

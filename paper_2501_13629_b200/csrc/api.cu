@@ -302,6 +302,31 @@ diffqkv_status diffqkv_cache_append(const void* k_new, const void* v_new, int32_
   return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
 
+size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape* shape, int32_t max_seqlen) {
+  if (check_shape(shape) != DIFFQKV_OK || max_seqlen < 0) return 0;
+  return topk_decode_workspace_bytes(*shape, max_seqlen);
+}
+
+diffqkv_status diffqkv_decode_topk(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape, int32_t topk,
+                                   void* workspace, size_t workspace_bytes, void* out, float* lse, int32_t* dev_status,
+                                   void* stream) {
+  diffqkv_status st = check_shape(shape);
+  if (st != DIFFQKV_OK) return st;
+  if (!q || !out || topk < 1) return DIFFQKV_ERR_INVALID_ARG;
+  st = check_cache(cache, shape);
+  if (st != DIFFQKV_OK) return st;
+  if (!aligned16(q) || !aligned16(out)) return DIFFQKV_ERR_ALIGNMENT;
+  if (shape->batch == 0) return DIFFQKV_OK;
+  int box_tok = 0;
+  if (!topk_decode_supported(*shape, *cache, topk, &box_tok)) return DIFFQKV_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < topk_decode_workspace_bytes(*shape, cache->max_seqlen)) return DIFFQKV_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DIFFQKV_ERR_ALIGNMENT;
+  const cudaError_t err = launch_decode_topk(q, *cache, *shape, topk, box_tok, workspace, out, lse, dev_status,
+                                             static_cast<cudaStream_t>(stream));
+  if (err == cudaErrorNotSupported) return DIFFQKV_ERR_UNSUPPORTED;
+  return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
+}
+
 const char* diffqkv_status_string(diffqkv_status status) {
   switch (status) {
     case DIFFQKV_OK: return "ok";

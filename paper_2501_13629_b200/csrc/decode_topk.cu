@@ -1,0 +1,566 @@
+// Selective V cache fetching for decode (paper Section "Selective V Cache Fetching"): only the V vectors of the
+// top-k attention scores of each query head enter the output, so V traffic drops from the whole cache to k rows
+// per head while K is still streamed once.  Two kernels:
+//
+//   decode_scores_kernel   persistent blocks stream the K cache (TMA ring of 128-token tiles, 128-byte swizzle) and
+//                          score every cached token against all query heads of its K head at once (mma.sync
+//                          m16n8k16, fp32 accumulation); scores go to a workspace as fp32, already multiplied by
+//                          scale * log2(e).  All (sequence, K head, tile) triples form one flat list divided evenly
+//                          over one block per SM; tiles are independent, so nothing has to be merged.
+//   topk_attend_kernel     one block per (sequence, query head): radix select (4 passes of 8 bits over an order-
+//                          preserving key) finds the k-th largest score; the kept tokens are compacted in token order
+//                          (equal scores: the earlier token first, as the definition says); softmax over the kept
+//                          scores; the k V rows are gathered with 16-byte loads and accumulated in fp32.
+// Both are launched with programmatic stream serialisation and wait on the device before touching their inputs.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+#include "tmap.cuh"
+
+namespace diffqkv {
+namespace {
+
+constexpr int kST = 128;            // tokens per K tile
+constexpr int kScoreWarps = 4;      // consumer warps, 32 tokens each
+constexpr int kScoreThreads = (kScoreWarps + 1) * 32;
+constexpr int kMaxBatchScores = 2048;
+constexpr int kMaxTopk = 1024;
+constexpr int kMaxGroups = 4;       // query heads per K head <= 8 * kMaxGroups
+constexpr int kAttendThreads = 256;
+
+struct ScoreParams {
+  const __nv_bfloat16* q;
+  const int* seqlens;
+  const int* page_table;
+  int page_size, max_pages_per_seq, num_blocks, max_seqlen;
+  int batch, n_q, n_k, g_k;  // g_k = query heads per K head
+  int groups;                // ceil(g_k / 8)
+  int box_tok, stages;
+  long long lpad;            // row length of the score matrix
+  float scale_log2;
+  float* scores;             // [batch, n_q, lpad]
+  int* dev_status;
+};
+
+// Position in the flat (sequence, K head, tile) list.
+struct TileWalker {
+  long long g;
+  int b, u, t, nt;
+  __device__ void seek(long long g0, const int* prefix, int batch, int n_units) {
+    g = g0;
+    int lo = 0, hi = batch;  // smallest b' with n_units * prefix[b'] > g; answer b = b' - 1
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if ((long long)n_units * prefix[mid] > g0) hi = mid; else lo = mid + 1;
+    }
+    b = lo - 1;
+    nt = prefix[b + 1] - prefix[b];
+    const long long rem = g0 - (long long)n_units * prefix[b];
+    u = (int)(rem / nt);
+    t = (int)(rem % nt);
+  }
+  __device__ void advance(const int* prefix, int batch, int n_units) {
+    ++g;
+    if (++t == nt) {
+      t = 0;
+      if (++u == n_units) {
+        u = 0;
+        do {
+          ++b;
+          nt = b < batch ? prefix[b + 1] - prefix[b] : 1;
+        } while (b < batch && nt == 0);
+      }
+    }
+  }
+};
+
+template <int D_QK>
+__global__ void __launch_bounds__(kScoreThreads, 1)
+decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScoreParams p) {
+  constexpr int HK = D_QK / 64;            // 64-channel halves per row
+  constexpr int K_TILE = kST * D_QK * 2;   // bytes of one K tile
+  constexpr int KS = D_QK / 16;
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * K_TILE);  // full[s], empty[s]
+  volatile int* abort_flag = reinterpret_cast<int*>(bars + 2 * p.stages);
+  int* prefix = const_cast<int*>(abort_flag) + 2;  // [batch + 1] tiles before each sequence
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t full0 = ptx::smem_u32(bars), empty0 = ptx::smem_u32(bars + p.stages);
+  if (tid == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < p.stages; ++s) {
+      ptx::mbar_init(full0 + 8 * s, 1);
+      ptx::mbar_init(empty0 + 8 * s, kScoreWarps);
+    }
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmap_k);
+  }
+  ptx::grid_dependency_wait();  // from here on: inputs that earlier work in the stream may still be producing
+  if (warp == 0) {
+    const int per = (p.batch + 31) / 32;
+    const int lo = min(p.batch, lane * per), hi = min(p.batch, lo + per);
+    int sum = 0;
+    for (int b = lo; b < hi; ++b) sum += (min(max(p.seqlens[b], 0), p.max_seqlen) + kST - 1) / kST;
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    int run = incl - sum;
+    for (int b = lo; b < hi; ++b) {
+      prefix[b] = run;
+      run += (min(max(p.seqlens[b], 0), p.max_seqlen) + kST - 1) / kST;
+    }
+    if (lane == 31) prefix[p.batch] = incl;
+  }
+  __syncthreads();
+  const long long total = (long long)p.n_k * prefix[p.batch];
+  const long long nblk = min((long long)gridDim.x, total);
+  if (blockIdx.x >= nblk) {
+    ptx::grid_launch_dependents();
+    return;
+  }
+  const long long g_begin = (total * blockIdx.x) / nblk, g_end = (total * (blockIdx.x + 1)) / nblk;
+  TileWalker w;
+  w.seek(g_begin, prefix, p.batch, p.n_k);
+
+  if (warp == kScoreWarps) {
+    // ------------------------------------------------------------------ producer warp: lane x owns token part x
+    const int parts = kST / p.box_tok;
+    const uint32_t my_off = lane * (p.box_tok * 128 * HK);
+    int stage = 0, issued = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (; w.g < g_end; w.advance(prefix, p.batch, p.n_k)) {
+      const int len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
+      const int tok0 = w.t * kST;
+      const int parts_valid = min(parts, (len - tok0 + p.box_tok - 1) / p.box_tok);
+      int blk = w.b, slot = tok0 + lane * p.box_tok;
+      if (p.page_table && lane < parts_valid) {
+        const int tok = slot;
+        blk = p.page_table[(long long)w.b * p.max_pages_per_seq + tok / p.page_size];
+        slot = tok % p.page_size;
+        if (blk < 0 || blk >= p.num_blocks) {  // never read outside the pool: flag it, read block 0 instead
+          report(p.dev_status, DIFFQKV_ERR_INDEX);
+          blk = 0;
+        }
+      }
+      if (issued >= p.stages && !ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) {
+        report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+        ok = false;
+        break;
+      }
+      const uint32_t bar = full0 + 8 * stage;
+      if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)parts_valid * p.box_tok * 128u * HK);
+      __syncwarp();
+      if (lane < parts_valid)
+        ptx::tma_load_5d(ptx::smem_u32(smem + (size_t)stage * K_TILE) + my_off, &tmap_k, bar, 0, slot, 0, w.u, blk);
+      ++issued;
+      if (++stage == p.stages) { stage = 0; phase ^= 1; }
+    }
+    ptx::grid_launch_dependents();
+    if (!ok) {
+      for (int s = 0; s < min(issued, p.stages); ++s) {
+        const int uses = (issued - s + p.stages - 1) / p.stages;
+        ptx::mbar_wait(full0 + 8 * s, (uint32_t)(uses - 1) & 1u, nullptr);
+      }
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- consumer warps
+  const int g8 = lane >> 2, t4 = lane & 3;
+  const int bt_shift = 31 - __clz(p.box_tok), bt_mask = p.box_tok - 1;
+  auto row_index = [&](int r, int h) { return (((r >> bt_shift) * HK + h) << bt_shift) + (r & bt_mask); };
+  int stage = 0;
+  uint32_t phase = 0;
+  int cur_b = -1, cur_u = -1;
+  uint32_t qf[kMaxGroups][KS][2];
+  for (; w.g < g_end; w.advance(prefix, p.batch, p.n_k)) {
+    if (w.b != cur_b || w.u != cur_u) {  // Q^T fragments of the query heads of this K head, 8 heads per group
+      cur_b = w.b; cur_u = w.u;
+#pragma unroll
+      for (int gq = 0; gq < kMaxGroups; ++gq) {
+        const int hq = gq * 8 + g8;
+        const bool use = gq < p.groups && hq < p.g_k;
+        const __nv_bfloat16* qrow = p.q + ((long long)w.b * p.n_q + (long long)w.u * p.g_k + (use ? hq : 0)) * D_QK;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+          qf[gq][ks][0] = use ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t4) : 0u;
+          qf[gq][ks][1] = use ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t4 + 8) : 0u;
+        }
+      }
+    }
+    if (!ptx::mbar_wait(full0 + 8 * stage, phase, abort_flag)) {  // all four warps give up at the same stage
+      report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+      break;
+    }
+    const int len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
+    const int n_valid = min(kST, len - w.t * kST);
+    const uint32_t st_u32 = ptx::smem_u32(smem + (size_t)stage * K_TILE);
+#pragma unroll
+    for (int rb = 0; rb < 2; ++rb) {
+      const int row0 = warp * 32 + rb * 16;
+      if (row0 >= n_valid) continue;
+      float s[kMaxGroups][4];
+#pragma unroll
+      for (int gq = 0; gq < kMaxGroups; ++gq)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[gq][e] = 0.f;
+      const int r = row0 + (lane & 7) + 8 * ((lane >> 3) & 1);
+      const int csel = lane >> 4;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        const int chunk = (ks % 4) * 2 + csel;
+        uint32_t a[4];
+        ptx::ldmatrix_x4(st_u32 + row_index(r, ks / 4) * 128 + ((chunk ^ (r & 7)) << 4), a);
+#pragma unroll
+        for (int gq = 0; gq < kMaxGroups; ++gq)
+          if (gq < p.groups) ptx::mma_bf16_16816(s[gq], a, qf[gq][ks][0], qf[gq][ks][1]);
+      }
+      // thread holds token rows g8, g8 + 8 of the block and head columns 2 t4, 2 t4 + 1 of each group
+      const long long tok = (long long)w.t * kST + row0 + g8;
+#pragma unroll
+      for (int gq = 0; gq < kMaxGroups; ++gq) {
+        if (gq >= p.groups) continue;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const int hq = gq * 8 + 2 * t4 + c;
+          if (hq >= p.g_k) continue;
+          float* dst = p.scores + ((long long)w.b * p.n_q + (long long)w.u * p.g_k + hq) * p.lpad + tok;
+          if (row0 + g8 < n_valid) dst[0] = s[gq][c] * p.scale_log2;
+          if (row0 + g8 + 8 < n_valid) dst[8] = s[gq][2 + c] * p.scale_log2;
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(empty0 + 8 * stage);
+    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+  }
+}
+
+struct AttendParams {
+  const float* scores;
+  long long lpad;
+  const __nv_bfloat16* v;
+  long long v_sb, v_sh, v_st;
+  const int* seqlens;
+  const int* page_table;
+  int page_size, max_pages_per_seq, num_blocks, max_seqlen;
+  int batch, n_q, n_v, d_v, topk;
+  void* out;
+  float* lse;
+  int out_is_f32;
+  int* dev_status;
+};
+
+// Larger float <=> larger key.
+__device__ __forceinline__ uint32_t order_key(float x) {
+  const uint32_t u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(kAttendThreads)
+topk_attend_kernel(const AttendParams p) {
+  __shared__ unsigned hist[256];
+  __shared__ int sel_idx[kMaxTopk];
+  __shared__ float sel_s[kMaxTopk];
+  __shared__ unsigned warp_tot[kAttendThreads / 32];
+  __shared__ unsigned sh_prefix, sh_need;
+  __shared__ float red[kAttendThreads / 32];
+  __shared__ float acc_s[kAttendThreads / 32][512];
+
+  ptx::grid_launch_dependents();
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = blockIdx.x / p.n_q, h = blockIdx.x % p.n_q;
+  const int hv = (int)(((long long)h * p.n_v) / p.n_q);  // Eq. (idx)
+  ptx::grid_dependency_wait();
+  const int len = min(max(p.seqlens[b], 0), p.max_seqlen);
+  const long long orow = ((long long)b * p.n_q + h) * p.d_v;
+  if (len == 0) {
+    for (int ch = tid; ch < p.d_v; ch += kAttendThreads) {
+      if (p.out_is_f32) reinterpret_cast<float*>(p.out)[orow + ch] = 0.f;
+      else reinterpret_cast<__nv_bfloat16*>(p.out)[orow + ch] = __float2bfloat16_rn(0.f);
+    }
+    if (p.lse && tid == 0) p.lse[(long long)b * p.n_q + h] = -INFINITY;
+    return;
+  }
+  const float* row = p.scores + ((long long)b * p.n_q + h) * p.lpad;
+  const int k = min(p.topk, len);
+
+  // ---- the key of the k-th largest score, 8 bits at a time from the top, and how many equal ones to take
+  unsigned thr = 0, need_eq = 0;
+  const bool all = len <= p.topk;
+  if (!all) {
+    unsigned prefix = 0, mask = 0, need = (unsigned)k;
+    for (int pass = 3; pass >= 0; --pass) {
+      for (int i = tid; i < 256; i += kAttendThreads) hist[i] = 0;
+      __syncthreads();
+      for (int i = tid; i < len; i += kAttendThreads) {
+        const unsigned key = order_key(row[i]);
+        if ((key & mask) == prefix) atomicAdd(&hist[(key >> (8 * pass)) & 255u], 1u);
+      }
+      __syncthreads();
+      if (warp == 0) {  // from the top bin down: the bin that holds the need-th largest of the remaining keys
+        unsigned mine = 0;  // lane owns bins 255 - 8 lane .. 248 - 8 lane
+#pragma unroll
+        for (int e = 0; e < 8; ++e) mine += hist[255 - (lane * 8 + e)];
+        unsigned incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += y;
+        }
+        const unsigned before = incl - mine;
+        if (before < need && need <= incl) {  // exactly one lane
+          unsigned cum = before;
+          for (int e = 0; e < 8; ++e) {
+            const int bin = 255 - (lane * 8 + e);
+            if (need <= cum + hist[bin]) {
+              sh_prefix = prefix | ((unsigned)bin << (8 * pass));
+              sh_need = need - cum;
+              break;
+            }
+            cum += hist[bin];
+          }
+        }
+      }
+      __syncthreads();
+      prefix = sh_prefix;
+      need = sh_need;
+      mask |= 0xffu << (8 * pass);
+    }
+    thr = prefix;
+    need_eq = need;
+  }
+
+  // ---- compaction in token order: kept = key > thr, or key == thr among the first need_eq such tokens
+  unsigned base_gt = 0, base_eq = 0;
+  for (int base = 0; base < len; base += kAttendThreads * 4) {
+    float sv[4];
+    unsigned fg = 0, fe = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int i = base + tid * 4 + e;
+      sv[e] = i < len ? row[i] : 0.f;
+      if (i < len) {
+        const unsigned key = order_key(sv[e]);
+        if (all || key > thr) fg |= 1u << e;
+        else if (key == thr) fe |= 1u << e;
+      }
+    }
+    const unsigned packed = __popc(fg) | ((unsigned)__popc(fe) << 16);
+    unsigned incl = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    unsigned before = incl - packed, chunk_tot = 0;
+#pragma unroll
+    for (int ww = 0; ww < kAttendThreads / 32; ++ww) {
+      if (ww < warp) before += warp_tot[ww];
+      chunk_tot += warp_tot[ww];
+    }
+    unsigned gt_before = base_gt + (before & 0xffffu), eq_before = base_eq + (before >> 16);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const bool g = (fg >> e) & 1u, q = (fe >> e) & 1u;
+      if (g || (q && eq_before < need_eq)) {
+        const unsigned pos = gt_before + min(eq_before, need_eq);
+        sel_idx[pos] = base + tid * 4 + e;
+        sel_s[pos] = sv[e];
+      }
+      gt_before += g;
+      eq_before += q;
+    }
+    base_gt += chunk_tot & 0xffffu;
+    base_eq += chunk_tot >> 16;
+    __syncthreads();  // warp_tot is reused by the next chunk
+  }
+
+  // ---- softmax over the kept scores (base-2 domain)
+  float m = -INFINITY;
+  for (int i = tid; i < k; i += kAttendThreads) m = fmaxf(m, sel_s[i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+  m = red[0];
+#pragma unroll
+  for (int ww = 1; ww < kAttendThreads / 32; ++ww) m = fmaxf(m, red[ww]);
+  __syncthreads();
+  float l = 0.f;
+  for (int i = tid; i < k; i += kAttendThreads) {
+    const float e = exp2f(sel_s[i] - m);
+    sel_s[i] = e;
+    l += e;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+  if (lane == 0) red[warp] = l;
+  __syncthreads();
+  l = 0.f;
+#pragma unroll
+  for (int ww = 0; ww < kAttendThreads / 32; ++ww) l += red[ww];
+
+  // ---- gather the kept V rows: a warp per row, a lane per 4 channels (128 channels per sweep)
+  for (int ch0 = 0; ch0 < p.d_v; ch0 += 128) {
+    const int ch = ch0 + lane * 4;
+    const bool in = ch < p.d_v;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = warp; i < k; i += kAttendThreads / 32) {
+      const int j = sel_idx[i];
+      long long blk = b, slot = j;
+      if (p.page_table) {
+        blk = p.page_table[(long long)b * p.max_pages_per_seq + j / p.page_size];
+        slot = j % p.page_size;
+        if (blk < 0 || blk >= p.num_blocks) {
+          report(p.dev_status, DIFFQKV_ERR_INDEX);
+          continue;
+        }
+      }
+      if (in) {
+        const uint2 raw = *reinterpret_cast<const uint2*>(p.v + blk * p.v_sb + (long long)hv * p.v_sh + slot * p.v_st + ch);
+        const float wgt = sel_s[i];
+        a.x = fmaf(wgt, __uint_as_float(raw.x << 16), a.x);
+        a.y = fmaf(wgt, __uint_as_float(raw.x & 0xffff0000u), a.y);
+        a.z = fmaf(wgt, __uint_as_float(raw.y << 16), a.z);
+        a.w = fmaf(wgt, __uint_as_float(raw.y & 0xffff0000u), a.w);
+      }
+    }
+    if (in) {
+      acc_s[warp][ch] = a.x; acc_s[warp][ch + 1] = a.y; acc_s[warp][ch + 2] = a.z; acc_s[warp][ch + 3] = a.w;
+    }
+  }
+  __syncthreads();
+  const float inv = 1.f / l;
+  for (int ch = tid; ch < p.d_v; ch += kAttendThreads) {
+    float o = 0.f;
+#pragma unroll
+    for (int ww = 0; ww < kAttendThreads / 32; ++ww) o += acc_s[ww][ch];
+    o *= inv;
+    if (p.out_is_f32) reinterpret_cast<float*>(p.out)[orow + ch] = o;
+    else reinterpret_cast<__nv_bfloat16*>(p.out)[orow + ch] = __float2bfloat16_rn(o);
+  }
+  if (p.lse && tid == 0) p.lse[(long long)b * p.n_q + h] = (m + log2f(l)) * kLn2;
+}
+
+int sm_count_topk() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  return sms;
+}
+
+}  // namespace
+
+bool topk_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, int topk, int* box_tok) {
+  if (s.dtype != DIFFQKV_BF16 || (s.d_qk != 64 && s.d_qk != 128)) return false;
+  if (s.d_v % 4 != 0 || s.d_v > 512 || topk < 1 || topk > kMaxTopk) return false;
+  if (s.batch < 1 || s.batch > kMaxBatchScores || s.n_q / s.n_k > 8 * kMaxGroups) return false;
+  if (c.v_stride_tok % 4 != 0 || c.v_stride_head % 4 != 0 || c.v_stride_blk % 4 != 0) return false;
+  int bt = kST;
+  if (c.page_table) {
+    if (c.page_size % 16 != 0) return false;
+    if (c.page_size < kST) { if (kST % c.page_size != 0) return false; bt = c.page_size; }
+    else if (c.page_size % kST != 0) return false;
+  }
+  *box_tok = bt;
+  return true;
+}
+
+size_t topk_decode_workspace_bytes(const diffqkv_shape& s, int max_seqlen) {
+  const size_t lpad = ((size_t)(max_seqlen > 0 ? max_seqlen : 1) + kST - 1) / kST * kST;
+  return ((size_t)s.batch * s.n_q * lpad * sizeof(float) + 255) / 256 * 256;
+}
+
+cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, int topk, int box_tok,
+                               void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream) {
+  const int sms = sm_count_topk();
+  if (sms <= 0) return cudaErrorUnknown;
+  int dev = 0, max_smem = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  const long long tok_extent = c.page_table ? c.page_size : c.max_seqlen;
+  CUtensorMap mk;
+  {
+    const cuuint64_t dims[5] = {64, (cuuint64_t)tok_extent, (cuuint64_t)(s.d_qk / 64), (cuuint64_t)s.n_k,
+                                (cuuint64_t)c.num_blocks};
+    const cuuint64_t strides[4] = {(cuuint64_t)c.k_stride_tok * 2, 128, (cuuint64_t)c.k_stride_head * 2,
+                                   (cuuint64_t)c.k_stride_blk * 2};
+    const cuuint32_t box[5] = {64, (cuuint32_t)box_tok, (cuuint32_t)(s.d_qk / 64), 1, 1};
+    if (!make_tmap_bf16_sw128(&mk, c.k_cache, 5, dims, strides, box)) return cudaErrorNotSupported;
+  }
+  ScoreParams sp;
+  sp.q = reinterpret_cast<const __nv_bfloat16*>(q);
+  sp.seqlens = c.seqlens; sp.page_table = c.page_table;
+  sp.page_size = c.page_size; sp.max_pages_per_seq = c.max_pages_per_seq;
+  sp.num_blocks = c.num_blocks; sp.max_seqlen = c.max_seqlen;
+  sp.batch = s.batch; sp.n_q = s.n_q; sp.n_k = s.n_k; sp.g_k = s.n_q / s.n_k;
+  sp.groups = (sp.g_k + 7) / 8;
+  sp.box_tok = box_tok;
+  sp.lpad = ((long long)(c.max_seqlen > 0 ? c.max_seqlen : 1) + kST - 1) / kST * kST;
+  sp.scale_log2 = s.scale * kLog2e;
+  sp.scores = reinterpret_cast<float*>(workspace);
+  sp.dev_status = dev_status;
+  const int k_tile = kST * s.d_qk * 2;
+  const int fixed = 1024 + 2 * 16 * 8 + (s.batch + 1) * 4 + 64;
+  int stages = (max_smem - fixed) / k_tile;
+  if (stages > 6) stages = 6;
+  if (stages < 2) return cudaErrorNotSupported;
+  sp.stages = stages;
+  const int smem = fixed + stages * k_tile;
+  const long long tiles_max = (long long)s.batch * s.n_k * ((c.max_seqlen + kST - 1) / kST);
+  long long grid = sms;
+  if (grid > tiles_max) grid = tiles_max;
+  if (grid < 1) grid = 1;
+
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kScoreThreads);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cudaError_t err;
+  if (s.d_qk == 128) {
+    err = cudaFuncSetAttribute(decode_scores_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (err == cudaSuccess) err = cudaLaunchKernelEx(&cfg, decode_scores_kernel<128>, mk, sp);
+  } else {
+    err = cudaFuncSetAttribute(decode_scores_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (err == cudaSuccess) err = cudaLaunchKernelEx(&cfg, decode_scores_kernel<64>, mk, sp);
+  }
+  if (err != cudaSuccess) return err;
+  count_launch();
+
+  AttendParams ap;
+  ap.scores = sp.scores; ap.lpad = sp.lpad;
+  ap.v = reinterpret_cast<const __nv_bfloat16*>(c.v_cache);
+  ap.v_sb = c.v_stride_blk; ap.v_sh = c.v_stride_head; ap.v_st = c.v_stride_tok;
+  ap.seqlens = c.seqlens; ap.page_table = c.page_table;
+  ap.page_size = c.page_size; ap.max_pages_per_seq = c.max_pages_per_seq;
+  ap.num_blocks = c.num_blocks; ap.max_seqlen = c.max_seqlen;
+  ap.batch = s.batch; ap.n_q = s.n_q; ap.n_v = s.n_v; ap.d_v = s.d_v; ap.topk = topk;
+  ap.out = out; ap.lse = lse; ap.out_is_f32 = s.out_dtype == DIFFQKV_F32;
+  ap.dev_status = dev_status;
+  cfg.gridDim = dim3((unsigned)(s.batch * s.n_q));
+  cfg.blockDim = dim3(kAttendThreads);
+  cfg.dynamicSmemBytes = 0;
+  err = cudaLaunchKernelEx(&cfg, topk_attend_kernel, ap);
+  if (err != cudaSuccess) return err;
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace diffqkv
