@@ -355,6 +355,43 @@ def time_context_sweep(api, W, device, steps):
     return rows
 
 
+def time_topk(api, W, device, host, steps, topk=100):
+    """Selective V fetching on the headline workload: the K cache is streamed once, of V only `topk` rows per query
+    head are read.  Algorithmic bytes = K bytes + gathered V rows + the fp32 scores written once and read once."""
+    import torch
+    cfg = host.cfg
+    case = DecodeCase(api, cfg, device, host_inputs=host)
+    shape = case.shape
+    nbytes = int(api._lib.diffqkv_decode_topk_workspace_bytes(__import__("ctypes").byref(shape), case.caches[0].max_seqlen, topk))
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    i = [0]
+
+    def step():
+        cache = case.caches[i[0] % case.rotate]
+        i[0] += 1
+        api.diffqkv_decode_topk(case.q, cache, cfg.n_k, cfg.n_v, cfg.scale, topk, workspace=ws, out=case.out,
+                                dev_status=case.status)
+
+    for _ in range(20):
+        step()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    assert int(case.status.item()) == 0
+    tokens = float(np.sum(host.seqlens.astype(np.int64)))
+    k_bytes = tokens * cfg.n_k * cfg.d_qk * 2
+    v_bytes = float(cfg.batch * cfg.n_q * topk * cfg.d_v * 2)
+    score_bytes = tokens * cfg.n_q * 4 * 2
+    return {"topk": topk, "ms_per_step": ms, "k_bytes": k_bytes, "v_bytes_gathered": v_bytes,
+            "score_bytes_written_and_read": score_bytes, "GB/s": (k_bytes + v_bytes + score_bytes) / ms / 1e6,
+            "k_stream_GB/s": k_bytes / ms / 1e6}
+
+
 def max_over_ranks(value: float, device) -> float:
     """The slowest rank's value (all-reduce MAX over the default process group; identity without one)."""
     import torch
@@ -444,6 +481,9 @@ def run_ours(args):
                                        "tokens_per_s_per_layer": cfg.batch / (t_ms * 1e-3)}
             line["diffqkv_vs_gqa_speedup_32k"] = t_ms / ms_per_step
             del twin
+            tk = time_topk(api, W, device, host, min(args.steps, 300))
+            tk["speedup_vs_full_v"] = ms_per_step / tk["ms_per_step"]
+            others["cfg3_selective_v_top100"] = tk
             for c in (W.CFG2, W.CFG2.gqa_twin(), W.CFG1):
                 cs = DecodeCase(api, c, device, host_inputs=W.make_decode_inputs(c))
                 c_ms = cs.time_steps(args.steps, args.warmup) / args.steps

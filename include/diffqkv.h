@@ -242,10 +242,11 @@ diffqkv_status diffqkv_cache_append(const void *k_new, const void *v_new, int32_
  * exactly the full attention of diffqkv_decode.
  *   q, cache, out, lse, dev_status as in diffqkv_decode; bf16 only, d_qk 64 or 128, at most 32 query heads per
  *   K head, 1 <= topk <= 1024, pages of 16, 32, 64 or a multiple of 128 tokens
- *   workspace  diffqkv_decode_topk_workspace_bytes(shape, cache->max_seqlen) bytes, 256-byte aligned: the fp32
- *              scores [batch, n_q, max_seqlen rounded up to 128]
+ *   workspace  diffqkv_decode_topk_workspace_bytes(shape, cache->max_seqlen, topk) bytes, 256-byte aligned: the fp32
+ *              scores [batch, n_q, max_seqlen rounded up to 128] and the per-8192-token candidates; topk times
+ *              the number of 8192-token chunks of max_seqlen may not exceed 8192
  */
-size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape *shape, int32_t max_seqlen);
+size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape *shape, int32_t max_seqlen, int32_t topk);
 diffqkv_status diffqkv_decode_topk(const void *q, const diffqkv_cache *cache, const diffqkv_shape *shape, int32_t topk,
                                    void *workspace, size_t workspace_bytes, void *out, float *lse,
                                    int32_t *dev_status, void *stream);

@@ -87,7 +87,7 @@ _lib.diffqkv_cache_append.restype = C.c_int
 _lib.diffqkv_cache_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(CacheStruct), C.POINTER(ShapeStruct),
                                       C.c_void_p, C.c_void_p]
 _lib.diffqkv_decode_topk_workspace_bytes.restype = C.c_size_t
-_lib.diffqkv_decode_topk_workspace_bytes.argtypes = [C.POINTER(ShapeStruct), C.c_int32]
+_lib.diffqkv_decode_topk_workspace_bytes.argtypes = [C.POINTER(ShapeStruct), C.c_int32, C.c_int32]
 _lib.diffqkv_decode_topk.restype = C.c_int
 _lib.diffqkv_decode_topk.argtypes = [C.c_void_p, C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_int32, C.c_void_p,
                                      C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -373,7 +373,7 @@ def diffqkv_decode_topk(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, sca
     out_dtype = out_dtype or (out.dtype if out is not None else q.dtype)
     shape = make_shape(batch, n_q, n_k, n_v, d_qk, d_v, q.dtype, out_dtype, scale)
     if workspace is None:
-        nbytes = int(_lib.diffqkv_decode_topk_workspace_bytes(C.byref(shape), cache.max_seqlen))
+        nbytes = int(_lib.diffqkv_decode_topk_workspace_bytes(C.byref(shape), cache.max_seqlen, int(topk)))
         workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
     if out is None:
         out = torch.empty((batch, n_q, d_v), dtype=out_dtype, device=q.device)

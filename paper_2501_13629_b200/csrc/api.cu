@@ -302,9 +302,9 @@ diffqkv_status diffqkv_cache_append(const void* k_new, const void* v_new, int32_
   return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
 
-size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape* shape, int32_t max_seqlen) {
-  if (check_shape(shape) != DIFFQKV_OK || max_seqlen < 0) return 0;
-  return topk_decode_workspace_bytes(*shape, max_seqlen);
+size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape* shape, int32_t max_seqlen, int32_t topk) {
+  if (check_shape(shape) != DIFFQKV_OK || max_seqlen < 0 || topk < 1) return 0;
+  return topk_decode_workspace_bytes(*shape, max_seqlen, topk);
 }
 
 diffqkv_status diffqkv_decode_topk(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape, int32_t topk,
@@ -319,7 +319,7 @@ diffqkv_status diffqkv_decode_topk(const void* q, const diffqkv_cache* cache, co
   if (shape->batch == 0) return DIFFQKV_OK;
   int box_tok = 0;
   if (!topk_decode_supported(*shape, *cache, topk, &box_tok)) return DIFFQKV_ERR_UNSUPPORTED;
-  if (!workspace || workspace_bytes < topk_decode_workspace_bytes(*shape, cache->max_seqlen)) return DIFFQKV_ERR_WORKSPACE;
+  if (!workspace || workspace_bytes < topk_decode_workspace_bytes(*shape, cache->max_seqlen, topk)) return DIFFQKV_ERR_WORKSPACE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DIFFQKV_ERR_ALIGNMENT;
   const cudaError_t err = launch_decode_topk(q, *cache, *shape, topk, box_tok, workspace, out, lse, dev_status,
                                              static_cast<cudaStream_t>(stream));

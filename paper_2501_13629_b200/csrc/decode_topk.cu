@@ -27,7 +27,7 @@ constexpr int kScoreThreads = (kScoreWarps + 1) * 32;
 constexpr int kMaxBatchScores = 2048;
 constexpr int kMaxTopk = 1024;
 constexpr int kMaxGroups = 4;       // query heads per K head <= 8 * kMaxGroups
-constexpr int kAttendThreads = 256;
+constexpr int kAttendThreads = 512;
 
 struct ScoreParams {
   const __nv_bfloat16* q;
@@ -244,9 +244,23 @@ decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScorePara
   }
 }
 
-struct AttendParams {
+constexpr int kChunk = 8192;  // scores one selection block holds in shared memory (16 per thread)
+
+struct SelectParams {
   const float* scores;
   long long lpad;
+  const int* seqlens;
+  int max_seqlen, n_q, topk, n_chunks;
+  int* cand_idx;    // [rows, n_chunks, topk] token ids of each chunk's best scores, in token order
+  float* cand_val;  // [rows, n_chunks, topk]
+  int* cand_cnt;    // [rows, n_chunks]
+};
+
+struct AttendParams {
+  const int* cand_idx;
+  const float* cand_val;
+  const int* cand_cnt;
+  int n_chunks;
   const __nv_bfloat16* v;
   long long v_sb, v_sh, v_st;
   const int* seqlens;
@@ -265,15 +279,229 @@ __device__ __forceinline__ uint32_t order_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+constexpr int kMaxCand = 2 * kMaxTopk;  // keys the fast path of the selection holds (they borrow the output arrays)
+
+struct SelectOut {
+  int pos[kMaxTopk];
+  float val[kMaxTopk];
+};
+
+struct SelectScratch {
+  unsigned hist[256];
+  unsigned warp_tot[kAttendThreads / 32];
+  float warp_max[kAttendThreads / 32];
+  unsigned prefix, need, count;
+};
+
+// The k-th largest of keys[0 .. n) (shared memory) by radix select, 8 bits a pass: returns its key in *thr and in
+// *need_eq how many keys equal to it belong to the k largest.  get_key(i) yields key i.  All threads call it.
+template <typename GetKey>
+__device__ void radix_kth(GetKey get_key, int n, int k, SelectScratch& sc, unsigned* thr, unsigned* need_eq) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  unsigned prefix = 0, mask = 0, need = (unsigned)k;
+  for (int pass = 3; pass >= 0; --pass) {
+    for (int i = tid; i < 256; i += kAttendThreads) sc.hist[i] = 0;
+    __syncthreads();
+    for (int i0 = 0; i0 < n; i0 += kAttendThreads) {
+      const int i = i0 + tid;
+      unsigned bin = 0xffffffffu;  // no contribution
+      if (i < n) {
+        const unsigned key = get_key(i);
+        if ((key & mask) == prefix) bin = (key >> (8 * pass)) & 255u;
+      }
+      // keys crowd into a few bins in the upper passes: lanes of a warp that hit the same bin add once
+      const unsigned peers = __match_any_sync(0xffffffffu, bin);
+      if (bin != 0xffffffffu && lane == __ffs(peers) - 1) atomicAdd(&sc.hist[bin], (unsigned)__popc(peers));
+    }
+    __syncthreads();
+    if (warp == 0) {  // from the top bin down: the bin that holds the need-th largest of the remaining keys
+      unsigned mine = 0;  // lane owns bins 255 - 8 lane .. 248 - 8 lane
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mine += sc.hist[255 - (lane * 8 + e)];
+      unsigned incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+      }
+      const unsigned before = incl - mine;
+      if (before < need && need <= incl) {  // exactly one lane
+        unsigned cum = before;
+        for (int e = 0; e < 8; ++e) {
+          const int bin = 255 - (lane * 8 + e);
+          if (need <= cum + sc.hist[bin]) {
+            sc.prefix = prefix | ((unsigned)bin << (8 * pass));
+            sc.need = need - cum;
+            break;
+          }
+          cum += sc.hist[bin];
+        }
+      }
+    }
+    __syncthreads();
+    prefix = sc.prefix;
+    need = sc.need;
+    mask |= 0xffu << (8 * pass);
+  }
+  *thr = prefix;
+  *need_eq = need;
+}
+
+// The k largest of vals[0 .. n) (shared or global memory, 16-byte aligned, n <= kChunk), equal values: the earlier
+// position first.  Their
+// positions and values are written to sel_pos / sel_val (shared memory, k entries) in position order.  All threads
+// of the block call it.  The k-th largest value is found among the few values within a growing distance of the
+// maximum (every value outside is smaller than every value inside, so the rank is the same); only when those do not
+// fit the candidate buffer does the radix select run over everything.
+__device__ void block_select(const float* vals, int n, int k, SelectOut& out, SelectScratch& sc) {
+  unsigned* cand_key = reinterpret_cast<unsigned*>(&out);  // dead before the output is written
+  int* sel_pos = out.pos;
+  float* sel_val = out.val;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr int kPer = kChunk / kAttendThreads;  // consecutive positions per thread
+  float sv[kPer];  // vals is 16-byte aligned: four 16-byte loads per thread
+#pragma unroll
+  for (int e4 = 0; e4 < kPer; e4 += 4) {
+    const int i = tid * kPer + e4;
+    float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    if (i + 3 < n) {
+      v = *reinterpret_cast<const float4*>(vals + i);
+    } else {
+      if (i < n) v.x = vals[i];
+      if (i + 1 < n) v.y = vals[i + 1];
+      if (i + 2 < n) v.z = vals[i + 2];
+    }
+    sv[e4] = v.x; sv[e4 + 1] = v.y; sv[e4 + 2] = v.z; sv[e4 + 3] = v.w;
+  }
+  unsigned thr = 0, need_eq = 0;
+  const bool all = n <= k;
+  if (!all) {
+    float m = -INFINITY;
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) m = fmaxf(m, sv[e]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) sc.warp_max[warp] = m;
+    __syncthreads();
+    m = sc.warp_max[0];
+#pragma unroll
+    for (int ww = 1; ww < kAttendThreads / 32; ++ww) m = fmaxf(m, sc.warp_max[ww]);
+    // widen the band below the maximum until it holds at least k values
+    float cut = m;
+    int count = 0;
+    for (float band = 1.f; band < 1e30f; band *= 2.f) {
+      cut = m - band;
+      int c = 0;
+#pragma unroll
+      for (int e = 0; e < kPer; ++e) c += sv[e] >= cut;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+      __syncthreads();  // the previous round's totals have been read
+      if (lane == 0) sc.warp_tot[warp] = (unsigned)c;
+      __syncthreads();
+      count = 0;
+#pragma unroll
+      for (int ww = 0; ww < kAttendThreads / 32; ++ww) count += (int)sc.warp_tot[ww];
+      if (count >= k) break;
+    }
+    if (count >= k && count <= kMaxCand) {
+      if (tid == 0) sc.count = 0;
+      __syncthreads();
+#pragma unroll
+      for (int e = 0; e < kPer; ++e) {
+        const bool c = sv[e] >= cut;
+        const unsigned vote = __ballot_sync(0xffffffffu, c);
+        unsigned base = 0;
+        if (lane == 0 && vote) base = atomicAdd(&sc.count, (unsigned)__popc(vote));
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (c) cand_key[base + __popc(vote & ((1u << lane) - 1u))] = order_key(sv[e]);
+      }
+      __syncthreads();
+      radix_kth([&](int i) { return cand_key[i]; }, count, k, sc, &thr, &need_eq);
+    } else {  // values too crowded (or not finite): select over all of them
+      radix_kth([&](int i) { return order_key(vals[i]); }, n, k, sc, &thr, &need_eq);
+    }
+  }
+  // compaction in position order: kept = key > thr, or key == thr among the first need_eq such positions
+  unsigned fg = 0, fe = 0;
+#pragma unroll
+  for (int e = 0; e < kPer; ++e) {
+    const int i = tid * kPer + e;
+    if (i < n) {
+      const unsigned key = order_key(sv[e]);
+      if (all || key > thr) fg |= 1u << e;
+      else if (key == thr) fe |= 1u << e;
+    }
+  }
+  const unsigned packed = __popc(fg) | ((unsigned)__popc(fe) << 16);
+  unsigned incl = packed;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  __syncthreads();  // earlier uses of warp_tot are over
+  if (lane == 31) sc.warp_tot[warp] = incl;
+  __syncthreads();
+  unsigned before = incl - packed;
+  for (int ww = 0; ww < warp; ++ww) before += sc.warp_tot[ww];
+  unsigned gt_before = before & 0xffffu, eq_before = before >> 16;
+#pragma unroll
+  for (int e = 0; e < kPer; ++e) {
+    const bool g = (fg >> e) & 1u, q = (fe >> e) & 1u;
+    if (g || (q && eq_before < need_eq)) {
+      const unsigned pos = gt_before + min(eq_before, need_eq);
+      sel_pos[pos] = tid * kPer + e;
+      sel_val[pos] = sv[e];
+    }
+    gt_before += g;
+    eq_before += q;
+  }
+  __syncthreads();
+}
+
+// Per (row, chunk of 8192 tokens): the chunk's topk best scores, as candidates for the row's selection.
+__global__ void __launch_bounds__(kAttendThreads)
+topk_select_kernel(const SelectParams p) {
+  __shared__ SelectOut sel;
+  __shared__ SelectScratch sc;
+  ptx::grid_launch_dependents();
+  const int tid = threadIdx.x;
+  const int rowid = blockIdx.x / p.n_chunks, chunk = blockIdx.x % p.n_chunks;
+  const int b = rowid / p.n_q;
+  ptx::grid_dependency_wait();
+  const int len = min(max(p.seqlens[b], 0), p.max_seqlen);
+  const int base = chunk * kChunk;
+  const int n = min(kChunk, len - base);
+  int* cnt = p.cand_cnt + (long long)rowid * p.n_chunks + chunk;
+  if (n <= 0) {
+    if (tid == 0) *cnt = 0;
+    return;
+  }
+  const float* row = p.scores + (long long)rowid * p.lpad + base;  // read straight into registers
+  const int k = min(p.topk, n);
+  block_select(row, n, k, sel, sc);
+  const long long out0 = ((long long)rowid * p.n_chunks + chunk) * p.topk;
+  for (int i = tid; i < k; i += kAttendThreads) {
+    p.cand_idx[out0 + i] = base + sel.pos[i];
+    p.cand_val[out0 + i] = sel.val[i];
+  }
+  if (tid == 0) *cnt = k;
+}
+
+// Per (sequence, query head): the topk best of the chunks' candidates, softmax over them, gather of their V rows.
 __global__ void __launch_bounds__(kAttendThreads)
 topk_attend_kernel(const AttendParams p) {
-  __shared__ unsigned hist[256];
-  __shared__ int sel_idx[kMaxTopk];
-  __shared__ float sel_s[kMaxTopk];
-  __shared__ unsigned warp_tot[kAttendThreads / 32];
-  __shared__ unsigned sh_prefix, sh_need;
+  extern __shared__ float attend_dyn[];  // vals[kChunk], tok[kChunk], acc[warps][d_v]
+  float* vals = attend_dyn;
+  int* tok = reinterpret_cast<int*>(attend_dyn + kChunk);
+  float* acc_dyn = attend_dyn + 2 * kChunk;
+  __shared__ SelectOut sel;
+  __shared__ SelectScratch sc;
+  __shared__ int chunk_off[65];
+  int* sel_idx = sel.pos;
+  float* sel_s = sel.val;
   __shared__ float red[kAttendThreads / 32];
-  __shared__ float acc_s[kAttendThreads / 32][512];
 
   ptx::grid_launch_dependents();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -290,101 +518,31 @@ topk_attend_kernel(const AttendParams p) {
     if (p.lse && tid == 0) p.lse[(long long)b * p.n_q + h] = -INFINITY;
     return;
   }
-  const float* row = p.scores + ((long long)b * p.n_q + h) * p.lpad;
-  const int k = min(p.topk, len);
-
-  // ---- the key of the k-th largest score, 8 bits at a time from the top, and how many equal ones to take
-  unsigned thr = 0, need_eq = 0;
-  const bool all = len <= p.topk;
-  if (!all) {
-    unsigned prefix = 0, mask = 0, need = (unsigned)k;
-    for (int pass = 3; pass >= 0; --pass) {
-      for (int i = tid; i < 256; i += kAttendThreads) hist[i] = 0;
-      __syncthreads();
-      for (int i = tid; i < len; i += kAttendThreads) {
-        const unsigned key = order_key(row[i]);
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> (8 * pass)) & 255u], 1u);
-      }
-      __syncthreads();
-      if (warp == 0) {  // from the top bin down: the bin that holds the need-th largest of the remaining keys
-        unsigned mine = 0;  // lane owns bins 255 - 8 lane .. 248 - 8 lane
-#pragma unroll
-        for (int e = 0; e < 8; ++e) mine += hist[255 - (lane * 8 + e)];
-        unsigned incl = mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
-          if (lane >= o) incl += y;
-        }
-        const unsigned before = incl - mine;
-        if (before < need && need <= incl) {  // exactly one lane
-          unsigned cum = before;
-          for (int e = 0; e < 8; ++e) {
-            const int bin = 255 - (lane * 8 + e);
-            if (need <= cum + hist[bin]) {
-              sh_prefix = prefix | ((unsigned)bin << (8 * pass));
-              sh_need = need - cum;
-              break;
-            }
-            cum += hist[bin];
-          }
-        }
-      }
-      __syncthreads();
-      prefix = sh_prefix;
-      need = sh_need;
-      mask |= 0xffu << (8 * pass);
+  // ---- the chunks' candidates, concatenated in token order
+  const long long rowid = blockIdx.x;
+  if (tid == 0) {
+    int run = 0;
+    for (int c = 0; c < p.n_chunks; ++c) {
+      chunk_off[c] = run;
+      run += p.cand_cnt[rowid * p.n_chunks + c];
     }
-    thr = prefix;
-    need_eq = need;
+    chunk_off[p.n_chunks] = run;
   }
-
-  // ---- compaction in token order: kept = key > thr, or key == thr among the first need_eq such tokens
-  unsigned base_gt = 0, base_eq = 0;
-  for (int base = 0; base < len; base += kAttendThreads * 4) {
-    float sv[4];
-    unsigned fg = 0, fe = 0;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int i = base + tid * 4 + e;
-      sv[e] = i < len ? row[i] : 0.f;
-      if (i < len) {
-        const unsigned key = order_key(sv[e]);
-        if (all || key > thr) fg |= 1u << e;
-        else if (key == thr) fe |= 1u << e;
-      }
+  __syncthreads();
+  const int n = chunk_off[p.n_chunks];
+  for (int c = 0; c < p.n_chunks; ++c) {
+    const int cnt = chunk_off[c + 1] - chunk_off[c];
+    const long long src = (rowid * p.n_chunks + c) * p.topk;
+    for (int i = tid; i < cnt; i += kAttendThreads) {
+      vals[chunk_off[c] + i] = p.cand_val[src + i];
+      tok[chunk_off[c] + i] = p.cand_idx[src + i];
     }
-    const unsigned packed = __popc(fg) | ((unsigned)__popc(fe) << 16);
-    unsigned incl = packed;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += y;
-    }
-    if (lane == 31) warp_tot[warp] = incl;
-    __syncthreads();
-    unsigned before = incl - packed, chunk_tot = 0;
-#pragma unroll
-    for (int ww = 0; ww < kAttendThreads / 32; ++ww) {
-      if (ww < warp) before += warp_tot[ww];
-      chunk_tot += warp_tot[ww];
-    }
-    unsigned gt_before = base_gt + (before & 0xffffu), eq_before = base_eq + (before >> 16);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const bool g = (fg >> e) & 1u, q = (fe >> e) & 1u;
-      if (g || (q && eq_before < need_eq)) {
-        const unsigned pos = gt_before + min(eq_before, need_eq);
-        sel_idx[pos] = base + tid * 4 + e;
-        sel_s[pos] = sv[e];
-      }
-      gt_before += g;
-      eq_before += q;
-    }
-    base_gt += chunk_tot & 0xffffu;
-    base_eq += chunk_tot >> 16;
-    __syncthreads();  // warp_tot is reused by the next chunk
   }
+  __syncthreads();
+  const int k = min(p.topk, n);
+  block_select(vals, n, k, sel, sc);
+  for (int i = tid; i < k; i += kAttendThreads) sel_idx[i] = tok[sel_idx[i]];
+  __syncthreads();
 
   // ---- softmax over the kept scores (base-2 domain)
   float m = -INFINITY;
@@ -437,7 +595,8 @@ topk_attend_kernel(const AttendParams p) {
       }
     }
     if (in) {
-      acc_s[warp][ch] = a.x; acc_s[warp][ch + 1] = a.y; acc_s[warp][ch + 2] = a.z; acc_s[warp][ch + 3] = a.w;
+      float* dst = acc_dyn + warp * p.d_v + ch;
+      dst[0] = a.x; dst[1] = a.y; dst[2] = a.z; dst[3] = a.w;
     }
   }
   __syncthreads();
@@ -445,7 +604,7 @@ topk_attend_kernel(const AttendParams p) {
   for (int ch = tid; ch < p.d_v; ch += kAttendThreads) {
     float o = 0.f;
 #pragma unroll
-    for (int ww = 0; ww < kAttendThreads / 32; ++ww) o += acc_s[ww][ch];
+    for (int ww = 0; ww < kAttendThreads / 32; ++ww) o += acc_dyn[ww * p.d_v + ch];
     o *= inv;
     if (p.out_is_f32) reinterpret_cast<float*>(p.out)[orow + ch] = o;
     else reinterpret_cast<__nv_bfloat16*>(p.out)[orow + ch] = __float2bfloat16_rn(o);
@@ -462,11 +621,15 @@ int sm_count_topk() {
 
 }  // namespace
 
+static int topk_chunks(int max_seqlen) { return ((max_seqlen > 0 ? max_seqlen : 1) + kChunk - 1) / kChunk; }
+
 bool topk_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, int topk, int* box_tok) {
   if (s.dtype != DIFFQKV_BF16 || (s.d_qk != 64 && s.d_qk != 128)) return false;
   if (s.d_v % 4 != 0 || s.d_v > 512 || topk < 1 || topk > kMaxTopk) return false;
   if (s.batch < 1 || s.batch > kMaxBatchScores || s.n_q / s.n_k > 8 * kMaxGroups) return false;
   if (c.v_stride_tok % 4 != 0 || c.v_stride_head % 4 != 0 || c.v_stride_blk % 4 != 0) return false;
+  const int chunks = topk_chunks(c.max_seqlen);
+  if (chunks > 64 || (long long)chunks * topk > kChunk) return false;  // the row's candidates must fit one block
   int bt = kST;
   if (c.page_table) {
     if (c.page_size % 16 != 0) return false;
@@ -477,9 +640,12 @@ bool topk_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, int t
   return true;
 }
 
-size_t topk_decode_workspace_bytes(const diffqkv_shape& s, int max_seqlen) {
+static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+
+size_t topk_decode_workspace_bytes(const diffqkv_shape& s, int max_seqlen, int topk) {
   const size_t lpad = ((size_t)(max_seqlen > 0 ? max_seqlen : 1) + kST - 1) / kST * kST;
-  return ((size_t)s.batch * s.n_q * lpad * sizeof(float) + 255) / 256 * 256;
+  const size_t rows = (size_t)s.batch * s.n_q, chunks = (size_t)topk_chunks(max_seqlen);
+  return up256(rows * lpad * sizeof(float)) + 2 * up256(rows * chunks * (size_t)topk * 4) + up256(rows * chunks * 4);
 }
 
 cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, int topk, int box_tok,
@@ -544,8 +710,26 @@ cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diff
   if (err != cudaSuccess) return err;
   count_launch();
 
+  const size_t rows = (size_t)s.batch * s.n_q;
+  const int chunks = topk_chunks(c.max_seqlen);
+  char* ws = reinterpret_cast<char*>(workspace) + up256(rows * (size_t)sp.lpad * sizeof(float));
+  SelectParams sel;
+  sel.scores = sp.scores; sel.lpad = sp.lpad; sel.seqlens = c.seqlens; sel.max_seqlen = c.max_seqlen;
+  sel.n_q = s.n_q; sel.topk = topk; sel.n_chunks = chunks;
+  sel.cand_idx = reinterpret_cast<int*>(ws);
+  ws += up256(rows * chunks * (size_t)topk * 4);
+  sel.cand_val = reinterpret_cast<float*>(ws);
+  ws += up256(rows * chunks * (size_t)topk * 4);
+  sel.cand_cnt = reinterpret_cast<int*>(ws);
+  cfg.gridDim = dim3((unsigned)(rows * chunks));
+  cfg.blockDim = dim3(kAttendThreads);
+  cfg.dynamicSmemBytes = 0;
+  err = cudaLaunchKernelEx(&cfg, topk_select_kernel, sel);
+  if (err != cudaSuccess) return err;
+  count_launch();
+
   AttendParams ap;
-  ap.scores = sp.scores; ap.lpad = sp.lpad;
+  ap.cand_idx = sel.cand_idx; ap.cand_val = sel.cand_val; ap.cand_cnt = sel.cand_cnt; ap.n_chunks = chunks;
   ap.v = reinterpret_cast<const __nv_bfloat16*>(c.v_cache);
   ap.v_sb = c.v_stride_blk; ap.v_sh = c.v_stride_head; ap.v_st = c.v_stride_tok;
   ap.seqlens = c.seqlens; ap.page_table = c.page_table;
@@ -554,9 +738,10 @@ cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diff
   ap.batch = s.batch; ap.n_q = s.n_q; ap.n_v = s.n_v; ap.d_v = s.d_v; ap.topk = topk;
   ap.out = out; ap.lse = lse; ap.out_is_f32 = s.out_dtype == DIFFQKV_F32;
   ap.dev_status = dev_status;
-  cfg.gridDim = dim3((unsigned)(s.batch * s.n_q));
-  cfg.blockDim = dim3(kAttendThreads);
-  cfg.dynamicSmemBytes = 0;
+  cfg.gridDim = dim3((unsigned)rows);
+  cfg.dynamicSmemBytes = (size_t)(2 * kChunk + (kAttendThreads / 32) * s.d_v) * sizeof(float);
+  err = cudaFuncSetAttribute(topk_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg.dynamicSmemBytes);
+  if (err != cudaSuccess) return err;
   err = cudaLaunchKernelEx(&cfg, topk_attend_kernel, ap);
   if (err != cudaSuccess) return err;
   count_launch();
