@@ -7,10 +7,11 @@
 //                          m16n8k16, fp32 accumulation); scores go to a workspace as fp32, already multiplied by
 //                          scale * log2(e).  All (sequence, K head, tile) triples form one flat list divided evenly
 //                          over one block per SM; tiles are independent, so nothing has to be merged.
-//   topk_attend_kernel     one block per (sequence, query head): radix select (4 passes of 8 bits over an order-
-//                          preserving key) finds the k-th largest score; the kept tokens are compacted in token order
-//                          (equal scores: the earlier token first, as the definition says); softmax over the kept
-//                          scores; the k V rows are gathered with 16-byte loads and accumulated in fp32.
+//   topk_attend_kernel     one block per (sequence, query head) holds the row's scores in registers (64 per thread,
+//                          32768 per pass), finds the k-th largest (radix select, 8 bits a pass over an order-
+//                          preserving key, run on the few scores near the maximum), compacts the kept tokens in
+//                          token order (equal scores: the earlier token first, as the definition says), takes the
+//                          softmax over the kept scores, gathers the k V rows and accumulates them in fp32.
 // Both are launched with programmatic stream serialisation and wait on the device before touching their inputs.
 #include <cuda.h>
 
@@ -22,7 +23,7 @@ namespace diffqkv {
 namespace {
 
 constexpr int kST = 128;            // tokens per K tile
-constexpr int kScoreWarps = 4;      // consumer warps, 32 tokens each
+constexpr int kScoreWarps = 8;      // consumer warps, 16 tokens each
 constexpr int kScoreThreads = (kScoreWarps + 1) * 32;
 constexpr int kMaxBatchScores = 2048;
 constexpr int kMaxTopk = 1024;
@@ -179,11 +180,21 @@ decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScorePara
   auto row_index = [&](int r, int h) { return (((r >> bt_shift) * HK + h) << bt_shift) + (r & bt_mask); };
   int stage = 0;
   uint32_t phase = 0;
-  int cur_b = -1, cur_u = -1;
+  int cur_b = -1, cur_u = -1, len = 0;
+  float* srow = nullptr;  // score row of the first query head of the current K head
   uint32_t qf[kMaxGroups][KS][2];
+  const int row0 = warp * 16;
+  const int r = row0 + (lane & 7) + 8 * ((lane >> 3) & 1);
+  const int csel = lane >> 4;
+  uint32_t a_off[KS];  // byte offset of this lane's ldmatrix row in a stage, per 16-channel step
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks)
+    a_off[ks] = row_index(r, ks / 4) * 128 + ((((ks % 4) * 2 + csel) ^ (r & 7)) << 4);
   for (; w.g < g_end; w.advance(prefix, p.batch, p.n_k)) {
     if (w.b != cur_b || w.u != cur_u) {  // Q^T fragments of the query heads of this K head, 8 heads per group
       cur_b = w.b; cur_u = w.u;
+      len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
+      srow = p.scores + ((long long)w.b * p.n_q + (long long)w.u * p.g_k) * p.lpad;
 #pragma unroll
       for (int gq = 0; gq < kMaxGroups; ++gq) {
         const int hq = gq * 8 + g8;
@@ -196,32 +207,25 @@ decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScorePara
         }
       }
     }
-    if (!ptx::mbar_wait(full0 + 8 * stage, phase, abort_flag)) {  // all four warps give up at the same stage
+    if (!ptx::mbar_wait(full0 + 8 * stage, phase, abort_flag)) {  // all warps give up at the same stage
       report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
       break;
     }
-    const int len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
     const int n_valid = min(kST, len - w.t * kST);
-    const uint32_t st_u32 = ptx::smem_u32(smem + (size_t)stage * K_TILE);
-#pragma unroll
-    for (int rb = 0; rb < 2; ++rb) {
-      const int row0 = warp * 32 + rb * 16;
-      if (row0 >= n_valid) continue;
-      float s[kMaxGroups][4];
+    if (row0 < n_valid) {
+      const uint32_t st_u32 = ptx::smem_u32(smem + (size_t)stage * K_TILE);
+      float s[kMaxGroups][2][4];  // two accumulation chains per group (even and odd 16-channel steps)
 #pragma unroll
       for (int gq = 0; gq < kMaxGroups; ++gq)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) s[gq][e] = 0.f;
-      const int r = row0 + (lane & 7) + 8 * ((lane >> 3) & 1);
-      const int csel = lane >> 4;
+        for (int e = 0; e < 4; ++e) s[gq][0][e] = s[gq][1][e] = 0.f;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
-        const int chunk = (ks % 4) * 2 + csel;
         uint32_t a[4];
-        ptx::ldmatrix_x4(st_u32 + row_index(r, ks / 4) * 128 + ((chunk ^ (r & 7)) << 4), a);
+        ptx::ldmatrix_x4(st_u32 + a_off[ks], a);
 #pragma unroll
         for (int gq = 0; gq < kMaxGroups; ++gq)
-          if (gq < p.groups) ptx::mma_bf16_16816(s[gq], a, qf[gq][ks][0], qf[gq][ks][1]);
+          if (gq < p.groups) ptx::mma_bf16_16816(s[gq][ks & 1], a, qf[gq][ks][0], qf[gq][ks][1]);
       }
       // thread holds token rows g8, g8 + 8 of the block and head columns 2 t4, 2 t4 + 1 of each group
       const long long tok = (long long)w.t * kST + row0 + g8;
@@ -232,9 +236,9 @@ decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScorePara
         for (int c = 0; c < 2; ++c) {
           const int hq = gq * 8 + 2 * t4 + c;
           if (hq >= p.g_k) continue;
-          float* dst = p.scores + ((long long)w.b * p.n_q + (long long)w.u * p.g_k + hq) * p.lpad + tok;
-          if (row0 + g8 < n_valid) dst[0] = s[gq][c] * p.scale_log2;
-          if (row0 + g8 + 8 < n_valid) dst[8] = s[gq][2 + c] * p.scale_log2;
+          float* dst = srow + (long long)hq * p.lpad + tok;
+          if (row0 + g8 < n_valid) dst[0] = (s[gq][0][c] + s[gq][1][c]) * p.scale_log2;
+          if (row0 + g8 + 8 < n_valid) dst[8] = (s[gq][0][2 + c] + s[gq][1][2 + c]) * p.scale_log2;
         }
       }
     }
@@ -244,23 +248,16 @@ decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScorePara
   }
 }
 
-constexpr int kChunk = 8192;  // scores one selection block holds in shared memory (16 per thread)
-
-struct SelectParams {
-  const float* scores;
-  long long lpad;
-  const int* seqlens;
-  int max_seqlen, n_q, topk, n_chunks;
-  int* cand_idx;    // [rows, n_chunks, topk] token ids of each chunk's best scores, in token order
-  float* cand_val;  // [rows, n_chunks, topk]
-  int* cand_cnt;    // [rows, n_chunks]
-};
+constexpr int kPiece = 32768;            // scores one selection holds in registers (64 per thread)
+constexpr int kPerThread = kPiece / kAttendThreads;
+constexpr int kQuads = kPerThread / 4;   // 16-byte loads per thread
+constexpr int kWarpSpan = 32 * kPerThread;
+constexpr int kMaxCand = 8192;           // keys the fast path of the selection holds; also the merge capacity
+constexpr int kAttendWarps = kAttendThreads / 32;
 
 struct AttendParams {
-  const int* cand_idx;
-  const float* cand_val;
-  const int* cand_cnt;
-  int n_chunks;
+  const float* scores;
+  long long lpad;
   const __nv_bfloat16* v;
   long long v_sb, v_sh, v_st;
   const int* seqlens;
@@ -279,8 +276,6 @@ __device__ __forceinline__ uint32_t order_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-constexpr int kMaxCand = 2 * kMaxTopk;  // keys the fast path of the selection holds (they borrow the output arrays)
-
 struct SelectOut {
   int pos[kMaxTopk];
   float val[kMaxTopk];
@@ -288,56 +283,52 @@ struct SelectOut {
 
 struct SelectScratch {
   unsigned hist[256];
-  unsigned warp_tot[kAttendThreads / 32];
-  float warp_max[kAttendThreads / 32];
+  unsigned warp_tot[2][kAttendWarps];
+  float warp_max[kAttendWarps];
   unsigned prefix, need, count;
 };
 
-// The k-th largest of keys[0 .. n) (shared memory) by radix select, 8 bits a pass: returns its key in *thr and in
-// *need_eq how many keys equal to it belong to the k largest.  get_key(i) yields key i.  All threads call it.
-template <typename GetKey>
-__device__ void radix_kth(GetKey get_key, int n, int k, SelectScratch& sc, unsigned* thr, unsigned* need_eq) {
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+// From the top bin down: the bin of sc.hist that holds the need-th largest of the keys counted there.  Warp 0 calls
+// it; the winning lane publishes the extended prefix and the rank that remains inside the bin.
+__device__ __forceinline__ void pick_bin(SelectScratch& sc, unsigned prefix, unsigned need, int pass) {
+  const int lane = threadIdx.x & 31;
+  unsigned mine = 0;  // lane owns bins 255 - 8 lane .. 248 - 8 lane
+#pragma unroll
+  for (int e = 0; e < 8; ++e) mine += sc.hist[255 - (lane * 8 + e)];
+  unsigned incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  const unsigned before = incl - mine;
+  if (before < need && need <= incl) {  // exactly one lane
+    unsigned cum = before;
+    for (int e = 0; e < 8; ++e) {
+      const int bin = 255 - (lane * 8 + e);
+      if (need <= cum + sc.hist[bin]) {
+        sc.prefix = prefix | ((unsigned)bin << (8 * pass));
+        sc.need = need - cum;
+        break;
+      }
+      cum += sc.hist[bin];
+    }
+  }
+}
+
+// The k-th largest of n keys by radix select, 8 bits a pass: its key in *thr, and in *need_eq how many keys equal to
+// it belong to the k largest.  count_pass(mask, prefix, pass) adds every key with (key & mask) == prefix to
+// sc.hist[(key >> 8 pass) & 255].  All threads of the block call it.
+template <typename CountPass>
+__device__ void radix_kth(CountPass count_pass, int k, SelectScratch& sc, unsigned* thr, unsigned* need_eq) {
+  const int tid = threadIdx.x;
   unsigned prefix = 0, mask = 0, need = (unsigned)k;
   for (int pass = 3; pass >= 0; --pass) {
     for (int i = tid; i < 256; i += kAttendThreads) sc.hist[i] = 0;
     __syncthreads();
-    for (int i0 = 0; i0 < n; i0 += kAttendThreads) {
-      const int i = i0 + tid;
-      unsigned bin = 0xffffffffu;  // no contribution
-      if (i < n) {
-        const unsigned key = get_key(i);
-        if ((key & mask) == prefix) bin = (key >> (8 * pass)) & 255u;
-      }
-      // keys crowd into a few bins in the upper passes: lanes of a warp that hit the same bin add once
-      const unsigned peers = __match_any_sync(0xffffffffu, bin);
-      if (bin != 0xffffffffu && lane == __ffs(peers) - 1) atomicAdd(&sc.hist[bin], (unsigned)__popc(peers));
-    }
+    count_pass(mask, prefix, pass);
     __syncthreads();
-    if (warp == 0) {  // from the top bin down: the bin that holds the need-th largest of the remaining keys
-      unsigned mine = 0;  // lane owns bins 255 - 8 lane .. 248 - 8 lane
-#pragma unroll
-      for (int e = 0; e < 8; ++e) mine += sc.hist[255 - (lane * 8 + e)];
-      unsigned incl = mine;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += y;
-      }
-      const unsigned before = incl - mine;
-      if (before < need && need <= incl) {  // exactly one lane
-        unsigned cum = before;
-        for (int e = 0; e < 8; ++e) {
-          const int bin = 255 - (lane * 8 + e);
-          if (need <= cum + sc.hist[bin]) {
-            sc.prefix = prefix | ((unsigned)bin << (8 * pass));
-            sc.need = need - cum;
-            break;
-          }
-          cum += sc.hist[bin];
-        }
-      }
-    }
+    if (tid < 32) pick_bin(sc, prefix, need, pass);
     __syncthreads();
     prefix = sc.prefix;
     need = sc.need;
@@ -347,22 +338,23 @@ __device__ void radix_kth(GetKey get_key, int n, int k, SelectScratch& sc, unsig
   *need_eq = need;
 }
 
-// The k largest of vals[0 .. n) (shared or global memory, 16-byte aligned, n <= kChunk), equal values: the earlier
-// position first.  Their
-// positions and values are written to sel_pos / sel_val (shared memory, k entries) in position order.  All threads
-// of the block call it.  The k-th largest value is found among the few values within a growing distance of the
-// maximum (every value outside is smaller than every value inside, so the rank is the same); only when those do not
-// fit the candidate buffer does the radix select run over everything.
-__device__ void block_select(const float* vals, int n, int k, SelectOut& out, SelectScratch& sc) {
-  unsigned* cand_key = reinterpret_cast<unsigned*>(&out);  // dead before the output is written
-  int* sel_pos = out.pos;
-  float* sel_val = out.val;
+// The k largest of vals[0 .. n) (shared or global memory, 16-byte aligned, n <= kPiece); of equal values the earlier
+// position wins.  Their positions and values go to `out` in position order.  All threads of the block call it.
+//
+// Every thread keeps 64 values in registers: warp w, 16-byte load j, lane l hold positions 2048 w + 128 j + 4 l + c,
+// so each load instruction of a warp reads 512 consecutive bytes.  The k-th largest value is first sought among the
+// few values within a distance `band` of the maximum (every value outside is smaller than every value inside, so the
+// rank is unchanged); the band doubles until it holds k values and is bisected back if it then holds more than the
+// candidate buffer.  Only when no band fits (values crowded on one point, or not finite) does the radix select run
+// over all values.
+__device__ __noinline__ void block_select(const float* vals, int n, int k, SelectOut& out, SelectScratch& sc,
+                                          unsigned* cand_key) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  constexpr int kPer = kChunk / kAttendThreads;  // consecutive positions per thread
-  float sv[kPer];  // vals is 16-byte aligned: four 16-byte loads per thread
+  const int my0 = warp * kWarpSpan + lane * 4;  // position of quad j, element c: my0 + 128 j + c
+  float sv[kPerThread];
 #pragma unroll
-  for (int e4 = 0; e4 < kPer; e4 += 4) {
-    const int i = tid * kPer + e4;
+  for (int j = 0; j < kQuads; ++j) {
+    const int i = my0 + j * 128;
     float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     if (i + 3 < n) {
       v = *reinterpret_cast<const float4*>(vals + i);
@@ -371,139 +363,174 @@ __device__ void block_select(const float* vals, int n, int k, SelectOut& out, Se
       if (i + 1 < n) v.y = vals[i + 1];
       if (i + 2 < n) v.z = vals[i + 2];
     }
-    sv[e4] = v.x; sv[e4 + 1] = v.y; sv[e4 + 2] = v.z; sv[e4 + 3] = v.w;
+    sv[4 * j] = v.x; sv[4 * j + 1] = v.y; sv[4 * j + 2] = v.z; sv[4 * j + 3] = v.w;
   }
   unsigned thr = 0, need_eq = 0;
   const bool all = n <= k;
   if (!all) {
     float m = -INFINITY;
 #pragma unroll
-    for (int e = 0; e < kPer; ++e) m = fmaxf(m, sv[e]);
+    for (int e = 0; e < kPerThread; ++e) m = fmaxf(m, sv[e]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     if (lane == 0) sc.warp_max[warp] = m;
     __syncthreads();
     m = sc.warp_max[0];
 #pragma unroll
-    for (int ww = 1; ww < kAttendThreads / 32; ++ww) m = fmaxf(m, sc.warp_max[ww]);
-    // widen the band below the maximum until it holds at least k values
-    float cut = m;
-    int count = 0;
-    for (float band = 1.f; band < 1e30f; band *= 2.f) {
-      cut = m - band;
+    for (int ww = 1; ww < kAttendWarps; ++ww) m = fmaxf(m, sc.warp_max[ww]);
+
+    int round = 0, mine = 0;
+    auto count_ge = [&](float cut) {  // values >= cut in the block (cut finite: the padding never counts)
       int c = 0;
 #pragma unroll
-      for (int e = 0; e < kPer; ++e) c += sv[e] >= cut;
+      for (int e = 0; e < kPerThread; ++e) c += sv[e] >= cut;
+      mine = c;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-      __syncthreads();  // the previous round's totals have been read
-      if (lane == 0) sc.warp_tot[warp] = (unsigned)c;
+      unsigned* tot = sc.warp_tot[round & 1];  // alternate buffers: one barrier a round is enough
+      ++round;
+      if (lane == 0) tot[warp] = (unsigned)c;
       __syncthreads();
-      count = 0;
+      int total = 0;
 #pragma unroll
-      for (int ww = 0; ww < kAttendThreads / 32; ++ww) count += (int)sc.warp_tot[ww];
-      if (count >= k) break;
+      for (int ww = 0; ww < kAttendWarps; ++ww) total += (int)tot[ww];
+      return total;
+    };
+    float cut = m, lo = 0.f, hi = 0.f;
+    int count = 0;
+    bool fits = false;
+    if (m > -INFINITY && m < INFINITY) {
+      for (hi = 1.f; hi < 1e30f; hi *= 2.f) {
+        cut = m - hi;
+        count = count_ge(cut);
+        if (count >= k) break;
+        lo = hi;
+      }
+      for (int it = 0; it < 12 && count > kMaxCand; ++it) {  // too many: bisect between the last two bands
+        const float mid = 0.5f * (lo + hi);
+        cut = m - mid;
+        count = count_ge(cut);
+        if (count < k) { lo = mid; count = kMaxCand + 1; } else hi = mid;
+      }
+      fits = count >= k && count <= kMaxCand;
     }
-    if (count >= k && count <= kMaxCand) {
+    if (fits) {
+      // every thread appends its own candidates (any order will do for the rank)
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+      }
       if (tid == 0) sc.count = 0;
       __syncthreads();
+      unsigned base = 0;
+      if (lane == 31 && incl) base = atomicAdd(&sc.count, (unsigned)incl);
+      base = __shfl_sync(0xffffffffu, base, 31) + (unsigned)(incl - mine);
 #pragma unroll
-      for (int e = 0; e < kPer; ++e) {
-        const bool c = sv[e] >= cut;
-        const unsigned vote = __ballot_sync(0xffffffffu, c);
-        unsigned base = 0;
-        if (lane == 0 && vote) base = atomicAdd(&sc.count, (unsigned)__popc(vote));
-        base = __shfl_sync(0xffffffffu, base, 0);
-        if (c) cand_key[base + __popc(vote & ((1u << lane) - 1u))] = order_key(sv[e]);
-      }
+      for (int e = 0; e < kPerThread; ++e)
+        if (sv[e] >= cut) cand_key[base++] = order_key(sv[e]);
       __syncthreads();
-      radix_kth([&](int i) { return cand_key[i]; }, count, k, sc, &thr, &need_eq);
-    } else {  // values too crowded (or not finite): select over all of them
-      radix_kth([&](int i) { return order_key(vals[i]); }, n, k, sc, &thr, &need_eq);
+      const int ncand = count;
+      radix_kth(
+          [&](unsigned mask, unsigned prefix, int pass) {
+            for (int i0 = 0; i0 < ncand; i0 += kAttendThreads) {
+              const int i = i0 + tid;
+              unsigned bin = 0xffffffffu;  // no contribution
+              if (i < ncand) {
+                const unsigned key = cand_key[i];
+                if ((key & mask) == prefix) bin = (key >> (8 * pass)) & 255u;
+              }
+              // keys crowd into a few bins in the upper passes: lanes of a warp that hit the same bin add once
+              const unsigned peers = __match_any_sync(0xffffffffu, bin);
+              if (bin != 0xffffffffu && lane == __ffs(peers) - 1) atomicAdd(&sc.hist[bin], (unsigned)__popc(peers));
+            }
+          },
+          k, sc, &thr, &need_eq);
+    } else {
+      radix_kth(
+          [&](unsigned mask, unsigned prefix, int pass) {
+#pragma unroll
+            for (int e = 0; e < kPerThread; ++e) {
+              const unsigned key = order_key(sv[e]);
+              if (my0 + (e >> 2) * 128 + (e & 3) < n && (key & mask) == prefix)
+                atomicAdd(&sc.hist[(key >> (8 * pass)) & 255u], 1u);
+            }
+          },
+          k, sc, &thr, &need_eq);
     }
   }
   // compaction in position order: kept = key > thr, or key == thr among the first need_eq such positions
-  unsigned fg = 0, fe = 0;
+  auto flags = [&](int j, unsigned& g4, unsigned& q4) {
+    g4 = 0; q4 = 0;
 #pragma unroll
-  for (int e = 0; e < kPer; ++e) {
-    const int i = tid * kPer + e;
-    if (i < n) {
-      const unsigned key = order_key(sv[e]);
-      if (all || key > thr) fg |= 1u << e;
-      else if (key == thr) fe |= 1u << e;
+    for (int c = 0; c < 4; ++c) {
+      const unsigned key = order_key(sv[4 * j + c]);
+      const bool valid = my0 + j * 128 + c < n;
+      if (valid && (all || key > thr)) g4 |= 1u << c;
+      else if (valid && key == thr) q4 |= 1u << c;
     }
-  }
-  const unsigned packed = __popc(fg) | ((unsigned)__popc(fe) << 16);
-  unsigned incl = packed;
+  };
+  unsigned packed = 0;  // kept-for-sure count in the low half, equal-to-threshold count in the high half
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += y;
+  for (int j = 0; j < kQuads; ++j) {
+    unsigned g4, q4;
+    flags(j, g4, q4);
+    packed += __popc(g4) | ((unsigned)__popc(q4) << 16);
   }
-  __syncthreads();  // earlier uses of warp_tot are over
-  if (lane == 31) sc.warp_tot[warp] = incl;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) packed += __shfl_xor_sync(0xffffffffu, packed, o);
+  unsigned* tot = sc.warp_tot[0];
+  __syncthreads();  // earlier uses of the totals are over
+  if (lane == 0) tot[warp] = packed;
   __syncthreads();
-  unsigned before = incl - packed;
-  for (int ww = 0; ww < warp; ++ww) before += sc.warp_tot[ww];
-  unsigned gt_before = before & 0xffffu, eq_before = before >> 16;
+  unsigned run = 0;
+  for (int ww = 0; ww < warp; ++ww) run += tot[ww];
 #pragma unroll
-  for (int e = 0; e < kPer; ++e) {
-    const bool g = (fg >> e) & 1u, q = (fe >> e) & 1u;
-    if (g || (q && eq_before < need_eq)) {
-      const unsigned pos = gt_before + min(eq_before, need_eq);
-      sel_pos[pos] = tid * kPer + e;
-      sel_val[pos] = sv[e];
+  for (int j = 0; j < kQuads; ++j) {
+    unsigned g4, q4;
+    flags(j, g4, q4);
+    if (__ballot_sync(0xffffffffu, (g4 | q4) != 0) == 0) continue;  // nothing of this warp's 128 positions is kept
+    const unsigned cnt = __popc(g4) | ((unsigned)__popc(q4) << 16);
+    unsigned incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
     }
-    gt_before += g;
-    eq_before += q;
+    const unsigned before = run + incl - cnt;
+    unsigned gt_before = before & 0xffffu, eq_before = before >> 16;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const bool g = (g4 >> c) & 1u, q = (q4 >> c) & 1u;
+      if (g || (q && eq_before < need_eq)) {
+        const unsigned pos = gt_before + min(eq_before, need_eq);
+        out.pos[pos] = my0 + j * 128 + c;
+        out.val[pos] = sv[4 * j + c];
+      }
+      gt_before += g;
+      eq_before += q;
+    }
+    run += __shfl_sync(0xffffffffu, incl, 31);
   }
   __syncthreads();
 }
 
-// Per (row, chunk of 8192 tokens): the chunk's topk best scores, as candidates for the row's selection.
-__global__ void __launch_bounds__(kAttendThreads)
-topk_select_kernel(const SelectParams p) {
-  __shared__ SelectOut sel;
-  __shared__ SelectScratch sc;
-  ptx::grid_launch_dependents();
-  const int tid = threadIdx.x;
-  const int rowid = blockIdx.x / p.n_chunks, chunk = blockIdx.x % p.n_chunks;
-  const int b = rowid / p.n_q;
-  ptx::grid_dependency_wait();
-  const int len = min(max(p.seqlens[b], 0), p.max_seqlen);
-  const int base = chunk * kChunk;
-  const int n = min(kChunk, len - base);
-  int* cnt = p.cand_cnt + (long long)rowid * p.n_chunks + chunk;
-  if (n <= 0) {
-    if (tid == 0) *cnt = 0;
-    return;
-  }
-  const float* row = p.scores + (long long)rowid * p.lpad + base;  // read straight into registers
-  const int k = min(p.topk, n);
-  block_select(row, n, k, sel, sc);
-  const long long out0 = ((long long)rowid * p.n_chunks + chunk) * p.topk;
-  for (int i = tid; i < k; i += kAttendThreads) {
-    p.cand_idx[out0 + i] = base + sel.pos[i];
-    p.cand_val[out0 + i] = sel.val[i];
-  }
-  if (tid == 0) *cnt = k;
-}
-
-// Per (sequence, query head): the topk best of the chunks' candidates, softmax over them, gather of their V rows.
-__global__ void __launch_bounds__(kAttendThreads)
+// Per (sequence, query head): the topk best scores of the row, softmax over them, gather of their V rows.  Rows longer
+// than one selection are taken in pieces whose winners are merged by one more selection.
+__global__ void __launch_bounds__(kAttendThreads, 1)
 topk_attend_kernel(const AttendParams p) {
-  extern __shared__ float attend_dyn[];  // vals[kChunk], tok[kChunk], acc[warps][d_v]
-  float* vals = attend_dyn;
-  int* tok = reinterpret_cast<int*>(attend_dyn + kChunk);
-  float* acc_dyn = attend_dyn + 2 * kChunk;
+  extern __shared__ __align__(16) float attend_dyn[];  // cand_key[kMaxCand], mval[kMaxCand], mtok[kMaxCand], acc
+  unsigned* cand_key = reinterpret_cast<unsigned*>(attend_dyn);
+  float* mval = attend_dyn + kMaxCand;
+  int* mtok = reinterpret_cast<int*>(attend_dyn + 2 * kMaxCand);
+  float* acc_dyn = attend_dyn + 3 * kMaxCand;
   __shared__ SelectOut sel;
   __shared__ SelectScratch sc;
-  __shared__ int chunk_off[65];
   int* sel_idx = sel.pos;
   float* sel_s = sel.val;
-  __shared__ float red[kAttendThreads / 32];
+  __shared__ float red[kAttendWarps];
 
-  ptx::grid_launch_dependents();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.x / p.n_q, h = blockIdx.x % p.n_q;
   const int hv = (int)(((long long)h * p.n_v) / p.n_q);  // Eq. (idx)
@@ -518,31 +545,27 @@ topk_attend_kernel(const AttendParams p) {
     if (p.lse && tid == 0) p.lse[(long long)b * p.n_q + h] = -INFINITY;
     return;
   }
-  // ---- the chunks' candidates, concatenated in token order
-  const long long rowid = blockIdx.x;
-  if (tid == 0) {
-    int run = 0;
-    for (int c = 0; c < p.n_chunks; ++c) {
-      chunk_off[c] = run;
-      run += p.cand_cnt[rowid * p.n_chunks + c];
+  const float* row = p.scores + (long long)blockIdx.x * p.lpad;
+  int k = min(p.topk, len);
+  if (len <= kPiece) {
+    block_select(row, len, k, sel, sc, cand_key);
+  } else {
+    int ncand = 0;
+    for (int base = 0; base < len; base += kPiece) {
+      const int n_p = min(kPiece, len - base), k_p = min(p.topk, n_p);
+      block_select(row + base, n_p, k_p, sel, sc, cand_key);
+      for (int i = tid; i < k_p; i += kAttendThreads) {
+        mval[ncand + i] = sel_s[i];
+        mtok[ncand + i] = base + sel_idx[i];
+      }
+      ncand += k_p;
+      __syncthreads();
     }
-    chunk_off[p.n_chunks] = run;
+    k = min(p.topk, ncand);
+    block_select(mval, ncand, k, sel, sc, cand_key);
+    for (int i = tid; i < k; i += kAttendThreads) sel_idx[i] = mtok[sel_idx[i]];
+    __syncthreads();
   }
-  __syncthreads();
-  const int n = chunk_off[p.n_chunks];
-  for (int c = 0; c < p.n_chunks; ++c) {
-    const int cnt = chunk_off[c + 1] - chunk_off[c];
-    const long long src = (rowid * p.n_chunks + c) * p.topk;
-    for (int i = tid; i < cnt; i += kAttendThreads) {
-      vals[chunk_off[c] + i] = p.cand_val[src + i];
-      tok[chunk_off[c] + i] = p.cand_idx[src + i];
-    }
-  }
-  __syncthreads();
-  const int k = min(p.topk, n);
-  block_select(vals, n, k, sel, sc);
-  for (int i = tid; i < k; i += kAttendThreads) sel_idx[i] = tok[sel_idx[i]];
-  __syncthreads();
 
   // ---- softmax over the kept scores (base-2 domain)
   float m = -INFINITY;
@@ -553,7 +576,7 @@ topk_attend_kernel(const AttendParams p) {
   __syncthreads();
   m = red[0];
 #pragma unroll
-  for (int ww = 1; ww < kAttendThreads / 32; ++ww) m = fmaxf(m, red[ww]);
+  for (int ww = 1; ww < kAttendWarps; ++ww) m = fmaxf(m, red[ww]);
   __syncthreads();
   float l = 0.f;
   for (int i = tid; i < k; i += kAttendThreads) {
@@ -567,31 +590,50 @@ topk_attend_kernel(const AttendParams p) {
   __syncthreads();
   l = 0.f;
 #pragma unroll
-  for (int ww = 0; ww < kAttendThreads / 32; ++ww) l += red[ww];
+  for (int ww = 0; ww < kAttendWarps; ++ww) l += red[ww];
 
-  // ---- gather the kept V rows: a warp per row, a lane per 4 channels (128 channels per sweep)
+  // ---- gather the kept V rows: a warp per row, a lane per 4 channels (128 channels per sweep), eight rows in flight
+  constexpr int kInFlight = 8;
   for (int ch0 = 0; ch0 < p.d_v; ch0 += 128) {
     const int ch = ch0 + lane * 4;
     const bool in = ch < p.d_v;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int i = warp; i < k; i += kAttendThreads / 32) {
-      const int j = sel_idx[i];
-      long long blk = b, slot = j;
-      if (p.page_table) {
-        blk = p.page_table[(long long)b * p.max_pages_per_seq + j / p.page_size];
-        slot = j % p.page_size;
-        if (blk < 0 || blk >= p.num_blocks) {
-          report(p.dev_status, DIFFQKV_ERR_INDEX);
-          continue;
+    for (int i0 = warp; i0 < k; i0 += kAttendWarps * kInFlight) {
+      const __nv_bfloat16* src[kInFlight];
+      float wgt[kInFlight];
+#pragma unroll
+      for (int f = 0; f < kInFlight; ++f) {
+        const int i = i0 + f * kAttendWarps;
+        src[f] = nullptr;
+        wgt[f] = 0.f;
+        if (i < k) {
+          const int j = sel_idx[i];
+          long long blk = b, slot = j;
+          bool ok = true;
+          if (p.page_table) {
+            blk = p.page_table[(long long)b * p.max_pages_per_seq + j / p.page_size];
+            slot = j % p.page_size;
+            if (blk < 0 || blk >= p.num_blocks) {
+              report(p.dev_status, DIFFQKV_ERR_INDEX);
+              ok = false;
+            }
+          }
+          if (ok) {
+            src[f] = p.v + blk * p.v_sb + (long long)hv * p.v_sh + slot * p.v_st + ch;
+            wgt[f] = sel_s[i];
+          }
         }
       }
-      if (in) {
-        const uint2 raw = *reinterpret_cast<const uint2*>(p.v + blk * p.v_sb + (long long)hv * p.v_sh + slot * p.v_st + ch);
-        const float wgt = sel_s[i];
-        a.x = fmaf(wgt, __uint_as_float(raw.x << 16), a.x);
-        a.y = fmaf(wgt, __uint_as_float(raw.x & 0xffff0000u), a.y);
-        a.z = fmaf(wgt, __uint_as_float(raw.y << 16), a.z);
-        a.w = fmaf(wgt, __uint_as_float(raw.y & 0xffff0000u), a.w);
+      uint2 raw[kInFlight];
+#pragma unroll
+      for (int f = 0; f < kInFlight; ++f)
+        raw[f] = (in && src[f]) ? *reinterpret_cast<const uint2*>(src[f]) : make_uint2(0u, 0u);
+#pragma unroll
+      for (int f = 0; f < kInFlight; ++f) {
+        a.x = fmaf(wgt[f], __uint_as_float(raw[f].x << 16), a.x);
+        a.y = fmaf(wgt[f], __uint_as_float(raw[f].x & 0xffff0000u), a.y);
+        a.z = fmaf(wgt[f], __uint_as_float(raw[f].y << 16), a.z);
+        a.w = fmaf(wgt[f], __uint_as_float(raw[f].y & 0xffff0000u), a.w);
       }
     }
     if (in) {
@@ -604,7 +646,7 @@ topk_attend_kernel(const AttendParams p) {
   for (int ch = tid; ch < p.d_v; ch += kAttendThreads) {
     float o = 0.f;
 #pragma unroll
-    for (int ww = 0; ww < kAttendThreads / 32; ++ww) o += acc_dyn[ww * p.d_v + ch];
+    for (int ww = 0; ww < kAttendWarps; ++ww) o += acc_dyn[ww * p.d_v + ch];
     o *= inv;
     if (p.out_is_f32) reinterpret_cast<float*>(p.out)[orow + ch] = o;
     else reinterpret_cast<__nv_bfloat16*>(p.out)[orow + ch] = __float2bfloat16_rn(o);
@@ -621,15 +663,14 @@ int sm_count_topk() {
 
 }  // namespace
 
-static int topk_chunks(int max_seqlen) { return ((max_seqlen > 0 ? max_seqlen : 1) + kChunk - 1) / kChunk; }
+static int topk_pieces(int max_seqlen) { return ((max_seqlen > 0 ? max_seqlen : 1) + kPiece - 1) / kPiece; }
 
 bool topk_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, int topk, int* box_tok) {
   if (s.dtype != DIFFQKV_BF16 || (s.d_qk != 64 && s.d_qk != 128)) return false;
   if (s.d_v % 4 != 0 || s.d_v > 512 || topk < 1 || topk > kMaxTopk) return false;
   if (s.batch < 1 || s.batch > kMaxBatchScores || s.n_q / s.n_k > 8 * kMaxGroups) return false;
   if (c.v_stride_tok % 4 != 0 || c.v_stride_head % 4 != 0 || c.v_stride_blk % 4 != 0) return false;
-  const int chunks = topk_chunks(c.max_seqlen);
-  if (chunks > 64 || (long long)chunks * topk > kChunk) return false;  // the row's candidates must fit one block
+  if ((long long)topk_pieces(c.max_seqlen) * topk > kMaxCand) return false;  // the pieces' winners are merged in one go
   int bt = kST;
   if (c.page_table) {
     if (c.page_size % 16 != 0) return false;
@@ -642,10 +683,9 @@ bool topk_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, int t
 
 static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
-size_t topk_decode_workspace_bytes(const diffqkv_shape& s, int max_seqlen, int topk) {
+size_t topk_decode_workspace_bytes(const diffqkv_shape& s, int max_seqlen, int /*topk*/) {
   const size_t lpad = ((size_t)(max_seqlen > 0 ? max_seqlen : 1) + kST - 1) / kST * kST;
-  const size_t rows = (size_t)s.batch * s.n_q, chunks = (size_t)topk_chunks(max_seqlen);
-  return up256(rows * lpad * sizeof(float)) + 2 * up256(rows * chunks * (size_t)topk * 4) + up256(rows * chunks * 4);
+  return up256((size_t)s.batch * s.n_q * lpad * sizeof(float));
 }
 
 cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, int topk, int box_tok,
@@ -711,25 +751,8 @@ cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diff
   count_launch();
 
   const size_t rows = (size_t)s.batch * s.n_q;
-  const int chunks = topk_chunks(c.max_seqlen);
-  char* ws = reinterpret_cast<char*>(workspace) + up256(rows * (size_t)sp.lpad * sizeof(float));
-  SelectParams sel;
-  sel.scores = sp.scores; sel.lpad = sp.lpad; sel.seqlens = c.seqlens; sel.max_seqlen = c.max_seqlen;
-  sel.n_q = s.n_q; sel.topk = topk; sel.n_chunks = chunks;
-  sel.cand_idx = reinterpret_cast<int*>(ws);
-  ws += up256(rows * chunks * (size_t)topk * 4);
-  sel.cand_val = reinterpret_cast<float*>(ws);
-  ws += up256(rows * chunks * (size_t)topk * 4);
-  sel.cand_cnt = reinterpret_cast<int*>(ws);
-  cfg.gridDim = dim3((unsigned)(rows * chunks));
-  cfg.blockDim = dim3(kAttendThreads);
-  cfg.dynamicSmemBytes = 0;
-  err = cudaLaunchKernelEx(&cfg, topk_select_kernel, sel);
-  if (err != cudaSuccess) return err;
-  count_launch();
-
   AttendParams ap;
-  ap.cand_idx = sel.cand_idx; ap.cand_val = sel.cand_val; ap.cand_cnt = sel.cand_cnt; ap.n_chunks = chunks;
+  ap.scores = sp.scores; ap.lpad = sp.lpad;
   ap.v = reinterpret_cast<const __nv_bfloat16*>(c.v_cache);
   ap.v_sb = c.v_stride_blk; ap.v_sh = c.v_stride_head; ap.v_st = c.v_stride_tok;
   ap.seqlens = c.seqlens; ap.page_table = c.page_table;
@@ -739,7 +762,8 @@ cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diff
   ap.out = out; ap.lse = lse; ap.out_is_f32 = s.out_dtype == DIFFQKV_F32;
   ap.dev_status = dev_status;
   cfg.gridDim = dim3((unsigned)rows);
-  cfg.dynamicSmemBytes = (size_t)(2 * kChunk + (kAttendThreads / 32) * s.d_v) * sizeof(float);
+  cfg.blockDim = dim3(kAttendThreads);
+  cfg.dynamicSmemBytes = (size_t)(3 * kMaxCand + kAttendWarps * s.d_v) * sizeof(float);
   err = cudaFuncSetAttribute(topk_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg.dynamicSmemBytes);
   if (err != cudaSuccess) return err;
   err = cudaLaunchKernelEx(&cfg, topk_attend_kernel, ap);
