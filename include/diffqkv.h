@@ -241,10 +241,11 @@ diffqkv_status diffqkv_cache_append(const void *k_new, const void *v_new, int32_
  * streamed once, of the V cache only topk rows per query head are read.  A sequence with at most topk tokens gives
  * exactly the full attention of diffqkv_decode.
  *   q, cache, out, lse, dev_status as in diffqkv_decode; bf16 only, d_qk 64 or 128, at most 32 query heads per
- *   K head, 1 <= topk <= 1024, pages of 16, 32, 64 or a multiple of 128 tokens
+ *   K head, 1 <= topk <= 1024, d_v a multiple of 8 with 16-byte aligned V rows, pages of 16, 32, 64 or a multiple
+ *   of 128 tokens; topk times the number of 32768-token pieces of max_seqlen may not exceed 8192
+ *   (DIFFQKV_ERR_UNSUPPORTED otherwise)
  *   workspace  diffqkv_decode_topk_workspace_bytes(shape, cache->max_seqlen, topk) bytes, 256-byte aligned: the fp32
- *              scores [batch, n_q, max_seqlen rounded up to 128] and the per-8192-token candidates; topk times
- *              the number of 8192-token chunks of max_seqlen may not exceed 8192
+ *              scores [batch, n_q, max_seqlen rounded up to 128]
  */
 size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape *shape, int32_t max_seqlen, int32_t topk);
 diffqkv_status diffqkv_decode_topk(const void *q, const diffqkv_cache *cache, const diffqkv_shape *shape, int32_t topk,
@@ -260,6 +261,13 @@ const char *diffqkv_status_string(diffqkv_status status);
  * cap is set.  Mainly for tests, which use it to move the places where sequences are cut.
  */
 void diffqkv_set_max_blocks(int32_t max_blocks);
+
+/*
+ * Test hook (process-wide host state): a non-zero value makes diffqkv_decode_topk always select over all scores of a
+ * row; 0 (the default) lets it first try the selection that reads only the 16-token blocks whose largest score can
+ * reach the top.  Both give the same result.
+ */
+void diffqkv_topk_general_only(int32_t on);
 
 /* Which split kernel the most recent decode call launched: 0 none yet, 1 generic, 2 TMA (for tests). */
 int32_t diffqkv_last_decode_kernel(void);

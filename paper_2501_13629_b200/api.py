@@ -29,7 +29,8 @@ EXPORTS = (
     "diffqkv_decode_num_splits", "diffqkv_decode_workspace_bytes", "diffqkv_decode", "gqa_decode",
     "diffqkv_combine", "diffqkv_prefill", "diffqkv_augq_workspace_bytes", "diffqkv_augq",
     "diffqkv_status_string", "diffqkv_launch_count", "diffqkv_profile_split_events", "diffqkv_decode_static",
-    "diffqkv_set_max_blocks", "diffqkv_last_decode_kernel", "diffqkv_augq_rope", "diffqkv_project",
+    "diffqkv_set_max_blocks", "diffqkv_topk_general_only", "diffqkv_last_decode_kernel", "diffqkv_augq_rope",
+    "diffqkv_project",
     "diffqkv_cache_append", "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes",
 )
 
@@ -94,6 +95,8 @@ _lib.diffqkv_decode_topk.argtypes = [C.c_void_p, C.POINTER(CacheStruct), C.POINT
 _lib.diffqkv_status_string.restype = C.c_char_p
 _lib.diffqkv_status_string.argtypes = [C.c_int]
 _lib.diffqkv_launch_count.restype = C.c_int64
+_lib.diffqkv_topk_general_only.restype = None
+_lib.diffqkv_topk_general_only.argtypes = [C.c_int32]
 _lib.diffqkv_set_max_blocks.restype = None
 _lib.diffqkv_set_max_blocks.argtypes = [C.c_int32]
 _lib.diffqkv_profile_split_events.restype = None
@@ -118,6 +121,11 @@ def set_split_events(before: Optional[torch.cuda.Event], after: Optional[torch.c
     """Benchmark hook: have decode calls record these events around their split kernel (None, None = off)."""
     _lib.diffqkv_profile_split_events(None if before is None else C.c_void_p(before.cuda_event),
                                       None if after is None else C.c_void_p(after.cuda_event))
+
+
+def topk_general_only(on: bool) -> None:
+    """Test hook: make diffqkv_decode_topk always select over all scores of a row; see diffqkv_topk_general_only."""
+    _lib.diffqkv_topk_general_only(int(bool(on)))
 
 
 def set_max_blocks(n: int) -> None:

@@ -94,6 +94,7 @@ cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, 
 // Selective V fetching (decode_topk.cu): K-only score pass, then top-k selection and V gather per query head.
 bool topk_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, int topk, int* box_tok);
 size_t topk_decode_workspace_bytes(const diffqkv_shape& s, int max_seqlen, int topk);
+void set_topk_general_only(int on);
 cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, int topk, int box_tok,
                                void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream);
 

@@ -23,8 +23,11 @@ namespace diffqkv {
 namespace {
 
 constexpr int kST = 128;            // tokens per K tile
-constexpr int kScoreWarps = 8;      // consumer warps, 16 tokens each
-constexpr int kScoreThreads = (kScoreWarps + 1) * 32;
+constexpr int kTileWarps = 8;       // warps that score one tile together, 16 tokens each
+// Teams of kTileWarps warps work on different tiles at the same time (team t takes every teams-th tile of the
+// block's range): one team alone spends most of a tile waiting on its own dependent instructions.
+__host__ __device__ constexpr int score_teams(int ng) { return ng <= 2 ? 2 : 1; }  // registers allow two up to 16 heads
+__host__ __device__ constexpr int score_threads(int ng) { return (score_teams(ng) * kTileWarps + 1) * 32; }
 constexpr int kMaxBatchScores = 2048;
 constexpr int kMaxTopk = 1024;
 constexpr int kMaxGroups = 4;       // query heads per K head <= 8 * kMaxGroups
@@ -41,6 +44,7 @@ struct ScoreParams {
   long long lpad;            // row length of the score matrix
   float scale_log2;
   float* scores;             // [batch, n_q, lpad]
+  float* bmax;               // [batch, n_q, lpad / 16] largest score of every 16 tokens
   int* dev_status;
 };
 
@@ -76,8 +80,8 @@ struct TileWalker {
   }
 };
 
-template <int D_QK>
-__global__ void __launch_bounds__(kScoreThreads, 1)
+template <int D_QK, int NG>  // NG: groups of 8 query heads per K head
+__global__ void __launch_bounds__(score_threads(NG), 1)
 decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScoreParams p) {
   constexpr int HK = D_QK / 64;            // 64-channel halves per row
   constexpr int K_TILE = kST * D_QK * 2;   // bytes of one K tile
@@ -95,7 +99,7 @@ decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScorePara
     *abort_flag = 0;
     for (int s = 0; s < p.stages; ++s) {
       ptx::mbar_init(full0 + 8 * s, 1);
-      ptx::mbar_init(empty0 + 8 * s, kScoreWarps);
+      ptx::mbar_init(empty0 + 8 * s, kTileWarps);
     }
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmap_k);
@@ -130,7 +134,8 @@ decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScorePara
   TileWalker w;
   w.seek(g_begin, prefix, p.batch, p.n_k);
 
-  if (warp == kScoreWarps) {
+  constexpr int kTeams = score_teams(NG);
+  if (warp == kTeams * kTileWarps) {
     // ------------------------------------------------------------------ producer warp: lane x owns token part x
     const int parts = kST / p.box_tok;
     const uint32_t my_off = lane * (p.box_tok * 128 * HK);
@@ -178,27 +183,32 @@ decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScorePara
   const int g8 = lane >> 2, t4 = lane & 3;
   const int bt_shift = 31 - __clz(p.box_tok), bt_mask = p.box_tok - 1;
   auto row_index = [&](int r, int h) { return (((r >> bt_shift) * HK + h) << bt_shift) + (r & bt_mask); };
-  int stage = 0;
-  uint32_t phase = 0;
+  const int team = warp / kTileWarps, tw = warp % kTileWarps;
   int cur_b = -1, cur_u = -1, len = 0;
   float* srow = nullptr;  // score row of the first query head of the current K head
-  uint32_t qf[kMaxGroups][KS][2];
-  const int row0 = warp * 16;
+  float* brow = nullptr;  // its row of 16-token maxima
+  const long long nbpad = p.lpad / 16;
+  uint32_t qf[NG][KS][2];
+  const int row0 = tw * 16;
   const int r = row0 + (lane & 7) + 8 * ((lane >> 3) & 1);
   const int csel = lane >> 4;
   uint32_t a_off[KS];  // byte offset of this lane's ldmatrix row in a stage, per 16-channel step
 #pragma unroll
   for (int ks = 0; ks < KS; ++ks)
     a_off[ks] = row_index(r, ks / 4) * 128 + ((((ks % 4) * 2 + csel) ^ (r & 7)) << 4);
-  for (; w.g < g_end; w.advance(prefix, p.batch, p.n_k)) {
+  for (int a = 0; a < team && w.g < g_end; ++a) w.advance(prefix, p.batch, p.n_k);
+  for (int it = team; w.g < g_end; it += kTeams) {  // `it` counts the block's tiles: tile `it` sits in stage it % stages
+    const int stage = it % p.stages;
+    const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
     if (w.b != cur_b || w.u != cur_u) {  // Q^T fragments of the query heads of this K head, 8 heads per group
       cur_b = w.b; cur_u = w.u;
       len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
       srow = p.scores + ((long long)w.b * p.n_q + (long long)w.u * p.g_k) * p.lpad;
+      brow = p.bmax + ((long long)w.b * p.n_q + (long long)w.u * p.g_k) * nbpad;
 #pragma unroll
-      for (int gq = 0; gq < kMaxGroups; ++gq) {
+      for (int gq = 0; gq < NG; ++gq) {
         const int hq = gq * 8 + g8;
-        const bool use = gq < p.groups && hq < p.g_k;
+        const bool use = hq < p.g_k;
         const __nv_bfloat16* qrow = p.q + ((long long)w.b * p.n_q + (long long)w.u * p.g_k + (use ? hq : 0)) * D_QK;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
@@ -214,9 +224,9 @@ decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScorePara
     const int n_valid = min(kST, len - w.t * kST);
     if (row0 < n_valid) {
       const uint32_t st_u32 = ptx::smem_u32(smem + (size_t)stage * K_TILE);
-      float s[kMaxGroups][2][4];  // two accumulation chains per group (even and odd 16-channel steps)
+      float s[NG][2][4];  // two accumulation chains per group (even and odd 16-channel steps)
 #pragma unroll
-      for (int gq = 0; gq < kMaxGroups; ++gq)
+      for (int gq = 0; gq < NG; ++gq)
 #pragma unroll
         for (int e = 0; e < 4; ++e) s[gq][0][e] = s[gq][1][e] = 0.f;
 #pragma unroll
@@ -224,27 +234,32 @@ decode_scores_kernel(const __grid_constant__ CUtensorMap tmap_k, const ScorePara
         uint32_t a[4];
         ptx::ldmatrix_x4(st_u32 + a_off[ks], a);
 #pragma unroll
-        for (int gq = 0; gq < kMaxGroups; ++gq)
-          if (gq < p.groups) ptx::mma_bf16_16816(s[gq][ks & 1], a, qf[gq][ks][0], qf[gq][ks][1]);
+        for (int gq = 0; gq < NG; ++gq) ptx::mma_bf16_16816(s[gq][ks & 1], a, qf[gq][ks][0], qf[gq][ks][1]);
       }
       // thread holds token rows g8, g8 + 8 of the block and head columns 2 t4, 2 t4 + 1 of each group
       const long long tok = (long long)w.t * kST + row0 + g8;
 #pragma unroll
-      for (int gq = 0; gq < kMaxGroups; ++gq) {
-        if (gq >= p.groups) continue;
+      for (int gq = 0; gq < NG; ++gq) {
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           const int hq = gq * 8 + 2 * t4 + c;
+          const float lo = (s[gq][0][c] + s[gq][1][c]) * p.scale_log2;
+          const float hi = (s[gq][0][2 + c] + s[gq][1][2 + c]) * p.scale_log2;
+          float bm = fmaxf(row0 + g8 < n_valid ? lo : -INFINITY, row0 + g8 + 8 < n_valid ? hi : -INFINITY);
+          bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));  // over the 16 tokens of the block
+          bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
+          bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
           if (hq >= p.g_k) continue;
           float* dst = srow + (long long)hq * p.lpad + tok;
-          if (row0 + g8 < n_valid) dst[0] = (s[gq][0][c] + s[gq][1][c]) * p.scale_log2;
-          if (row0 + g8 + 8 < n_valid) dst[8] = (s[gq][0][2 + c] + s[gq][1][2 + c]) * p.scale_log2;
+          if (row0 + g8 < n_valid) dst[0] = lo;
+          if (row0 + g8 + 8 < n_valid) dst[8] = hi;
+          if (g8 == 0) brow[(long long)hq * nbpad + w.t * (kST / 16) + tw] = bm;
         }
       }
     }
     __syncwarp();
     if (lane == 0) ptx::mbar_arrive(empty0 + 8 * stage);
-    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+    for (int a = 0; a < kTeams && w.g < g_end; ++a) w.advance(prefix, p.batch, p.n_k);
   }
 }
 
@@ -255,9 +270,13 @@ constexpr int kWarpSpan = 32 * kPerThread;
 constexpr int kMaxCand = 8192;           // keys the fast path of the selection holds; also the merge capacity
 constexpr int kAttendWarps = kAttendThreads / 32;
 
+constexpr int kMaxFlag = 4096;           // 16-token blocks the fast selection expands
+
 struct AttendParams {
   const float* scores;
+  const float* bmax;
   long long lpad;
+  int general_only;  // test hook: skip the selection driven by the block maxima
   const __nv_bfloat16* v;
   long long v_sb, v_sh, v_st;
   const int* seqlens;
@@ -282,19 +301,20 @@ struct SelectOut {
 };
 
 struct SelectScratch {
-  unsigned hist[256];
+  unsigned hist[4][256];  // one histogram per radix pass
   unsigned warp_tot[2][kAttendWarps];
-  float warp_max[kAttendWarps];
+  float warp_max[kAttendWarps], warp_min[kAttendWarps];
   unsigned prefix, need, count;
 };
 
-// From the top bin down: the bin of sc.hist that holds the need-th largest of the keys counted there.  Warp 0 calls
-// it; the winning lane publishes the extended prefix and the rank that remains inside the bin.
-__device__ __forceinline__ void pick_bin(SelectScratch& sc, unsigned prefix, unsigned need, int pass) {
+// From the top bin down: the bin of hist that holds the need-th largest of the keys counted there.  Warp 0 calls it;
+// the winning lane publishes the prefix extended by the bin (at bit `shift`) and the rank that remains inside the bin.
+__device__ __forceinline__ void pick_bin(const unsigned* hist, SelectScratch& sc, unsigned prefix, unsigned need,
+                                         int shift) {
   const int lane = threadIdx.x & 31;
   unsigned mine = 0;  // lane owns bins 255 - 8 lane .. 248 - 8 lane
 #pragma unroll
-  for (int e = 0; e < 8; ++e) mine += sc.hist[255 - (lane * 8 + e)];
+  for (int e = 0; e < 8; ++e) mine += hist[255 - (lane * 8 + e)];
   unsigned incl = mine;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -306,36 +326,45 @@ __device__ __forceinline__ void pick_bin(SelectScratch& sc, unsigned prefix, uns
     unsigned cum = before;
     for (int e = 0; e < 8; ++e) {
       const int bin = 255 - (lane * 8 + e);
-      if (need <= cum + sc.hist[bin]) {
-        sc.prefix = prefix | ((unsigned)bin << (8 * pass));
+      if (need <= cum + hist[bin]) {
+        sc.prefix = prefix | ((unsigned)bin << shift);
         sc.need = need - cum;
         break;
       }
-      cum += sc.hist[bin];
+      cum += hist[bin];
     }
   }
 }
 
-// The k-th largest of n keys by radix select, 8 bits a pass: its key in *thr, and in *need_eq how many keys equal to
-// it belong to the k largest.  count_pass(mask, prefix, pass) adds every key with (key & mask) == prefix to
-// sc.hist[(key >> 8 pass) & 255].  All threads of the block call it.
+// The k-th largest of a set of keys below 2^bits by radix select, up to 8 bits a pass from the top bit down: its key
+// in *thr, and in *need_eq how many keys equal to it belong to the k largest.  count_pass(hist, top, shift, prefix)
+// adds every key that agrees with prefix above bit `top` to hist[(key >> shift) & 255] (top - shift <= 8).  All
+// threads of the block call it.  After max_passes passes it stops: *thr is then a lower bound (low bits zero).
 template <typename CountPass>
-__device__ void radix_kth(CountPass count_pass, int k, SelectScratch& sc, unsigned* thr, unsigned* need_eq) {
+__device__ void radix_kth(CountPass count_pass, int bits, int k, SelectScratch& sc, unsigned* thr, unsigned* need_eq,
+                          int max_passes = 4) {
   const int tid = threadIdx.x;
-  unsigned prefix = 0, mask = 0, need = (unsigned)k;
-  for (int pass = 3; pass >= 0; --pass) {
-    for (int i = tid; i < 256; i += kAttendThreads) sc.hist[i] = 0;
+  for (int i = tid; i < 4 * 256; i += kAttendThreads) (&sc.hist[0][0])[i] = 0;
+  __syncthreads();
+  unsigned prefix = 0, need = (unsigned)k;
+  int pass = 0;
+  for (int top = bits; top > 0 && pass < max_passes; ++pass) {
+    const int shift = max(top - 8, 0);
+    count_pass(sc.hist[pass], top, shift, prefix);
     __syncthreads();
-    count_pass(mask, prefix, pass);
-    __syncthreads();
-    if (tid < 32) pick_bin(sc, prefix, need, pass);
+    if (tid < 32) pick_bin(sc.hist[pass], sc, prefix, need, shift);
     __syncthreads();
     prefix = sc.prefix;
     need = sc.need;
-    mask |= 0xffu << (8 * pass);
+    top = shift;
   }
   *thr = prefix;
   *need_eq = need;
+}
+
+// Do key and prefix agree in the bits from `top` up?
+__device__ __forceinline__ bool same_above(unsigned key, unsigned prefix, int top) {
+  return top >= 32 || (key >> top) == (prefix >> top);
 }
 
 // The k largest of vals[0 .. n) (shared or global memory, 16-byte aligned, n <= kPiece); of equal values the earlier
@@ -345,26 +374,32 @@ __device__ void radix_kth(CountPass count_pass, int k, SelectScratch& sc, unsign
 // so each load instruction of a warp reads 512 consecutive bytes.  The k-th largest value is first sought among the
 // few values within a distance `band` of the maximum (every value outside is smaller than every value inside, so the
 // rank is unchanged); the band doubles until it holds k values and is bisected back if it then holds more than the
-// candidate buffer.  Only when no band fits (values crowded on one point, or not finite) does the radix select run
-// over all values.
+// candidate buffer.  The candidates' keys are stored relative to the key of the band's lower end, which leaves few
+// significant bits for the radix select.  Only when no band fits (values crowded on one point, or not finite) does
+// the radix select run over all values.  A 64-bit mask per thread marks its candidates, so that the later steps touch
+// only the 4-value groups that hold one.
 __device__ __noinline__ void block_select(const float* vals, int n, int k, SelectOut& out, SelectScratch& sc,
                                           unsigned* cand_key) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int my0 = warp * kWarpSpan + lane * 4;  // position of quad j, element c: my0 + 128 j + c
   float sv[kPerThread];
+  unsigned cm[2] = {0u, 0u};  // candidates: bit e of the pair; starts as "position below n"
 #pragma unroll
   for (int j = 0; j < kQuads; ++j) {
     const int i = my0 + j * 128;
     float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     if (i + 3 < n) {
       v = *reinterpret_cast<const float4*>(vals + i);
-    } else {
-      if (i < n) v.x = vals[i];
+      cm[j >> 3] |= 15u << (4 * (j & 7));
+    } else if (i < n) {
+      v.x = vals[i];
       if (i + 1 < n) v.y = vals[i + 1];
       if (i + 2 < n) v.z = vals[i + 2];
+      cm[j >> 3] |= ((1u << (n - i)) - 1u) << (4 * (j & 7));
     }
     sv[4 * j] = v.x; sv[4 * j + 1] = v.y; sv[4 * j + 2] = v.z; sv[4 * j + 3] = v.w;
   }
+  auto quad = [](const unsigned (&mk)[2], int j) { return (mk[j >> 3] >> (4 * (j & 7))) & 15u; };
   unsigned thr = 0, need_eq = 0;
   const bool all = n <= k;
   if (!all) {
@@ -379,12 +414,13 @@ __device__ __noinline__ void block_select(const float* vals, int n, int k, Selec
 #pragma unroll
     for (int ww = 1; ww < kAttendWarps; ++ww) m = fmaxf(m, sc.warp_max[ww]);
 
-    int round = 0, mine = 0;
+    int round = 0;
+    unsigned ge[2] = {0u, 0u};
     auto count_ge = [&](float cut) {  // values >= cut in the block (cut finite: the padding never counts)
-      int c = 0;
+      ge[0] = ge[1] = 0u;
 #pragma unroll
-      for (int e = 0; e < kPerThread; ++e) c += sv[e] >= cut;
-      mine = c;
+      for (int e = 0; e < kPerThread; ++e) ge[e >> 5] |= (unsigned)(sv[e] >= cut) << (e & 31);
+      int c = __popc(ge[0]) + __popc(ge[1]);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
       unsigned* tot = sc.warp_tot[round & 1];  // alternate buffers: one barrier a round is enough
@@ -398,7 +434,6 @@ __device__ __noinline__ void block_select(const float* vals, int n, int k, Selec
     };
     float cut = m, lo = 0.f, hi = 0.f;
     int count = 0;
-    bool fits = false;
     if (m > -INFINITY && m < INFINITY) {
       for (hi = 1.f; hi < 1e30f; hi *= 2.f) {
         cut = m - hi;
@@ -412,10 +447,11 @@ __device__ __noinline__ void block_select(const float* vals, int n, int k, Selec
         count = count_ge(cut);
         if (count < k) { lo = mid; count = kMaxCand + 1; } else hi = mid;
       }
-      fits = count >= k && count <= kMaxCand;
     }
-    if (fits) {
+    if (count >= k && count <= kMaxCand) {
+      cm[0] = ge[0]; cm[1] = ge[1];
       // every thread appends its own candidates (any order will do for the rank)
+      const int mine = __popc(cm[0]) + __popc(cm[1]);
       int incl = mine;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -427,57 +463,57 @@ __device__ __noinline__ void block_select(const float* vals, int n, int k, Selec
       unsigned base = 0;
       if (lane == 31 && incl) base = atomicAdd(&sc.count, (unsigned)incl);
       base = __shfl_sync(0xffffffffu, base, 31) + (unsigned)(incl - mine);
+      const unsigned key_cut = order_key(cut);
 #pragma unroll
-      for (int e = 0; e < kPerThread; ++e)
-        if (sv[e] >= cut) cand_key[base++] = order_key(sv[e]);
+      for (int j = 0; j < kQuads; ++j) {
+        const unsigned c4 = quad(cm, j);
+        if (c4 == 0) continue;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if ((c4 >> c) & 1u) cand_key[base++] = order_key(sv[4 * j + c]) - key_cut;
+      }
       __syncthreads();
       const int ncand = count;
+      const unsigned span = order_key(m) - key_cut;
       radix_kth(
-          [&](unsigned mask, unsigned prefix, int pass) {
-            for (int i0 = 0; i0 < ncand; i0 += kAttendThreads) {
-              const int i = i0 + tid;
-              unsigned bin = 0xffffffffu;  // no contribution
-              if (i < ncand) {
-                const unsigned key = cand_key[i];
-                if ((key & mask) == prefix) bin = (key >> (8 * pass)) & 255u;
-              }
-              // keys crowd into a few bins in the upper passes: lanes of a warp that hit the same bin add once
-              const unsigned peers = __match_any_sync(0xffffffffu, bin);
-              if (bin != 0xffffffffu && lane == __ffs(peers) - 1) atomicAdd(&sc.hist[bin], (unsigned)__popc(peers));
+          [&](unsigned* hist, int top, int shift, unsigned prefix) {
+            for (int i = tid; i < ncand; i += kAttendThreads) {
+              const unsigned key = cand_key[i];
+              if (same_above(key, prefix, top)) atomicAdd(&hist[(key >> shift) & 255u], 1u);
             }
           },
-          k, sc, &thr, &need_eq);
+          span ? 32 - __clz(span) : 0, k, sc, &thr, &need_eq);
+      thr += key_cut;
     } else {
       radix_kth(
-          [&](unsigned mask, unsigned prefix, int pass) {
+          [&](unsigned* hist, int top, int shift, unsigned prefix) {
 #pragma unroll
             for (int e = 0; e < kPerThread; ++e) {
               const unsigned key = order_key(sv[e]);
-              if (my0 + (e >> 2) * 128 + (e & 3) < n && (key & mask) == prefix)
-                atomicAdd(&sc.hist[(key >> (8 * pass)) & 255u], 1u);
+              if (((cm[e >> 5] >> (e & 31)) & 1u) && same_above(key, prefix, top))
+                atomicAdd(&hist[(key >> shift) & 255u], 1u);
             }
           },
-          k, sc, &thr, &need_eq);
+          32, k, sc, &thr, &need_eq);
     }
   }
   // compaction in position order: kept = key > thr, or key == thr among the first need_eq such positions
-  auto flags = [&](int j, unsigned& g4, unsigned& q4) {
-    g4 = 0; q4 = 0;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const unsigned key = order_key(sv[4 * j + c]);
-      const bool valid = my0 + j * 128 + c < n;
-      if (valid && (all || key > thr)) g4 |= 1u << c;
-      else if (valid && key == thr) q4 |= 1u << c;
-    }
-  };
-  unsigned packed = 0;  // kept-for-sure count in the low half, equal-to-threshold count in the high half
+  unsigned gm[2] = {0u, 0u}, qm[2] = {0u, 0u};
 #pragma unroll
   for (int j = 0; j < kQuads; ++j) {
-    unsigned g4, q4;
-    flags(j, g4, q4);
-    packed += __popc(g4) | ((unsigned)__popc(q4) << 16);
+    const unsigned c4 = quad(cm, j);
+    if (c4 == 0) continue;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      if (!((c4 >> c) & 1u)) continue;
+      const unsigned key = order_key(sv[4 * j + c]);
+      const unsigned bit = 1u << (4 * (j & 7) + c);
+      if (all || key > thr) gm[j >> 3] |= bit;
+      else if (key == thr) qm[j >> 3] |= bit;
+    }
   }
+  // kept-for-sure count in the low half, equal-to-threshold count in the high half
+  unsigned packed = (__popc(gm[0]) + __popc(gm[1])) | ((unsigned)(__popc(qm[0]) + __popc(qm[1])) << 16);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) packed += __shfl_xor_sync(0xffffffffu, packed, o);
   unsigned* tot = sc.warp_tot[0];
@@ -488,8 +524,7 @@ __device__ __noinline__ void block_select(const float* vals, int n, int k, Selec
   for (int ww = 0; ww < warp; ++ww) run += tot[ww];
 #pragma unroll
   for (int j = 0; j < kQuads; ++j) {
-    unsigned g4, q4;
-    flags(j, g4, q4);
+    const unsigned g4 = quad(gm, j), q4 = quad(qm, j);
     if (__ballot_sync(0xffffffffu, (g4 | q4) != 0) == 0) continue;  // nothing of this warp's 128 positions is kept
     const unsigned cnt = __popc(g4) | ((unsigned)__popc(q4) << 16);
     unsigned incl = cnt;
@@ -500,31 +535,228 @@ __device__ __noinline__ void block_select(const float* vals, int n, int k, Selec
     }
     const unsigned before = run + incl - cnt;
     unsigned gt_before = before & 0xffffu, eq_before = before >> 16;
+    if (g4 | q4) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const bool g = (g4 >> c) & 1u, q = (q4 >> c) & 1u;
-      if (g || (q && eq_before < need_eq)) {
-        const unsigned pos = gt_before + min(eq_before, need_eq);
-        out.pos[pos] = my0 + j * 128 + c;
-        out.val[pos] = sv[4 * j + c];
+      for (int c = 0; c < 4; ++c) {
+        const bool g = (g4 >> c) & 1u, q = (q4 >> c) & 1u;
+        if (g || (q && eq_before < need_eq)) {
+          const unsigned pos = gt_before + min(eq_before, need_eq);
+          out.pos[pos] = my0 + j * 128 + c;
+          out.val[pos] = sv[4 * j + c];
+        }
+        gt_before += g;
+        eq_before += q;
       }
-      gt_before += g;
-      eq_before += q;
     }
     run += __shfl_sync(0xffffffffu, incl, 31);
   }
   __syncthreads();
 }
 
+// Exclusive prefix of v over the threads of the block, in thread order, and the block's total.
+__device__ __forceinline__ unsigned block_scan(unsigned v, unsigned* total, SelectScratch& sc) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  unsigned incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  __syncthreads();  // earlier readers of the totals are done
+  if (lane == 31) sc.warp_tot[0][warp] = incl;
+  __syncthreads();
+  unsigned before = incl - v, t = 0;
+#pragma unroll
+  for (int ww = 0; ww < kAttendWarps; ++ww) {
+    const unsigned x = sc.warp_tot[0][ww];
+    if (ww < warp) before += x;
+    t += x;
+  }
+  *total = t;
+  return before;
+}
+
+// The same result as block_select over a whole row of `len` scores, found from the maxima of its 16-token blocks
+// (bm): the k-th largest block maximum is a lower bound of the k-th largest score (k blocks hold k scores at least
+// that large), so only blocks whose maximum reaches it can hold a kept score.  Those few blocks are read again, their
+// scores at or above the bound become the candidates (in token order), the exact k-th largest is found among them
+// and the kept ones are compacted in token order.  The bound is taken from two radix passes only, i.e. rounded down
+// to 16 significant bits of the maxima's range.  Returns false, the same for all threads, when the values do not
+// suit it (not finite, or so crowded that the blocks or candidates overflow their buffers); nothing is written then.
+__device__ __noinline__ bool block_select_sparse(const float* row, const float* bm, int len, int k, SelectOut& out,
+                                                 SelectScratch& sc, unsigned* cand_key, float* cval, int* cpos,
+                                                 int* flag_id, int* foff) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nblk = (len + 15) >> 4;
+  float mx = -INFINITY, mn = INFINITY;
+  for (int i = tid; i < nblk; i += kAttendThreads) {
+    const float v = bm[i];
+    mx = fmaxf(mx, v);
+    mn = fminf(mn, v);
+    if (!(v == v)) mn = -INFINITY;  // not a number: give up below
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+  }
+  __syncthreads();
+  if (lane == 0) { sc.warp_max[warp] = mx; sc.warp_min[warp] = mn; }
+  __syncthreads();
+#pragma unroll
+  for (int ww = 0; ww < kAttendWarps; ++ww) {
+    mx = fmaxf(mx, sc.warp_max[ww]);
+    mn = fminf(mn, sc.warp_min[ww]);
+  }
+  if (!(mx < INFINITY && mn > -INFINITY)) return false;
+  const unsigned key_min = order_key(mn);
+  const unsigned span = order_key(mx) - key_min;
+  unsigned pre = 0, dummy = 0;
+  radix_kth(
+      [&](unsigned* hist, int top, int shift, unsigned prefix) {
+        for (int i = tid; i < nblk; i += kAttendThreads) {
+          const unsigned key = order_key(bm[i]) - key_min;
+          if (same_above(key, prefix, top)) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+      },
+      span ? 32 - __clz(span) : 0, k, sc, &pre, &dummy, 2);
+  const unsigned cut_key = key_min + pre;  // at most the k-th largest block maximum
+
+  // ---- the blocks that can hold a kept score, in order
+  const int per = (nblk + kAttendThreads - 1) / kAttendThreads;
+  const int b_lo = min(nblk, tid * per), b_hi = min(nblk, b_lo + per);
+  unsigned cnt = 0;
+  for (int i = b_lo; i < b_hi; ++i) cnt += order_key(bm[i]) >= cut_key;
+  unsigned nflag = 0;
+  unsigned at = block_scan(cnt, &nflag, sc);
+  if (nflag > (unsigned)kMaxFlag) return false;
+  for (int i = b_lo; i < b_hi; ++i)
+    if (order_key(bm[i]) >= cut_key) flag_id[at++] = i;
+  __syncthreads();
+
+  // ---- their scores at or above the bound, in token order: four lanes per block (16 bytes each), kBatch blocks
+  // per lane group in flight, i.e. one trip to memory per kRound blocks; the scores wait in registers while the
+  // round's counts are turned into offsets
+  constexpr int kBatch = 8;
+  constexpr int kStep = 8 * kAttendWarps;  // blocks the thread block takes per step
+  constexpr int kRound = kStep * kBatch;
+  static_assert(kRound == 2 * kAttendThreads, "the offsets of a round are scanned two per thread");
+  const int quarter = lane & 3, slot = lane >> 2;
+  unsigned ncand = 0;
+  for (int base = 0; base < (int)nflag; base += kRound) {
+    const int nr = min(kRound, (int)nflag - base);
+    float4 v[kBatch];
+    unsigned c4[kBatch], excl[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {  // this lane's 4 scores of block fr of the round
+      const int fr = u * kStep + warp * 8 + slot;
+      v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      c4[u] = 0;
+      if (fr < nr) {
+        const int pos = flag_id[base + fr] * 16 + quarter * 4;
+        if (pos + 3 < len) {
+          v[u] = *reinterpret_cast<const float4*>(row + pos);
+        } else {
+          if (pos < len) v[u].x = row[pos];
+          if (pos + 1 < len) v[u].y = row[pos + 1];
+          if (pos + 2 < len) v[u].z = row[pos + 2];
+        }
+        c4[u] = (unsigned)(pos < len && order_key(v[u].x) >= cut_key) |
+                ((unsigned)(pos + 1 < len && order_key(v[u].y) >= cut_key) << 1) |
+                ((unsigned)(pos + 2 < len && order_key(v[u].z) >= cut_key) << 2) |
+                ((unsigned)(pos + 3 < len && order_key(v[u].w) >= cut_key) << 3);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {  // counts: scan over the 4 lanes of a block
+      const int fr = u * kStep + warp * 8 + slot;
+      const unsigned n4 = __popc(c4[u]);
+      unsigned t = n4;
+      unsigned y = __shfl_up_sync(0xffffffffu, t, 1);
+      if (quarter >= 1) t += y;
+      y = __shfl_up_sync(0xffffffffu, t, 2);
+      if (quarter >= 2) t += y;
+      excl[u] = t - n4;
+      if (quarter == 3 && fr < nr) foff[fr] = (int)t;
+    }
+    __syncthreads();
+    const int i0 = tid * 2;
+    const unsigned c0 = i0 < nr ? (unsigned)foff[i0] : 0u, c1 = i0 + 1 < nr ? (unsigned)foff[i0 + 1] : 0u;
+    unsigned tot = 0;
+    const unsigned at0 = ncand + block_scan(c0 + c1, &tot, sc);
+    if (ncand + tot > (unsigned)kMaxCand) return false;
+    if (i0 < nr) foff[i0] = (int)at0;
+    if (i0 + 1 < nr) foff[i0 + 1] = (int)(at0 + c0);
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      if (c4[u] == 0) continue;
+      const int fr = u * kStep + warp * 8 + slot;
+      int idx = foff[fr] + (int)excl[u];
+      const int pos = flag_id[base + fr] * 16 + quarter * 4;
+      const float vv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        if ((c4[u] >> c) & 1u) {
+          cand_key[idx] = order_key(vv[c]) - cut_key;
+          cval[idx] = vv[c];
+          cpos[idx] = pos + c;
+          ++idx;
+        }
+    }
+    ncand += tot;
+    __syncthreads();
+  }
+  // ---- the exact k-th largest among the candidates
+  unsigned thr = 0, need_eq = 0;
+  const unsigned span2 = order_key(mx) - cut_key;
+  radix_kth(
+      [&](unsigned* hist, int top, int shift, unsigned prefix) {
+        for (int i = tid; i < (int)ncand; i += kAttendThreads) {
+          const unsigned key = cand_key[i];
+          if (same_above(key, prefix, top)) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+      },
+      span2 ? 32 - __clz(span2) : 0, k, sc, &thr, &need_eq);
+
+  // ---- compaction in token order: kept = key > thr, or key == thr among the first need_eq such candidates
+  const int per3 = ((int)ncand + kAttendThreads - 1) / kAttendThreads;
+  const int c_lo = min((int)ncand, tid * per3), c_hi = min((int)ncand, c_lo + per3);
+  unsigned packed = 0;
+  for (int i = c_lo; i < c_hi; ++i) {
+    const unsigned key = cand_key[i];
+    packed += key > thr ? 1u : (key == thr ? 1u << 16 : 0u);
+  }
+  unsigned tot_unused = 0;
+  const unsigned before = block_scan(packed, &tot_unused, sc);
+  unsigned gt_before = before & 0xffffu, eq_before = before >> 16;
+  for (int i = c_lo; i < c_hi; ++i) {
+    const unsigned key = cand_key[i];
+    const bool g = key > thr, q = key == thr;
+    if (g || (q && eq_before < need_eq)) {
+      const unsigned pos = gt_before + min(eq_before, need_eq);
+      out.pos[pos] = cpos[i];
+      out.val[pos] = cval[i];
+    }
+    gt_before += g;
+    eq_before += q;
+  }
+  __syncthreads();
+  return true;
+}
+
 // Per (sequence, query head): the topk best scores of the row, softmax over them, gather of their V rows.  Rows longer
 // than one selection are taken in pieces whose winners are merged by one more selection.
 __global__ void __launch_bounds__(kAttendThreads, 1)
 topk_attend_kernel(const AttendParams p) {
-  extern __shared__ __align__(16) float attend_dyn[];  // cand_key[kMaxCand], mval[kMaxCand], mtok[kMaxCand], acc
+  // cand_key[kMaxCand], mval[kMaxCand], mtok[kMaxCand], flag_id[kMaxFlag], foff[kMaxFlag], acc[warps][d_v]
+  extern __shared__ __align__(16) float attend_dyn[];
   unsigned* cand_key = reinterpret_cast<unsigned*>(attend_dyn);
   float* mval = attend_dyn + kMaxCand;
   int* mtok = reinterpret_cast<int*>(attend_dyn + 2 * kMaxCand);
-  float* acc_dyn = attend_dyn + 3 * kMaxCand;
+  int* flag_id = reinterpret_cast<int*>(attend_dyn + 3 * kMaxCand);
+  int* foff = flag_id + kMaxFlag;
+  float* acc_dyn = attend_dyn + 3 * kMaxCand + 2 * kMaxFlag;
   __shared__ SelectOut sel;
   __shared__ SelectScratch sc;
   int* sel_idx = sel.pos;
@@ -547,7 +779,13 @@ topk_attend_kernel(const AttendParams p) {
   }
   const float* row = p.scores + (long long)blockIdx.x * p.lpad;
   int k = min(p.topk, len);
-  if (len <= kPiece) {
+  // worth trying when the bound from the block maxima cuts deep: at least two blocks per kept score
+  const bool sparse = !p.general_only && 32LL * k <= len &&
+                      block_select_sparse(row, p.bmax + (long long)blockIdx.x * (p.lpad / 16), len, k, sel, sc,
+                                          cand_key, mval, mtok, flag_id, foff);
+  if (sparse) {
+    // sel holds the kept tokens
+  } else if (len <= kPiece) {
     block_select(row, len, k, sel, sc, cand_key);
   } else {
     int ncand = 0;
@@ -592,53 +830,64 @@ topk_attend_kernel(const AttendParams p) {
 #pragma unroll
   for (int ww = 0; ww < kAttendWarps; ++ww) l += red[ww];
 
-  // ---- gather the kept V rows: a warp per row, a lane per 4 channels (128 channels per sweep), eight rows in flight
+  // ---- where the kept V rows start (element offsets; -1: page out of range), one table look-up per row, all at once
+  long long* row_off = reinterpret_cast<long long*>(cand_key);  // the candidate keys are dead by now
+  for (int i = tid; i < k; i += kAttendThreads) {
+    const int j = sel_idx[i];
+    long long blk = b, slot = j;
+    if (p.page_table) {
+      blk = p.page_table[(long long)b * p.max_pages_per_seq + j / p.page_size];
+      slot = j % p.page_size;
+    }
+    long long off = blk * p.v_sb + (long long)hv * p.v_sh + slot * p.v_st;
+    if (blk < 0 || blk >= p.num_blocks) {
+      report(p.dev_status, DIFFQKV_ERR_INDEX);
+      off = -1;
+    }
+    row_off[i] = off;
+  }
+  __syncthreads();
+  // ---- gather: half a warp per row, a lane per 8 channels (128 channels per sweep), eight rows in flight per lane
   constexpr int kInFlight = 8;
+  const int half = lane >> 4, hl = lane & 15;
   for (int ch0 = 0; ch0 < p.d_v; ch0 += 128) {
-    const int ch = ch0 + lane * 4;
+    const int ch = ch0 + hl * 8;
     const bool in = ch < p.d_v;
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int i0 = warp; i0 < k; i0 += kAttendWarps * kInFlight) {
-      const __nv_bfloat16* src[kInFlight];
+    float a[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) a[e] = 0.f;
+    for (int i0 = warp * 2 + half; i0 < k; i0 += 2 * kAttendWarps * kInFlight) {
+      uint4 raw[kInFlight];
       float wgt[kInFlight];
 #pragma unroll
       for (int f = 0; f < kInFlight; ++f) {
-        const int i = i0 + f * kAttendWarps;
-        src[f] = nullptr;
+        const int i = i0 + f * 2 * kAttendWarps;
+        raw[f] = make_uint4(0u, 0u, 0u, 0u);
         wgt[f] = 0.f;
-        if (i < k) {
-          const int j = sel_idx[i];
-          long long blk = b, slot = j;
-          bool ok = true;
-          if (p.page_table) {
-            blk = p.page_table[(long long)b * p.max_pages_per_seq + j / p.page_size];
-            slot = j % p.page_size;
-            if (blk < 0 || blk >= p.num_blocks) {
-              report(p.dev_status, DIFFQKV_ERR_INDEX);
-              ok = false;
-            }
-          }
-          if (ok) {
-            src[f] = p.v + blk * p.v_sb + (long long)hv * p.v_sh + slot * p.v_st + ch;
+        if (i < k && in) {
+          const long long off = row_off[i];
+          if (off >= 0) {
+            raw[f] = *reinterpret_cast<const uint4*>(p.v + off + ch);
             wgt[f] = sel_s[i];
           }
         }
       }
-      uint2 raw[kInFlight];
-#pragma unroll
-      for (int f = 0; f < kInFlight; ++f)
-        raw[f] = (in && src[f]) ? *reinterpret_cast<const uint2*>(src[f]) : make_uint2(0u, 0u);
 #pragma unroll
       for (int f = 0; f < kInFlight; ++f) {
-        a.x = fmaf(wgt[f], __uint_as_float(raw[f].x << 16), a.x);
-        a.y = fmaf(wgt[f], __uint_as_float(raw[f].x & 0xffff0000u), a.y);
-        a.z = fmaf(wgt[f], __uint_as_float(raw[f].y << 16), a.z);
-        a.w = fmaf(wgt[f], __uint_as_float(raw[f].y & 0xffff0000u), a.w);
+        const uint32_t wd[4] = {raw[f].x, raw[f].y, raw[f].z, raw[f].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          a[2 * e] = fmaf(wgt[f], __uint_as_float(wd[e] << 16), a[2 * e]);
+          a[2 * e + 1] = fmaf(wgt[f], __uint_as_float(wd[e] & 0xffff0000u), a[2 * e + 1]);
+        }
       }
     }
-    if (in) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) a[e] += __shfl_xor_sync(0xffffffffu, a[e], 16);
+    if (in && half == 0) {
       float* dst = acc_dyn + warp * p.d_v + ch;
-      dst[0] = a.x; dst[1] = a.y; dst[2] = a.z; dst[3] = a.w;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) dst[e] = a[e];
     }
   }
   __syncthreads();
@@ -667,9 +916,10 @@ static int topk_pieces(int max_seqlen) { return ((max_seqlen > 0 ? max_seqlen : 
 
 bool topk_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, int topk, int* box_tok) {
   if (s.dtype != DIFFQKV_BF16 || (s.d_qk != 64 && s.d_qk != 128)) return false;
-  if (s.d_v % 4 != 0 || s.d_v > 512 || topk < 1 || topk > kMaxTopk) return false;
+  if (s.d_v % 8 != 0 || s.d_v > 512 || topk < 1 || topk > kMaxTopk) return false;
   if (s.batch < 1 || s.batch > kMaxBatchScores || s.n_q / s.n_k > 8 * kMaxGroups) return false;
-  if (c.v_stride_tok % 4 != 0 || c.v_stride_head % 4 != 0 || c.v_stride_blk % 4 != 0) return false;
+  if (c.v_stride_tok % 8 != 0 || c.v_stride_head % 8 != 0 || c.v_stride_blk % 8 != 0) return false;  // 16-byte loads
+  if ((reinterpret_cast<uintptr_t>(c.v_cache) & 15u) != 0) return false;
   if ((long long)topk_pieces(c.max_seqlen) * topk > kMaxCand) return false;  // the pieces' winners are merged in one go
   int bt = kST;
   if (c.page_table) {
@@ -685,8 +935,12 @@ static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
 size_t topk_decode_workspace_bytes(const diffqkv_shape& s, int max_seqlen, int /*topk*/) {
   const size_t lpad = ((size_t)(max_seqlen > 0 ? max_seqlen : 1) + kST - 1) / kST * kST;
-  return up256((size_t)s.batch * s.n_q * lpad * sizeof(float));
+  const size_t rows = (size_t)s.batch * s.n_q;
+  return up256(rows * lpad * sizeof(float)) + up256(rows * (lpad / 16) * sizeof(float));
 }
+
+static int g_topk_general_only = 0;  // test hook
+void set_topk_general_only(int on) { g_topk_general_only = on != 0; }
 
 cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, int topk, int box_tok,
                                void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream) {
@@ -712,10 +966,13 @@ cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diff
   sp.num_blocks = c.num_blocks; sp.max_seqlen = c.max_seqlen;
   sp.batch = s.batch; sp.n_q = s.n_q; sp.n_k = s.n_k; sp.g_k = s.n_q / s.n_k;
   sp.groups = (sp.g_k + 7) / 8;
+  const int ng = sp.groups;
   sp.box_tok = box_tok;
   sp.lpad = ((long long)(c.max_seqlen > 0 ? c.max_seqlen : 1) + kST - 1) / kST * kST;
   sp.scale_log2 = s.scale * kLog2e;
   sp.scores = reinterpret_cast<float*>(workspace);
+  sp.bmax = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) +
+                                     up256((size_t)s.batch * s.n_q * (size_t)sp.lpad * sizeof(float)));
   sp.dev_status = dev_status;
   const int k_tile = kST * s.d_qk * 2;
   const int fixed = 1024 + 2 * 16 * 8 + (s.batch + 1) * 4 + 64;
@@ -737,22 +994,31 @@ cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diff
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kScoreThreads);
+  cfg.blockDim = dim3((unsigned)score_threads(ng));
   cfg.dynamicSmemBytes = (size_t)smem;
-  cudaError_t err;
+  cudaError_t err = cudaErrorNotSupported;
+  auto launch = [&](auto kernel) {
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (err == cudaSuccess) err = cudaLaunchKernelEx(&cfg, kernel, mk, sp);
+  };
   if (s.d_qk == 128) {
-    err = cudaFuncSetAttribute(decode_scores_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (err == cudaSuccess) err = cudaLaunchKernelEx(&cfg, decode_scores_kernel<128>, mk, sp);
+    if (ng == 1) launch(decode_scores_kernel<128, 1>);
+    else if (ng == 2) launch(decode_scores_kernel<128, 2>);
+    else if (ng == 3) launch(decode_scores_kernel<128, 3>);
+    else if (ng == 4) launch(decode_scores_kernel<128, 4>);
   } else {
-    err = cudaFuncSetAttribute(decode_scores_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (err == cudaSuccess) err = cudaLaunchKernelEx(&cfg, decode_scores_kernel<64>, mk, sp);
+    if (ng == 1) launch(decode_scores_kernel<64, 1>);
+    else if (ng == 2) launch(decode_scores_kernel<64, 2>);
+    else if (ng == 3) launch(decode_scores_kernel<64, 3>);
+    else if (ng == 4) launch(decode_scores_kernel<64, 4>);
   }
   if (err != cudaSuccess) return err;
   count_launch();
 
   const size_t rows = (size_t)s.batch * s.n_q;
   AttendParams ap;
-  ap.scores = sp.scores; ap.lpad = sp.lpad;
+  ap.scores = sp.scores; ap.bmax = sp.bmax; ap.lpad = sp.lpad;
+  ap.general_only = g_topk_general_only;
   ap.v = reinterpret_cast<const __nv_bfloat16*>(c.v_cache);
   ap.v_sb = c.v_stride_blk; ap.v_sh = c.v_stride_head; ap.v_st = c.v_stride_tok;
   ap.seqlens = c.seqlens; ap.page_table = c.page_table;
@@ -763,7 +1029,7 @@ cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diff
   ap.dev_status = dev_status;
   cfg.gridDim = dim3((unsigned)rows);
   cfg.blockDim = dim3(kAttendThreads);
-  cfg.dynamicSmemBytes = (size_t)(3 * kMaxCand + kAttendWarps * s.d_v) * sizeof(float);
+  cfg.dynamicSmemBytes = (size_t)(3 * kMaxCand + 2 * kMaxFlag + kAttendWarps * s.d_v) * sizeof(float);
   err = cudaFuncSetAttribute(topk_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg.dynamicSmemBytes);
   if (err != cudaSuccess) return err;
   err = cudaLaunchKernelEx(&cfg, topk_attend_kernel, ap);

@@ -113,11 +113,64 @@ def test_topk_ties_take_the_earlier_tokens(api):
         assert np.abs(out[0, h] - v[0, h // 4, :10].mean(axis=0)).max() <= 1e-5
 
 
-def test_topk_config3_full_size(api, oracle):
+@pytest.fixture
+def general_only(api):
+    """Switches diffqkv_decode_topk to the selection over all scores and back."""
+    yield api.topk_general_only
+    api.topk_general_only(False)
+
+
+def test_topk_partial_ties_at_the_cut(api, oracle, general_only):
+    """All keys equal except a few: the kept set is the few that score higher plus the earliest of the equal ones,
+    so the cut falls inside a run of exactly equal scores.  Checked in both selection paths."""
+    cfg = dataclasses.replace(SMALL, batch=1, n_q=8, n_k=2, n_v=4, kv_len=2000, seed=94)
+    inp = W.make_decode_inputs(cfg)
+    special = np.array([3, 517, 1024, 1999, 1500])
+    keep = inp.k[:, :, special].copy()
+    inp.k[:] = inp.k[:, :, 7:8]
+    inp.k[:, :, special] = keep
+    ref, lse_ref, sel, _ = oracle.decode_topk(inp.q, oracle_cache(oracle, inp), cfg.n_q, cfg.n_k, cfg.n_v, cfg.d_qk,
+                                              cfg.d_v, cfg.scale, 20)
+    for h in range(cfg.n_q):  # the definition's choice: the tokens that beat the common score, then the earliest
+        kept = np.sort(sel[0, h])
+        common = np.setdiff1d(kept, special)
+        assert np.array_equal(common, np.setdiff1d(np.arange(2000), special)[:len(common)])
+    for on in (False, True):
+        general_only(on)
+        out, lse = run_topk(api, inp, 20)
+        check_bf16(out, ref, f"partial ties, general_only={on}")
+        check_lse(lse, lse_ref, 2e-2)
+
+
+@pytest.mark.parametrize("lens,topk", [((3000, 129, 64), 50), ((2500, 2048, 33), 7)])
+def test_topk_selection_paths_agree_bitwise(api, general_only, lens, topk):
+    """The selection driven by the block maxima and the one over all scores keep the same tokens in the same order."""
+    inp = W.make_decode_inputs(SMALL, seqlens=np.array(lens, np.int32))
+    out, lse = run_topk(api, inp, topk)
+    general_only(True)
+    out_g, lse_g = run_topk(api, inp, topk)
+    assert np.array_equal(out, out_g) and np.array_equal(lse, lse_g)
+
+
+def test_topk_rows_longer_than_one_selection_pass(api, oracle, general_only):
+    """70000 tokens: the selection over all scores takes the row in 32768-token pieces and merges their winners."""
+    cfg = dataclasses.replace(SMALL, batch=2, n_q=8, n_k=1, n_v=2, kv_len=70000, seed=95)
+    inp = W.make_decode_inputs(cfg, seqlens=np.array([70000, 32769], np.int32))
+    out, lse = run_topk(api, inp, 100)
+    check_against_oracle(oracle, inp, 100, out, lse, "70000 tokens")
+    general_only(True)
+    out_g, lse_g = run_topk(api, inp, 100)
+    assert np.array_equal(out, out_g) and np.array_equal(lse, lse_g)
+
+
+def test_topk_config3_full_size(api, oracle, general_only):
     """The long-context configuration (batch 4, 32/4/8 heads, d 128, 32768 tokens) with the paper's 100 scores."""
     inp = W.make_decode_inputs(W.CFG3)
     out, lse = run_topk(api, inp, 100)
     check_against_oracle(oracle, inp, 100, out, lse, "cfg3 top-100")
+    general_only(True)
+    out_g, lse_g = run_topk(api, inp, 100)
+    assert np.array_equal(out, out_g) and np.array_equal(lse, lse_g)
 
 
 def test_topk_argument_errors(api):
