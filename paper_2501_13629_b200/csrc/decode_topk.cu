@@ -763,6 +763,9 @@ topk_attend_kernel(const AttendParams p) {
   float* sel_s = sel.val;
   __shared__ float red[kAttendWarps];
 
+  // whatever follows in the stream may take the SMs this grid leaves free; it waits for this grid's end before it
+  // touches memory
+  ptx::grid_launch_dependents();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.x / p.n_q, h = blockIdx.x % p.n_q;
   const int hv = (int)(((long long)h * p.n_v) / p.n_q);  // Eq. (idx)
