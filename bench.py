@@ -426,6 +426,12 @@ def run_ours(args):
 
     cfg = W.CFG3
     host = W.make_decode_inputs(cfg)
+    if args.workload == "topk":  # selective V fetching on the headline workload alone (the command profilers wrap)
+        if rank == 0:
+            print(json.dumps({"workload": cfg.name + " top-100 / top-1024",
+                              "top100": time_topk(api, W, device, host, max(1, min(args.steps, 300)), 100),
+                              "top1024": time_topk(api, W, device, host, max(1, min(args.steps, 300)), 1024)}))
+        return
     case = DecodeCase(api, cfg, device, host_inputs=host)
     launches0 = api.launch_count()
     with ClockSampler(local_rank) as clocks:
@@ -593,8 +599,9 @@ def main():
     ap.add_argument("--quick", action="store_true", help="headline workload only")
     ap.add_argument("--budget-s", type=float, default=150.0,
                     help="--impl reference: seconds of oracle time the whole run may take (sizes the per-step sample)")
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill"],
-                    help="decode = the headline line (default); prefill = only the config 4 timings")
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "topk"],
+                    help="decode = the headline line (default); prefill = only the config 4 timings; "
+                         "topk = only selective V fetching on the headline workload")
     ap.add_argument("--profile", action="store_true",
                     help="only the timed loop of the headline workload (the command profilers wrap)")
     args = ap.parse_args()
