@@ -270,7 +270,7 @@ constexpr int kWarpSpan = 32 * kPerThread;
 constexpr int kMaxCand = 8192;           // keys the fast path of the selection holds; also the merge capacity
 constexpr int kAttendWarps = kAttendThreads / 32;
 
-constexpr int kMaxFlag = 4096;           // 16-token blocks the fast selection expands
+constexpr int kMaxFlag = 1536;           // 16-token blocks the sparse selection copies to shared memory
 
 struct AttendParams {
   const float* scores;
@@ -554,7 +554,7 @@ __device__ __noinline__ void block_select(const float* vals, int n, int k, Selec
 }
 
 // Exclusive prefix of v over the threads of the block, in thread order, and the block's total.
-__device__ __forceinline__ unsigned block_scan(unsigned v, unsigned* total, SelectScratch& sc) {
+__device__ __noinline__ unsigned block_scan(unsigned v, unsigned* total, SelectScratch& sc) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   unsigned incl = v;
 #pragma unroll
@@ -566,7 +566,7 @@ __device__ __forceinline__ unsigned block_scan(unsigned v, unsigned* total, Sele
   if (lane == 31) sc.warp_tot[0][warp] = incl;
   __syncthreads();
   unsigned before = incl - v, t = 0;
-#pragma unroll
+#pragma unroll 1
   for (int ww = 0; ww < kAttendWarps; ++ww) {
     const unsigned x = sc.warp_tot[0][ww];
     if (ww < warp) before += x;
@@ -576,21 +576,45 @@ __device__ __forceinline__ unsigned block_scan(unsigned v, unsigned* total, Sele
   return before;
 }
 
+// radix_kth over keys[i] - rebase, i < n, keys in shared memory.  One copy of the code serves both selections of the
+// sparse path: the kernel runs once per block, so what it costs is mostly the instructions it has to fetch.
+__device__ __noinline__ void radix_kth_shared(const unsigned* keys, int n, unsigned rebase, int bits, int k,
+                                              int max_passes, SelectScratch& sc, unsigned* thr, unsigned* need_eq) {
+  const int tid = threadIdx.x;
+  radix_kth(
+      [&](unsigned* hist, int top, int shift, unsigned prefix) {
+#pragma unroll 1
+        for (int i = tid; i < n; i += kAttendThreads) {
+          const unsigned key = keys[i] - rebase;
+          if (same_above(key, prefix, top)) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+      },
+      bits, k, sc, thr, need_eq, max_passes);
+}
+
+constexpr int kSparseCand = 4096;  // candidates the sparse selection holds
+
 // The same result as block_select over a whole row of `len` scores, found from the maxima of its 16-token blocks
 // (bm): the k-th largest block maximum is a lower bound of the k-th largest score (k blocks hold k scores at least
-// that large), so only blocks whose maximum reaches it can hold a kept score.  Those few blocks are read again, their
-// scores at or above the bound become the candidates (in token order), the exact k-th largest is found among them
-// and the kept ones are compacted in token order.  The bound is taken from two radix passes only, i.e. rounded down
-// to 16 significant bits of the maxima's range.  Returns false, the same for all threads, when the values do not
-// suit it (not finite, or so crowded that the blocks or candidates overflow their buffers); nothing is written then.
+// that large), so only blocks whose maximum reaches it can hold a kept score.  Those few blocks are copied to shared
+// memory, their scores at or above the bound become the candidates (in token order), the exact k-th largest is found
+// among them and the kept ones are compacted in token order.  The bound is taken from two radix passes only, i.e.
+// rounded down to 16 significant bits of the maxima's range.  Returns false, the same for all threads, when the
+// values do not suit it (not finite, or so crowded that the blocks or candidates overflow their buffers); nothing is
+// written to `out` then.  The loops are kept rolled and the helpers shared on purpose (see radix_kth_shared).
+//   keys      kMaxCand words: the block maxima's keys, later the candidates' keys (first half) and values (second)
+//   cpos      kSparseCand candidates' tokens;  flag_id, foff: kMaxFlag words each;  stage: kMaxFlag * 16 scores
 __device__ __noinline__ bool block_select_sparse(const float* row, const float* bm, int len, int k, SelectOut& out,
-                                                 SelectScratch& sc, unsigned* cand_key, float* cval, int* cpos,
-                                                 int* flag_id, int* foff) {
+                                                 SelectScratch& sc, unsigned* keys, int* cpos, int* flag_id,
+                                                 int* foff, float4* stage) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nblk = (len + 15) >> 4;
+  if (nblk > kMaxCand) return false;
   float mx = -INFINITY, mn = INFINITY;
+#pragma unroll 1
   for (int i = tid; i < nblk; i += kAttendThreads) {
     const float v = bm[i];
+    keys[i] = order_key(v);
     mx = fmaxf(mx, v);
     mn = fminf(mn, v);
     if (!(v == v)) mn = -INFINITY;  // not a number: give up below
@@ -603,126 +627,111 @@ __device__ __noinline__ bool block_select_sparse(const float* row, const float* 
   __syncthreads();
   if (lane == 0) { sc.warp_max[warp] = mx; sc.warp_min[warp] = mn; }
   __syncthreads();
-#pragma unroll
+#pragma unroll 1
   for (int ww = 0; ww < kAttendWarps; ++ww) {
     mx = fmaxf(mx, sc.warp_max[ww]);
     mn = fminf(mn, sc.warp_min[ww]);
   }
   if (!(mx < INFINITY && mn > -INFINITY)) return false;
-  const unsigned key_min = order_key(mn);
-  const unsigned span = order_key(mx) - key_min;
+  const unsigned key_min = order_key(mn), key_max = order_key(mx);
   unsigned pre = 0, dummy = 0;
-  radix_kth(
-      [&](unsigned* hist, int top, int shift, unsigned prefix) {
-        for (int i = tid; i < nblk; i += kAttendThreads) {
-          const unsigned key = order_key(bm[i]) - key_min;
-          if (same_above(key, prefix, top)) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-        }
-      },
-      span ? 32 - __clz(span) : 0, k, sc, &pre, &dummy, 2);
+  radix_kth_shared(keys, nblk, key_min, key_max != key_min ? 32 - __clz(key_max - key_min) : 0, k, 2, sc, &pre, &dummy);
   const unsigned cut_key = key_min + pre;  // at most the k-th largest block maximum
 
   // ---- the blocks that can hold a kept score, in order
   const int per = (nblk + kAttendThreads - 1) / kAttendThreads;
   const int b_lo = min(nblk, tid * per), b_hi = min(nblk, b_lo + per);
   unsigned cnt = 0;
-  for (int i = b_lo; i < b_hi; ++i) cnt += order_key(bm[i]) >= cut_key;
+#pragma unroll 1
+  for (int i = b_lo; i < b_hi; ++i) cnt += keys[i] >= cut_key;
   unsigned nflag = 0;
   unsigned at = block_scan(cnt, &nflag, sc);
   if (nflag > (unsigned)kMaxFlag) return false;
+#pragma unroll 1
   for (int i = b_lo; i < b_hi; ++i)
-    if (order_key(bm[i]) >= cut_key) flag_id[at++] = i;
+    if (keys[i] >= cut_key) flag_id[at++] = i;
   __syncthreads();
 
-  // ---- their scores at or above the bound, in token order: four lanes per block (16 bytes each), kBatch blocks
-  // per lane group in flight, i.e. one trip to memory per kRound blocks; the scores wait in registers while the
-  // round's counts are turned into offsets
-  constexpr int kBatch = 8;
-  constexpr int kStep = 8 * kAttendWarps;  // blocks the thread block takes per step
-  constexpr int kRound = kStep * kBatch;
-  static_assert(kRound == 2 * kAttendThreads, "the offsets of a round are scanned two per thread");
-  const int quarter = lane & 3, slot = lane >> 2;
+  // ---- copy them to shared memory, 16 bytes per thread and step (one trip to memory for all of them; positions past
+  // the row's end become -inf); block f's quad q goes to stage[4 f + (q ^ (f & 3))], which spreads the banks
+#pragma unroll 4
+  for (int i = tid; i < 4 * (int)nflag; i += kAttendThreads) {
+    const int f = i >> 2, q = i & 3;
+    const int pos = flag_id[f] * 16 + q * 4;
+    float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    if (pos + 3 < len) {
+      v = *reinterpret_cast<const float4*>(row + pos);
+    } else {
+      if (pos < len) v.x = row[pos];
+      if (pos + 1 < len) v.y = row[pos + 1];
+      if (pos + 2 < len) v.z = row[pos + 2];
+    }
+    stage[4 * f + (q ^ (f & 3))] = v;
+  }
+  __syncthreads();
+  // ---- candidates = staged scores at or above the bound: a thread per block counts, the counts become offsets, the
+  // thread copies its block's candidates in token order
+#pragma unroll 1
+  for (int f = tid; f < (int)nflag; f += kAttendThreads) {
+    int c = 0;
+#pragma unroll 1
+    for (int q = 0; q < 4; ++q) {
+      const float4 v = stage[4 * f + (q ^ (f & 3))];
+      c += (order_key(v.x) >= cut_key) + (order_key(v.y) >= cut_key) + (order_key(v.z) >= cut_key) +
+           (order_key(v.w) >= cut_key);
+    }
+    foff[f] = c;
+  }
+  __syncthreads();
+  const int per2 = ((int)nflag + kAttendThreads - 1) / kAttendThreads;
+  const int f_lo = min((int)nflag, tid * per2), f_hi = min((int)nflag, f_lo + per2);
+  cnt = 0;
+#pragma unroll 1
+  for (int i = f_lo; i < f_hi; ++i) cnt += (unsigned)foff[i];
   unsigned ncand = 0;
-  for (int base = 0; base < (int)nflag; base += kRound) {
-    const int nr = min(kRound, (int)nflag - base);
-    float4 v[kBatch];
-    unsigned c4[kBatch], excl[kBatch];
+  at = block_scan(cnt, &ncand, sc);
+  if (ncand > (unsigned)kSparseCand) return false;
+#pragma unroll 1
+  for (int i = f_lo; i < f_hi; ++i) {
+    const unsigned c = (unsigned)foff[i];
+    foff[i] = (int)at;
+    at += c;
+  }
+  __syncthreads();  // also: the block maxima's keys are dead, the candidates take their place
+  unsigned* cand_key = keys;
+  float* cval = reinterpret_cast<float*>(keys + kSparseCand);
+#pragma unroll 1
+  for (int f = tid; f < (int)nflag; f += kAttendThreads) {
+    int idx = foff[f];
+    const int pos0 = flag_id[f] * 16;
+#pragma unroll 1
+    for (int q = 0; q < 4; ++q) {
+      const float4 v = stage[4 * f + (q ^ (f & 3))];
+      const float vv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-    for (int u = 0; u < kBatch; ++u) {  // this lane's 4 scores of block fr of the round
-      const int fr = u * kStep + warp * 8 + slot;
-      v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      c4[u] = 0;
-      if (fr < nr) {
-        const int pos = flag_id[base + fr] * 16 + quarter * 4;
-        if (pos + 3 < len) {
-          v[u] = *reinterpret_cast<const float4*>(row + pos);
-        } else {
-          if (pos < len) v[u].x = row[pos];
-          if (pos + 1 < len) v[u].y = row[pos + 1];
-          if (pos + 2 < len) v[u].z = row[pos + 2];
-        }
-        c4[u] = (unsigned)(pos < len && order_key(v[u].x) >= cut_key) |
-                ((unsigned)(pos + 1 < len && order_key(v[u].y) >= cut_key) << 1) |
-                ((unsigned)(pos + 2 < len && order_key(v[u].z) >= cut_key) << 2) |
-                ((unsigned)(pos + 3 < len && order_key(v[u].w) >= cut_key) << 3);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < kBatch; ++u) {  // counts: scan over the 4 lanes of a block
-      const int fr = u * kStep + warp * 8 + slot;
-      const unsigned n4 = __popc(c4[u]);
-      unsigned t = n4;
-      unsigned y = __shfl_up_sync(0xffffffffu, t, 1);
-      if (quarter >= 1) t += y;
-      y = __shfl_up_sync(0xffffffffu, t, 2);
-      if (quarter >= 2) t += y;
-      excl[u] = t - n4;
-      if (quarter == 3 && fr < nr) foff[fr] = (int)t;
-    }
-    __syncthreads();
-    const int i0 = tid * 2;
-    const unsigned c0 = i0 < nr ? (unsigned)foff[i0] : 0u, c1 = i0 + 1 < nr ? (unsigned)foff[i0 + 1] : 0u;
-    unsigned tot = 0;
-    const unsigned at0 = ncand + block_scan(c0 + c1, &tot, sc);
-    if (ncand + tot > (unsigned)kMaxCand) return false;
-    if (i0 < nr) foff[i0] = (int)at0;
-    if (i0 + 1 < nr) foff[i0 + 1] = (int)(at0 + c0);
-    __syncthreads();
-#pragma unroll
-    for (int u = 0; u < kBatch; ++u) {
-      if (c4[u] == 0) continue;
-      const int fr = u * kStep + warp * 8 + slot;
-      int idx = foff[fr] + (int)excl[u];
-      const int pos = flag_id[base + fr] * 16 + quarter * 4;
-      const float vv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-      for (int c = 0; c < 4; ++c)
-        if ((c4[u] >> c) & 1u) {
-          cand_key[idx] = order_key(vv[c]) - cut_key;
+      for (int c = 0; c < 4; ++c) {
+        const unsigned key = order_key(vv[c]);
+        if (key >= cut_key) {
+          cand_key[idx] = key - cut_key;
           cval[idx] = vv[c];
-          cpos[idx] = pos + c;
+          cpos[idx] = pos0 + q * 4 + c;
           ++idx;
         }
+      }
     }
-    ncand += tot;
-    __syncthreads();
   }
+  __syncthreads();
+
   // ---- the exact k-th largest among the candidates
   unsigned thr = 0, need_eq = 0;
-  const unsigned span2 = order_key(mx) - cut_key;
-  radix_kth(
-      [&](unsigned* hist, int top, int shift, unsigned prefix) {
-        for (int i = tid; i < (int)ncand; i += kAttendThreads) {
-          const unsigned key = cand_key[i];
-          if (same_above(key, prefix, top)) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-        }
-      },
-      span2 ? 32 - __clz(span2) : 0, k, sc, &thr, &need_eq);
+  radix_kth_shared(cand_key, (int)ncand, 0u, key_max != cut_key ? 32 - __clz(key_max - cut_key) : 0, k, 4, sc, &thr,
+                   &need_eq);
 
   // ---- compaction in token order: kept = key > thr, or key == thr among the first need_eq such candidates
   const int per3 = ((int)ncand + kAttendThreads - 1) / kAttendThreads;
   const int c_lo = min((int)ncand, tid * per3), c_hi = min((int)ncand, c_lo + per3);
   unsigned packed = 0;
+#pragma unroll 1
   for (int i = c_lo; i < c_hi; ++i) {
     const unsigned key = cand_key[i];
     packed += key > thr ? 1u : (key == thr ? 1u << 16 : 0u);
@@ -730,6 +739,7 @@ __device__ __noinline__ bool block_select_sparse(const float* row, const float* 
   unsigned tot_unused = 0;
   const unsigned before = block_scan(packed, &tot_unused, sc);
   unsigned gt_before = before & 0xffffu, eq_before = before >> 16;
+#pragma unroll 1
   for (int i = c_lo; i < c_hi; ++i) {
     const unsigned key = cand_key[i];
     const bool g = key > thr, q = key == thr;
@@ -749,14 +759,18 @@ __device__ __noinline__ bool block_select_sparse(const float* row, const float* 
 // than one selection are taken in pieces whose winners are merged by one more selection.
 __global__ void __launch_bounds__(kAttendThreads, 1)
 topk_attend_kernel(const AttendParams p) {
-  // cand_key[kMaxCand], mval[kMaxCand], mtok[kMaxCand], flag_id[kMaxFlag], foff[kMaxFlag], acc[warps][d_v]
+  // stage[kMaxFlag][16] (the all-scores selection keeps mval[kMaxCand], mtok[kMaxCand] there), cand_key[kMaxCand],
+  // cpos[kSparseCand], flag_id[kMaxFlag], foff[kMaxFlag], acc[warps][d_v]
   extern __shared__ __align__(16) float attend_dyn[];
-  unsigned* cand_key = reinterpret_cast<unsigned*>(attend_dyn);
-  float* mval = attend_dyn + kMaxCand;
-  int* mtok = reinterpret_cast<int*>(attend_dyn + 2 * kMaxCand);
-  int* flag_id = reinterpret_cast<int*>(attend_dyn + 3 * kMaxCand);
+  static_assert(kMaxFlag * 16 >= 2 * kMaxCand, "the merge arrays share the staging area");
+  float4* stage = reinterpret_cast<float4*>(attend_dyn);
+  float* mval = attend_dyn;
+  int* mtok = reinterpret_cast<int*>(attend_dyn + kMaxCand);
+  unsigned* cand_key = reinterpret_cast<unsigned*>(attend_dyn + kMaxFlag * 16);
+  int* cpos = reinterpret_cast<int*>(attend_dyn + kMaxFlag * 16 + kMaxCand);
+  int* flag_id = cpos + kSparseCand;
   int* foff = flag_id + kMaxFlag;
-  float* acc_dyn = attend_dyn + 3 * kMaxCand + 2 * kMaxFlag;
+  float* acc_dyn = reinterpret_cast<float*>(foff + kMaxFlag);
   __shared__ SelectOut sel;
   __shared__ SelectScratch sc;
   int* sel_idx = sel.pos;
@@ -785,7 +799,7 @@ topk_attend_kernel(const AttendParams p) {
   // worth trying when the bound from the block maxima cuts deep: at least two blocks per kept score
   const bool sparse = !p.general_only && 32LL * k <= len &&
                       block_select_sparse(row, p.bmax + (long long)blockIdx.x * (p.lpad / 16), len, k, sel, sc,
-                                          cand_key, mval, mtok, flag_id, foff);
+                                          cand_key, cpos, flag_id, foff, stage);
   if (sparse) {
     // sel holds the kept tokens
   } else if (len <= kPiece) {
@@ -1032,7 +1046,8 @@ cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diff
   ap.dev_status = dev_status;
   cfg.gridDim = dim3((unsigned)rows);
   cfg.blockDim = dim3(kAttendThreads);
-  cfg.dynamicSmemBytes = (size_t)(3 * kMaxCand + 2 * kMaxFlag + kAttendWarps * s.d_v) * sizeof(float);
+  cfg.dynamicSmemBytes =
+      (size_t)(kMaxFlag * 16 + kMaxCand + kSparseCand + 2 * kMaxFlag + kAttendWarps * s.d_v) * sizeof(float);
   err = cudaFuncSetAttribute(topk_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg.dynamicSmemBytes);
   if (err != cudaSuccess) return err;
   err = cudaLaunchKernelEx(&cfg, topk_attend_kernel, ap);
