@@ -171,7 +171,9 @@ diffqkv_status diffqkv_combine(const float *o_partial, const float *lse_partial,
  *          both pools are overwritten; seqlens itself is not modified (the caller adds q_len)
  *   out    [batch, q_len, n_q, d_v] out_dtype; query row i sees tokens 0 .. past_b + i
  *   lse    [batch, q_len, n_q] fp32 or NULL
- * Requires bf16, d_qk == d_v == 128 (tensor-core tiles).
+ * bf16 with d_qk == d_v == 128 (and pages of at least 8 tokens that divide or are multiples of 128) runs on the
+ * tensor cores; every other shape diffqkv_decode accepts (fp32, other head dimensions, d_qk != d_v) runs the same
+ * two steps on a plain fp32-FMA kernel, one block per query row, which is a correctness path, not a fast one.
  */
 diffqkv_status diffqkv_prefill(const void *q, const void *k_new, const void *v_new, int32_t q_len,
                                const diffqkv_cache *cache, const diffqkv_shape *shape, void *out, float *lse,
@@ -268,6 +270,9 @@ void diffqkv_set_max_blocks(int32_t max_blocks);
  * reach the top.  Both give the same result.
  */
 void diffqkv_topk_general_only(int32_t on);
+
+/* Which attention kernel the most recent diffqkv_prefill call launched: 0 none yet, 1 generic, 2 tensor-core (for tests). */
+int32_t diffqkv_last_prefill_kernel(void);
 
 /* Which split kernel the most recent decode call launched: 0 none yet, 1 generic, 2 TMA (for tests). */
 int32_t diffqkv_last_decode_kernel(void);

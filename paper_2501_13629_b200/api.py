@@ -29,9 +29,9 @@ EXPORTS = (
     "diffqkv_decode_num_splits", "diffqkv_decode_workspace_bytes", "diffqkv_decode", "gqa_decode",
     "diffqkv_combine", "diffqkv_prefill", "diffqkv_augq_workspace_bytes", "diffqkv_augq",
     "diffqkv_status_string", "diffqkv_launch_count", "diffqkv_profile_split_events", "diffqkv_decode_static",
-    "diffqkv_set_max_blocks", "diffqkv_topk_general_only", "diffqkv_last_decode_kernel", "diffqkv_augq_rope",
-    "diffqkv_project",
-    "diffqkv_cache_append", "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes",
+    "diffqkv_set_max_blocks", "diffqkv_topk_general_only", "diffqkv_last_decode_kernel",
+    "diffqkv_last_prefill_kernel", "diffqkv_augq_rope", "diffqkv_project", "diffqkv_cache_append",
+    "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes",
 )
 
 
@@ -95,6 +95,8 @@ _lib.diffqkv_decode_topk.argtypes = [C.c_void_p, C.POINTER(CacheStruct), C.POINT
 _lib.diffqkv_status_string.restype = C.c_char_p
 _lib.diffqkv_status_string.argtypes = [C.c_int]
 _lib.diffqkv_launch_count.restype = C.c_int64
+_lib.diffqkv_last_prefill_kernel.restype = C.c_int32
+_lib.diffqkv_last_prefill_kernel.argtypes = []
 _lib.diffqkv_topk_general_only.restype = None
 _lib.diffqkv_topk_general_only.argtypes = [C.c_int32]
 _lib.diffqkv_set_max_blocks.restype = None
@@ -134,6 +136,11 @@ def set_max_blocks(n: int) -> None:
 
 
 KERNEL_NONE, KERNEL_GENERIC, KERNEL_TMA = 0, 1, 2
+
+
+def last_prefill_kernel() -> int:
+    """0 = no prefill yet, 1 = generic kernel, 2 = tensor-core kernel (most recent diffqkv_prefill call)."""
+    return int(_lib.diffqkv_last_prefill_kernel())
 
 
 def last_decode_kernel() -> int:

@@ -211,6 +211,8 @@ diffqkv_status diffqkv_combine(const float* o_partial, const float* lse_partial,
   return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
 
+static int g_last_prefill_kernel = 0;  // 0 none yet, 1 generic, 2 tensor-core (for tests)
+
 diffqkv_status diffqkv_prefill(const void* q, const void* k_new, const void* v_new, int32_t q_len,
                                const diffqkv_cache* cache, const diffqkv_shape* shape, void* out, float* lse,
                                int32_t* dev_status, void* stream) {
@@ -221,14 +223,34 @@ diffqkv_status diffqkv_prefill(const void* q, const void* k_new, const void* v_n
   if (st != DIFFQKV_OK) return st;
   if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return DIFFQKV_ERR_ALIGNMENT;
   if (q_len > cache->max_seqlen) return DIFFQKV_ERR_INVALID_ARG;
-  int box_tok = 0;
-  if (!prefill_supported(*shape, *cache, &box_tok)) return DIFFQKV_ERR_UNSUPPORTED;
   if (shape->batch == 0 || q_len == 0) return DIFFQKV_OK;
-  const cudaError_t err = launch_prefill(q, k_new, v_new, q_len, *cache, *shape, box_tok, out, lse, dev_status,
-                                         static_cast<cudaStream_t>(stream));
+  cudaStream_t st_ = static_cast<cudaStream_t>(stream);
+  int box_tok = 0;
+  cudaError_t err = cudaErrorNotSupported;
+  if (prefill_supported(*shape, *cache, &box_tok))  // bf16, d 128: cache update + tensor-core attention
+    err = launch_prefill(q, k_new, v_new, q_len, *cache, *shape, box_tok, out, lse, dev_status, st_);
+  if (err == cudaErrorNotSupported) {  // everything else: the same two steps on the generic kernels
+    err = launch_cache_append(k_new, v_new, q_len, *cache, *shape, dev_status, st_);
+    if (err != cudaSuccess) return DIFFQKV_ERR_CUDA;
+    DecodeParams p;
+    p.q = q;
+    p.cache = view_of(cache);
+    p.batch = shape->batch; p.n_q = shape->n_q; p.n_k = shape->n_k; p.n_v = shape->n_v;
+    p.d_qk = shape->d_qk; p.d_v = shape->d_v;
+    p.scale_log2 = shape->scale * kLog2e;
+    p.chunk = 0; p.splits = 1;
+    p.o_partial = nullptr; p.lse_partial = nullptr;
+    p.dev_status = dev_status;
+    err = launch_prefill_generic(p, shape->dtype, q_len, out, shape->out_dtype == DIFFQKV_F32, lse, st_);
+    g_last_prefill_kernel = 1;
+  } else {
+    g_last_prefill_kernel = 2;
+  }
   if (err == cudaErrorNotSupported) return DIFFQKV_ERR_UNSUPPORTED;
   return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
+
+int32_t diffqkv_last_prefill_kernel(void) { return g_last_prefill_kernel; }
 
 size_t diffqkv_augq_workspace_bytes(int64_t T, int32_t d_q0, int32_t d_aug) {
   if (T < 0 || d_q0 <= 0 || d_aug <= 0) return 0;

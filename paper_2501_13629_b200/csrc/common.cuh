@@ -54,6 +54,8 @@ __device__ __forceinline__ void report(int* dev_status, int code) {
 
 // Launchers (defined next to their kernels).
 cudaError_t launch_decode_generic(const DecodeParams& p, diffqkv_dtype dtype, cudaStream_t stream);
+cudaError_t launch_prefill_generic(const DecodeParams& p, diffqkv_dtype dtype, int q_len, void* out, int out_is_f32,
+                                   float* lse, cudaStream_t stream);
 cudaError_t launch_combine(const float* o_partial, const float* lse_partial, int rows, int d_v, int splits,
                            diffqkv_dtype out_dtype, void* out, float* lse, cudaStream_t stream);
 void count_launch(int n = 1);

@@ -206,9 +206,9 @@ def test_argument_errors(api):
     z = lambda *s: torch.zeros(s, dtype=torch.bfloat16, device=dev)
     lens = torch.zeros(1, dtype=torch.int32, device=dev)
     cache = api.KVCache(z(1, 2, 64, 64), z(1, 2, 64, 64), lens, 64)
-    with pytest.raises(api.DiffQKVError) as e:  # head dimension 64 has no tensor-core prefill kernel
-        api.diffqkv_prefill(z(1, 8, 4, 64), z(1, 8, 2, 64), z(1, 8, 2, 64), cache, 0.125)
-    assert e.value.status == api.ERR_UNSUPPORTED
+    with pytest.raises(api.DiffQKVError) as e:  # 3 query heads cannot share 2 K heads
+        api.diffqkv_prefill(z(1, 8, 3, 64), z(1, 8, 2, 64), z(1, 8, 1, 64), cache, 0.125)
+    assert e.value.status == api.ERR_INVALID_ARG
     cache = api.KVCache(z(1, 2, 64, 128), z(1, 2, 64, 128), lens, 64)
     with pytest.raises(api.DiffQKVError) as e:  # more new tokens than the cache can hold
         api.diffqkv_prefill(z(1, 100, 4, 128), z(1, 100, 2, 128), z(1, 100, 2, 128), cache, 0.1)
