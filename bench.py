@@ -314,6 +314,19 @@ def time_prefill(api, W, device, peaks, steps):
     res["augq_rope"] = {"ms": augq_rope_ms, "TFLOP/s": augq_flops / augq_rope_ms / 1e9}
     res["attention"]["note"] = "causal flops (lower triangle incl. diagonal); time includes the cache-update kernel"
     res["working_set"] = "weights 92 MB + activations 0.5 GB per step: larger than L2"
+    # the same causal attention with SIGMA-1.5B's heads (32 query / 4 K / 16 V heads of 64 channels)
+    d64, nk64, nv64 = 64, 4, 16
+    q64 = rn(cfg.batch, cfg.seq, cfg.n_q, d64)
+    k64n, v64n = rn(cfg.batch, cfg.seq, nk64, d64), rn(cfg.batch, cfg.seq, nv64, d64)
+    cache64 = api.KVCache(torch.zeros(cfg.batch, nk64, cfg.seq, d64, dtype=torch.bfloat16, device=device),
+                          torch.zeros(cfg.batch, nv64, cfg.seq, d64, dtype=torch.bfloat16, device=device),
+                          torch.zeros(cfg.batch, dtype=torch.int32, device=device), cfg.seq)
+    out64 = torch.empty(cfg.batch, cfg.seq, cfg.n_q, d64, dtype=torch.bfloat16, device=device)
+    ms64 = timed(lambda: api.diffqkv_prefill(q64, k64n, v64n, cache64, d64 ** -0.5, out=out64, dev_status=status))
+    assert int(status.item()) == 0, "device status reported an error"
+    fl64 = 2.0 * cfg.batch * cfg.n_q * (cfg.seq * (cfg.seq + 1) / 2) * (2 * d64)
+    res["attention_sigma1p5b_heads_d64"] = {"ms": ms64, "TFLOP/s": fl64 / ms64 / 1e9, "flops": fl64,
+                                            "heads": "32 query / 4 K / 16 V, 64 channels"}
     return res
 
 

@@ -171,8 +171,8 @@ diffqkv_status diffqkv_combine(const float *o_partial, const float *lse_partial,
  *          both pools are overwritten; seqlens itself is not modified (the caller adds q_len)
  *   out    [batch, q_len, n_q, d_v] out_dtype; query row i sees tokens 0 .. past_b + i
  *   lse    [batch, q_len, n_q] fp32 or NULL
- * bf16 with d_qk == d_v == 128 (and pages of at least 8 tokens that divide or are multiples of 128) runs on the
- * tensor cores; every other shape diffqkv_decode accepts (fp32, other head dimensions, d_qk != d_v) runs the same
+ * bf16 with d_qk == d_v == 128 or 64 (and pages of at least 8 tokens that divide or are multiples of 128) runs on
+ * the tensor cores; every other shape diffqkv_decode accepts (fp32, other head dimensions, d_qk != d_v) runs the same
  * two steps on a plain fp32-FMA kernel, one block per query row, which is a correctness path, not a fast one.
  */
 diffqkv_status diffqkv_prefill(const void *q, const void *k_new, const void *v_new, int32_t q_len,

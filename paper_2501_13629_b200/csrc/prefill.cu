@@ -12,12 +12,14 @@
 //                 token-major tile); the two M-tiles alternate, so the tensor core works on one while the softmax
 //                 warps work on the other.  Operands are what bounds these products (about 100 bytes per cycle
 //                 reach the tensor core from shared memory), hence 128-wide tiles and P kept out of shared memory.
-//     warps 2-5   softmax of M-tile 0, warps 6-9 of M-tile 1: one thread per query row (= TMEM lane).  Pass 1 reads
-//                 the 128 scores (tcgen05.ld) for the row maximum; a running reference maximum is only raised when
-//                 exceeded by 2^8 (then O is rescaled in TMEM).  Pass 2 reads them again 32 at a time, computes
-//                 P = 2^(S scale - m), sums it in fp32 and writes it as packed bf16 over the scores it has already
-//                 consumed (tcgen05.st), where the second product reads it.
+//     warps 2-5   softmax of M-tile 0, warps 6-9 of M-tile 1: one thread per query row (= TMEM lane).  The thread
+//                 reads its 128 scores into registers (tcgen05.ld), takes the row maximum (a running reference
+//                 maximum is only raised when exceeded by 2^8; then O is rescaled in TMEM), computes
+//                 P = 2^(S scale - m), sums it in fp32 and writes it as packed bf16 over the first 64 score columns
+//                 (tcgen05.st), where the second product reads it.
 //   fp32 scores, softmax statistics and output accumulation; P is rounded to bf16 for the second product.
+//   The kernel is a template on the head dimension (128 or 64 channels for Q/K and V alike): with 64 the tiles are
+//   half as wide, the first product takes four K steps instead of eight and O takes 64 TMEM columns per M-tile.
 // Every wait is bounded; on expiry the block reports DIFFQKV_ERR_TIMEOUT, drains and frees its TMEM.
 #include "common.cuh"
 #include "ptx.cuh"
@@ -29,13 +31,12 @@ namespace {
 
 constexpr int kQT = 128;  // query rows per M-tile
 constexpr int kKT = 128;  // cached tokens per KV tile
-constexpr int kD = 128;   // channels per head (Q/K and V)
+constexpr int kDMax = 128;  // channels per head (Q/K and V): the kernel is built for 128 and for 64
 constexpr int kKSlots = 3, kVSlots = 2;
-constexpr int kQBytes = kQT * kD * 2;  // 32 KB: [half][128 rows][128 B]
-constexpr int kTBytes = kKT * kD * 2;  // 32 KB, a K tile or a V tile: [half][128 rows][128 B]
 constexpr int kPrefillThreads = 320;
-constexpr int kTmemCols = 512;         // S[t] (and P[t] over its first 64 columns) at 128 t, O[t] at 256 + 128 t
-constexpr int kPrefillSmem = 1024 + 2 * kQBytes + (kKSlots + kVSlots) * kTBytes + 256;
+constexpr int kTmemCols = 512;         // S[t] (and P[t] over its first 64 columns) at 128 t, O[t] at 256 + D t
+// Shared memory is sized for D = 128 whatever D is: one block per SM, since a block takes all of the tensor memory.
+constexpr int kPrefillSmem = 1024 + 2 * (kQT * kDMax * 2) + (kKSlots + kVSlots) * (kKT * kDMax * 2) + 256;
 constexpr float kRescaleThreshold = 8.f;  // log2 domain
 
 struct PrefillParams {
@@ -71,9 +72,13 @@ __device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity, volatil
   return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity, abort_flag));
 }
 
+template <int kD>  // channels per head, 64 or 128
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, const PrefillParams p) {
+  constexpr int kHalves = kD / 64;          // 64-channel halves of a row
+  constexpr int kQBytes = kQT * kD * 2;     // a Q tile: [half][128 rows][128 B]
+  constexpr int kTBytes = kKT * kD * 2;     // a K tile or a V tile: [half][128 rows][128 B]
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* q_s = smem;                      // 2 M-tiles
@@ -150,8 +155,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     }
     // One box per (token part, channel half) of a tile: lane x owns box x of every K tile and of every V tile.
     const int parts = kKT / p.box_tok;
-    const int boxes = 2 * parts;
-    const int my_part = lane >> 1, my_half = lane & 1;
+    const int boxes = kHalves * parts;
+    const int my_part = lane / kHalves, my_half = lane % kHalves;
     const uint32_t my_off = my_half * (kKT * 128) + my_part * (p.box_tok * 128);
     int ks = 0, vs = 0, issued_k = 0, issued_v = 0;
     uint32_t kph = 0, vph = 0;
@@ -170,7 +175,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           blk = 0;
         }
       }
-      const uint32_t tx = (uint32_t)parts_valid * p.box_tok * 128u * 2u;
+      const uint32_t tx = (uint32_t)parts_valid * p.box_tok * 128u * kHalves;
       if (!wait_warp(k_empty0 + 8 * ks, kph ^ 1, abort_flag)) { ok = false; break; }
       if (lane == 0) ptx::mbar_arrive_expect_tx(k_full0 + 8 * ks, tx);
       __syncwarp();
@@ -196,7 +201,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (one thread)
     constexpr uint32_t idesc = tc::idesc_bf16_f32(kQT, 128, 0, 0);     // S: Q and K both K-major, N = 128 tokens
-    constexpr uint32_t idesc_pv = tc::idesc_bf16_f32(kQT, kD, 0, 1);   // O: V is N-major, N = 128 channels
+    constexpr uint32_t idesc_pv = tc::idesc_bf16_f32(kQT, kD, 0, 1);   // O: V is N-major, N = kD channels
     constexpr uint32_t hi = tc::smem_desc_hi_sw128(1024);              // 8-row groups are 1024 bytes apart everywhere
     bool ok = true;
     if (lane == 0) {
@@ -341,7 +346,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           if (!wait_warp(v_full0 + 8 * vslot, (j / kVSlots) & 1, abort_flag)) { ok = false; break; }
           if (r >= kv_len - k0) {
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
+            for (int half = 0; half < kHalves; ++half) {
               uint4* dst = reinterpret_cast<uint4*>(v_s + vslot * kTBytes + half * (kKT * 128) + r * 128);
 #pragma unroll
               for (int e = 0; e < 8; ++e) dst[e] = make_uint4(0, 0, 0, 0);
@@ -454,9 +459,9 @@ __global__ void __launch_bounds__(256) cache_append_kernel(const AppendParams p)
 
 // Tensor map over one cache pool: dims (64 channels, token slot, channel half, head, block); a box brings
 // box_tok tokens of one 64-channel half.
-bool make_cache_map(CUtensorMap* map, const void* base, long long tok_extent, int heads, long long blocks,
+bool make_cache_map(CUtensorMap* map, const void* base, int d, long long tok_extent, int heads, long long blocks,
                     long long st_tok, long long st_head, long long st_blk, int box_tok) {
-  const cuuint64_t dims[5] = {64, (cuuint64_t)tok_extent, (cuuint64_t)(kD / 64), (cuuint64_t)heads, (cuuint64_t)blocks};
+  const cuuint64_t dims[5] = {64, (cuuint64_t)tok_extent, (cuuint64_t)(d / 64), (cuuint64_t)heads, (cuuint64_t)blocks};
   const cuuint64_t strides[4] = {(cuuint64_t)st_tok * 2, 128, (cuuint64_t)st_head * 2, (cuuint64_t)st_blk * 2};
   const cuuint32_t box[5] = {64, (cuuint32_t)box_tok, 1, 1, 1};
   return make_tmap_bf16_sw128(map, base, 5, dims, strides, box);
@@ -465,7 +470,7 @@ bool make_cache_map(CUtensorMap* map, const void* base, long long tok_extent, in
 }  // namespace
 
 bool prefill_supported(const diffqkv_shape& s, const diffqkv_cache& c, int* box_tok) {
-  if (s.dtype != DIFFQKV_BF16 || s.d_qk != kD || s.d_v != kD) return false;
+  if (s.dtype != DIFFQKV_BF16 || s.d_qk != s.d_v || (s.d_qk != 64 && s.d_qk != 128)) return false;
   int bt = kKT;
   if (c.page_table) {
     if (c.page_size >= kKT) { if (c.page_size % kKT != 0) return false; }
@@ -509,18 +514,19 @@ cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, 
   if (err != cudaSuccess) return err;
 
   // ---- step 2: attention over the cache
+  const int d = s.d_qk;  // == d_v, 64 or 128
   CUtensorMap mq, mk, mv;
   {
-    const cuuint64_t dims[5] = {64, (cuuint64_t)q_len, (cuuint64_t)(kD / 64), (cuuint64_t)s.n_q, (cuuint64_t)s.batch};
-    const cuuint64_t strides[4] = {(cuuint64_t)s.n_q * kD * 2, 128, (cuuint64_t)kD * 2,
-                                   (cuuint64_t)q_len * s.n_q * kD * 2};
-    const cuuint32_t box[5] = {64, kQT, kD / 64, 1, 1};
+    const cuuint64_t dims[5] = {64, (cuuint64_t)q_len, (cuuint64_t)(d / 64), (cuuint64_t)s.n_q, (cuuint64_t)s.batch};
+    const cuuint64_t strides[4] = {(cuuint64_t)s.n_q * d * 2, 128, (cuuint64_t)d * 2,
+                                   (cuuint64_t)q_len * s.n_q * d * 2};
+    const cuuint32_t box[5] = {64, kQT, (cuuint32_t)(d / 64), 1, 1};
     if (!make_tmap_bf16_sw128(&mq, q, 5, dims, strides, box)) return cudaErrorNotSupported;
   }
   const long long tok_extent = c.page_table ? c.page_size : c.max_seqlen;
-  if (!make_cache_map(&mk, c.k_cache, tok_extent, s.n_k, c.num_blocks, c.k_stride_tok, c.k_stride_head,
+  if (!make_cache_map(&mk, c.k_cache, d, tok_extent, s.n_k, c.num_blocks, c.k_stride_tok, c.k_stride_head,
                       c.k_stride_blk, box_tok) ||
-      !make_cache_map(&mv, c.v_cache, tok_extent, s.n_v, c.num_blocks, c.v_stride_tok, c.v_stride_head,
+      !make_cache_map(&mv, c.v_cache, d, tok_extent, s.n_v, c.num_blocks, c.v_stride_tok, c.v_stride_head,
                       c.v_stride_blk, box_tok))
     return cudaErrorNotSupported;
   PrefillParams p;
@@ -534,9 +540,15 @@ cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, 
   p.out = out; p.out_is_f32 = s.out_dtype == DIFFQKV_F32; p.lse = lse; p.dev_status = dev_status;
   const long long grid = (long long)p.n_qpairs * s.batch * s.n_q;
   if (grid > 0x7fffffffLL) return cudaErrorNotSupported;
-  err = cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrefillSmem);
-  if (err != cudaSuccess) return err;
-  prefill_attn_kernel<<<(unsigned)grid, kPrefillThreads, kPrefillSmem, stream>>>(mq, mk, mv, p);
+  if (d == 128) {
+    err = cudaFuncSetAttribute(prefill_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrefillSmem);
+    if (err != cudaSuccess) return err;
+    prefill_attn_kernel<128><<<(unsigned)grid, kPrefillThreads, kPrefillSmem, stream>>>(mq, mk, mv, p);
+  } else {
+    err = cudaFuncSetAttribute(prefill_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrefillSmem);
+    if (err != cudaSuccess) return err;
+    prefill_attn_kernel<64><<<(unsigned)grid, kPrefillThreads, kPrefillSmem, stream>>>(mq, mk, mv, p);
+  }
   count_launch();
   return cudaGetLastError();
 }

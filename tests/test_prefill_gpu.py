@@ -23,8 +23,9 @@ def api():
 class Case:
     """Seeded prefill problem with a contiguous [batch, head, S, d] cache holding `past` earlier tokens."""
 
-    def __init__(self, seed, batch, q_len, heads, past, S=None, q_std=1.0, garbage=None):
+    def __init__(self, seed, batch, q_len, heads, past, S=None, q_std=1.0, garbage=None, d=D):
         n_q, n_k, n_v = heads
+        self.d = D = d
         self.batch, self.q_len, self.heads = batch, q_len, heads
         self.past = np.asarray(past, dtype=np.int32)
         self.S = S or int(self.past.max() + q_len)
@@ -40,7 +41,7 @@ class Case:
         self.scale = D ** -0.5
 
     def strides(self, n):
-        return (n * self.S * D, self.S * D, D)
+        return (n * self.S * self.d, self.S * self.d, self.d)
 
 
 def run_gpu(api, case, paged=None, out_dtype=torch.float32):
@@ -53,7 +54,7 @@ def run_gpu(api, case, paged=None, out_dtype=torch.float32):
         cache = api.KVCache(k, v, seqlens, case.S, k_strides=case.strides(n_k), v_strides=case.strides(n_v),
                             num_blocks=case.batch)
     else:
-        inp = W.DecodeInputs(W.DecodeConfig("t", case.batch, n_q, n_k, n_v, D, D, case.S), None, case.k, case.v,
+        inp = W.DecodeInputs(W.DecodeConfig("t", case.batch, n_q, n_k, n_v, case.d, case.d, case.S), None, case.k, case.v,
                              case.past, case.strides(n_k), case.strides(n_v), max_seqlen=case.S)
         pg = W.paginate(inp, paged, seed=99)
         k, v = W.to_torch(pg.k, dev), W.to_torch(pg.v, dev)
@@ -85,7 +86,7 @@ def run_oracle(oracle, case, rows=None):
     k, v = case.k.copy(), case.v.copy()
     cache = oracle.Cache(k, v, case.strides(n_k), case.strides(n_v), case.past)
     oracle.cache_append(case.k_new, case.v_new, cache)
-    out, lse = oracle.prefill(case.q, case.past, cache, n_k, n_v, D, case.scale, rows=rows)
+    out, lse = oracle.prefill(case.q, case.past, cache, n_k, n_v, case.d, case.scale, rows=rows)
     return out, lse, k, v
 
 
@@ -199,6 +200,18 @@ def test_config4_full_size_sampled_rows(api, oracle):
     check_bf16(got, ref, "cfg4 sampled rows")
     check_lse(lse[rows[:, 0], rows[:, 1], rows[:, 2]], lse_ref, 2e-2, "cfg4 lse")
     assert np.isfinite(out).all()
+
+
+@pytest.mark.parametrize("q_len,past", [(1, [0, 0]), (129, [0, 70]), (300, [257, 5]), (700, [0, 0])])
+def test_head_dimension_64_on_the_tensor_cores(api, oracle, q_len, past):
+    """SIGMA-1.5B's head size: the same kernel with half-width tiles."""
+    check_case(api, oracle, Case(800 + q_len, 2, q_len, (8, 2, 4), past, d=64), f"d=64 q_len={q_len} past={past}")
+    assert api.last_prefill_kernel() == 2
+
+
+@pytest.mark.parametrize("page", [16, 128])
+def test_head_dimension_64_paged(api, oracle, page):
+    check_case(api, oracle, Case(850 + page, 2, 200, (32, 4, 16), [100, 0], d=64), f"d=64 page={page}", paged=page)
 
 
 def test_argument_errors(api):
