@@ -271,6 +271,14 @@ void diffqkv_set_max_blocks(int32_t max_blocks);
  */
 void diffqkv_topk_general_only(int32_t on);
 
+/*
+ * Test hook (process-wide host state): the projections (diffqkv_augq, diffqkv_augq_rope, diffqkv_project) take a
+ * weight-streaming kernel when there are at most 64 rows (decode: one token per sequence) and the tensor-core GEMM
+ * otherwise; a non-zero value makes them always take the tensor-core GEMM.  Both round x and a to bf16 once and
+ * accumulate in fp32; they differ in summation order only.
+ */
+void diffqkv_force_tensor_gemm(int32_t on);
+
 /* Which attention kernel the most recent diffqkv_prefill call launched: 0 none yet, 1 generic, 2 tensor-core (for tests). */
 int32_t diffqkv_last_prefill_kernel(void);
 

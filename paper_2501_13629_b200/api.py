@@ -30,7 +30,7 @@ EXPORTS = (
     "diffqkv_combine", "diffqkv_prefill", "diffqkv_augq_workspace_bytes", "diffqkv_augq",
     "diffqkv_status_string", "diffqkv_launch_count", "diffqkv_profile_split_events", "diffqkv_decode_static",
     "diffqkv_set_max_blocks", "diffqkv_topk_general_only", "diffqkv_last_decode_kernel",
-    "diffqkv_last_prefill_kernel", "diffqkv_augq_rope", "diffqkv_project", "diffqkv_cache_append",
+    "diffqkv_last_prefill_kernel", "diffqkv_force_tensor_gemm", "diffqkv_augq_rope", "diffqkv_project", "diffqkv_cache_append",
     "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes",
 )
 
@@ -95,6 +95,8 @@ _lib.diffqkv_decode_topk.argtypes = [C.c_void_p, C.POINTER(CacheStruct), C.POINT
 _lib.diffqkv_status_string.restype = C.c_char_p
 _lib.diffqkv_status_string.argtypes = [C.c_int]
 _lib.diffqkv_launch_count.restype = C.c_int64
+_lib.diffqkv_force_tensor_gemm.restype = None
+_lib.diffqkv_force_tensor_gemm.argtypes = [C.c_int32]
 _lib.diffqkv_last_prefill_kernel.restype = C.c_int32
 _lib.diffqkv_last_prefill_kernel.argtypes = []
 _lib.diffqkv_topk_general_only.restype = None
@@ -136,6 +138,11 @@ def set_max_blocks(n: int) -> None:
 
 
 KERNEL_NONE, KERNEL_GENERIC, KERNEL_TMA = 0, 1, 2
+
+
+def force_tensor_gemm(on: bool) -> None:
+    """Test hook: make the projections always take the tensor-core GEMM; see diffqkv_force_tensor_gemm."""
+    _lib.diffqkv_force_tensor_gemm(int(bool(on)))
 
 
 def last_prefill_kernel() -> int:

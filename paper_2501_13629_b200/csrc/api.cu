@@ -181,6 +181,8 @@ void diffqkv_set_max_blocks(int32_t max_blocks) { set_tma_max_blocks(max_blocks)
 
 void diffqkv_topk_general_only(int32_t on) { set_topk_general_only(on); }
 
+void diffqkv_force_tensor_gemm(int32_t on) { set_force_tensor_gemm(on); }
+
 int32_t diffqkv_last_decode_kernel(void) { return g_last_kernel; }
 
 diffqkv_status diffqkv_decode(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape,

@@ -281,10 +281,15 @@ int sm_count() {
   return sms;
 }
 
+int g_force_tensor_gemm = 0;  // test hook: 1 = never take the weight-streaming kernel for few rows
+
 // C[M, N] = A[M, K] . B0[N, K]^T, or with B1: C[M, N] = silu(A.B0^T) * (A.B1^T).
 cudaError_t launch_gemm(const void* A, const void* B0, const void* B1, void* C, long long M, int N, int K,
                         int* dev_status, cudaStream_t stream, const float* rope_cos = nullptr,
                         const float* rope_sin = nullptr, int head_dim = 0) {
+  // a handful of rows (decode): the weight-streaming kernel; its tiles would leave most SMs of this one idle
+  if (!g_force_tensor_gemm && linear_skinny_supported(M, N, K, B1 != nullptr, head_dim, rope_cos != nullptr))
+    return launch_linear_skinny(A, B0, B1, C, M, N, K, dev_status, stream, rope_cos, rope_sin, head_dim);
   CUtensorMap ma, mb0, mb1;
   if (!make_operand_map(&ma, A, M, K) || !make_operand_map(&mb0, B0, N, K) ||
       !make_operand_map(&mb1, B1 ? B1 : B0, N, K))
@@ -314,6 +319,8 @@ cudaError_t launch_gemm(const void* A, const void* B0, const void* B1, void* C, 
 }
 
 }  // namespace
+
+void set_force_tensor_gemm(int on) { g_force_tensor_gemm = on != 0; }
 
 size_t augq_workspace_bytes(long long T, int d_q0, int d_aug) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };

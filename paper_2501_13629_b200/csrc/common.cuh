@@ -59,6 +59,16 @@ cudaError_t launch_prefill_generic(const DecodeParams& p, diffqkv_dtype dtype, i
 cudaError_t launch_combine(const float* o_partial, const float* lse_partial, int rows, int d_v, int splits,
                            diffqkv_dtype out_dtype, void* out, float* lse, cudaStream_t stream);
 void count_launch(int n = 1);
+
+// Linear layers for at most kSkinnyMaxRows rows of x (weight-streaming kernel, linear_skinny.cu); same operands as the
+// tensor-core GEMM of augq.cu: C[M, N] = A[M, K] . B0[N, K]^T, with B1 silu(A.B0^T) * (A.B1^T), with rope_cos/rope_sin
+// the rotate-half rotary embedding per head of head_dim channels.
+constexpr int kSkinnyMaxRows = 64;
+void set_force_tensor_gemm(int on);
+bool linear_skinny_supported(long long M, int N, int K, bool dual, int head_dim, bool rotary);
+cudaError_t launch_linear_skinny(const void* A, const void* B0, const void* B1, void* C, long long M, int N, int K,
+                                 int* dev_status, cudaStream_t stream, const float* rope_cos, const float* rope_sin,
+                                 int head_dim);
 void profile_after_split(cudaStream_t stream);  // records the benchmark hook's second event, if armed
 
 // TMA decode path (decode_tma.cu): persistent blocks over a flat (sequence, unit, tile) list.

@@ -1,0 +1,269 @@
+// Linear layers for a handful of rows (decode: one new token per sequence): y[M, N] = x[M, K] . W[N, K]^T with the
+// epilogues of the projection chain (plain; silu(gate) * up over two weight matrices; rotate-half rotary embedding).
+//
+// With M <= 64 rows the tensor-core GEMM of augq.cu has 16 to 24 column tiles for 148 SMs and every tile streams its
+// weight panel alone, so the step is bound by how few SMs pull on HBM (74 us for the aug-Q chain of config 4's widths
+// where the weights, read once, take 14 us).  Here the weights are the streamed operand and the rows the stationary
+// one, as in the decode kernels:
+//   item       16 weight rows over the whole K: two groups of 8 rows that the epilogue needs side by side (plain: rows
+//              16 i .. 16 i + 7 and 16 i + 8 .. 16 i + 15; gate/up: rows 8 i .. of W_gate and the same rows of W_up;
+//              rotary: channels c .. c + 7 of a head and their partners c + d/2 ..), times a pass of 16 rows of x.
+//              Items are dealt round-robin to one persistent block per SM, passes of an item back to back (the
+//              second pass finds the weight rows in L2).
+//   producer   one warp; a stage is 512 columns of K: two 8-row weight boxes (8 KB each) and a 16-row box of x
+//              (16 KB, from L2), TMA with 128-byte swizzle into a ring of 6 stages, bounded waits
+//   consumers  8 warps; a stage has 32 steps of 16 columns, warp w takes steps w, w + 8, ...: ldmatrix of the weight
+//              rows (A, 16 x 16) and of the x rows (B, 16 columns x 16 rows), two mma.sync.m16n8k16 into fp32
+//              accumulators; at the end of an item the eight partial sums meet in shared memory and warp 0 applies
+//              the epilogue: rows g and g + 8 of the accumulator tile, i.e. the two groups, sit in the same thread.
+// HBM-bound by design (2 flops per weight byte and row of x), hence mma.sync and not tcgen05.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+#include "tmap.cuh"
+
+namespace diffqkv {
+namespace {
+
+constexpr int kKC = 512;                  // columns of K per stage
+constexpr int kChunks = kKC / 64;         // 64-column chunks (128 bytes) per stage
+constexpr int kSkStages = 6;
+constexpr int kSkWarps = 8;               // consumer warps
+constexpr int kSkThreads = (kSkWarps + 1) * 32;
+constexpr int kWBox = kChunks * 8 * 128;  // one 8-row weight box
+constexpr int kXBox = kChunks * 16 * 128; // the 16-row box of x
+constexpr int kStageBytes = 2 * kWBox + kXBox;
+constexpr int kRedBytes = 2 * kSkWarps * 32 * 8 * 4;
+constexpr int kSkSmem = 1024 + kSkStages * kStageBytes + kRedBytes + 256;
+
+enum { kPlain = 0, kGateUp = 1, kRotary = 2 };
+
+struct SkinnyParams {
+  __nv_bfloat16* C;
+  int ldc, M, N, K;
+  int mode, head_dim;
+  int items, passes;  // items of 16 weight rows; passes of 16 rows of x
+  const float* rope_cos;
+  const float* rope_sin;
+  int* dev_status;
+};
+
+__device__ __forceinline__ void item_rows(const SkinnyParams& p, int item, int& row_a, int& row_b) {
+  if (p.mode == kGateUp) {
+    row_a = row_b = 8 * item;
+  } else if (p.mode == kRotary) {
+    const int half = p.head_dim >> 1, per_head = half >> 3;
+    row_a = (item / per_head) * p.head_dim + 8 * (item % per_head);
+    row_b = row_a + half;
+  } else {
+    row_a = 16 * item;
+    row_b = row_a + 8;
+  }
+}
+
+__global__ void __launch_bounds__(kSkThreads, 1)
+linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_wa,
+                     const __grid_constant__ CUtensorMap tmap_wb, const SkinnyParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  float* red = reinterpret_cast<float*>(smem + kSkStages * kStageBytes);  // [2][warp][lane][8]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSkStages * kStageBytes + kRedBytes);  // full[s], empty[s]
+  volatile int* abort_flag = reinterpret_cast<int*>(bars + 2 * kSkStages);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t full0 = ptx::smem_u32(bars), empty0 = ptx::smem_u32(bars + kSkStages);
+  if (tid == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < kSkStages; ++s) {
+      ptx::mbar_init(full0 + 8 * s, 1);
+      ptx::mbar_init(empty0 + 8 * s, kSkWarps);
+    }
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmap_x);
+    ptx::prefetch_tmap(&tmap_wa);
+    ptx::prefetch_tmap(&tmap_wb);
+  }
+  __syncthreads();
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();  // x may be the output of the grid before this one
+
+  const int total = p.items * p.passes;
+  const int n_chunks = (p.K + kKC - 1) / kKC;  // stages per item (columns past K read as zero)
+  const uint32_t smem_u32 = ptx::smem_u32(smem);
+
+  if (warp == kSkWarps) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      int stage = 0, issued = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; it < total && ok; it += gridDim.x) {
+        int row_a, row_b;
+        item_rows(p, it / p.passes, row_a, row_b);
+        const int xrow = 16 * (it % p.passes);
+        for (int c = 0; c < n_chunks; ++c) {
+          if (issued >= kSkStages && !ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) {
+            report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+            ok = false;
+            break;
+          }
+          const uint32_t bar = full0 + 8 * stage, dst = smem_u32 + stage * kStageBytes;
+          ptx::mbar_arrive_expect_tx(bar, kStageBytes);
+          ptx::tma_load_3d(dst, &tmap_wa, bar, 0, row_a, c * kChunks);
+          ptx::tma_load_3d(dst + kWBox, &tmap_wb, bar, 0, row_b, c * kChunks);
+          ptx::tma_load_3d(dst + 2 * kWBox, &tmap_x, bar, 0, xrow, c * kChunks);
+          ++issued;
+          if (++stage == kSkStages) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {  // give copies in flight a bounded chance to land before the block's shared memory is released
+        for (int s = 0; s < min(issued, kSkStages); ++s) {
+          const int uses = (issued - s + kSkStages - 1) / kSkStages;
+          ptx::mbar_wait(full0 + 8 * s, (uint32_t)(uses - 1) & 1u, nullptr);
+        }
+      }
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- consumers
+  const int mi = lane >> 3, rr = lane & 7;
+  // A (weights): matrices (rows 0-7, k 0-7), (rows 8-15, k 0-7), (rows 0-7, k 8-15), (rows 8-15, k 8-15); rows 8-15
+  // are the second box.  B (x): matrices (rows 0-7, k 0-7), (rows 0-7, k 8-15), (rows 8-15, k 0-7), (rows 8-15, k 8-15).
+  const uint32_t a_base = (mi & 1) * kWBox + rr * 128, a_half = mi >> 1;
+  const int xr = (mi >> 1) * 8 + rr;
+  const uint32_t b_base = 2 * kWBox + xr * 128, b_half = mi & 1;
+  int stage = 0, n_item = 0;
+  uint32_t phase = 0;
+  bool dead = false;
+  for (int it = blockIdx.x; it < total; it += gridDim.x, ++n_item) {
+    float acc[2][4];
+#pragma unroll
+    for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[nb][e] = 0.f;
+    for (int c = 0; c < n_chunks; ++c) {
+      if (!ptx::mbar_wait(full0 + 8 * stage, phase, abort_flag)) {
+        if (!dead) report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+        dead = true;  // keep walking the loops (no more waits succeed) so that the block's barriers still meet
+      }
+      if (!dead) {
+        const uint32_t st = smem_u32 + stage * kStageBytes;
+#pragma unroll
+        for (int s4 = 0; s4 < 32 / kSkWarps; ++s4) {
+          const int s = warp + s4 * kSkWarps;  // 16-column step of the stage
+          const uint32_t chunk = s >> 2, unit = (s & 3) * 2;
+          uint32_t a[4], b[4];
+          ptx::ldmatrix_x4(st + a_base + chunk * 1024 + (((unit + a_half) ^ rr) << 4), a);
+          ptx::ldmatrix_x4(st + b_base + chunk * 2048 + (((unit + b_half) ^ rr) << 4), b);
+          ptx::mma_bf16_16816(acc[0], a, b[0], b[1]);
+          ptx::mma_bf16_16816(acc[1], a, b[2], b[3]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(empty0 + 8 * stage);
+      if (++stage == kSkStages) { stage = 0; phase ^= 1; }
+    }
+    // ---- the eight partial sums meet; warp 0 finishes the item
+    float* buf = red + (n_item & 1) * (kSkWarps * 32 * 8);
+    float4* mine = reinterpret_cast<float4*>(buf + (warp * 32 + lane) * 8);
+    mine[0] = make_float4(acc[0][0], acc[0][1], acc[0][2], acc[0][3]);
+    mine[1] = make_float4(acc[1][0], acc[1][1], acc[1][2], acc[1][3]);
+    asm volatile("bar.sync 1, %0;" ::"n"(kSkWarps * 32) : "memory");
+    if (warp == 0 && !dead) {
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = 0.f;
+#pragma unroll
+      for (int w = 0; w < kSkWarps; ++w) {
+        const float4* src = reinterpret_cast<const float4*>(buf + (w * 32 + lane) * 8);
+        const float4 lo = src[0], hi = src[1];
+        v[0] += lo.x; v[1] += lo.y; v[2] += lo.z; v[3] += lo.w;
+        v[4] += hi.x; v[5] += hi.y; v[6] += hi.z; v[7] += hi.w;
+      }
+      int row_a, row_b;
+      item_rows(p, it / p.passes, row_a, row_b);
+      const int g8 = lane >> 2, t4 = lane & 3;
+      // thread: weight rows g8 of either group, rows 2 t4 and 2 t4 + 1 of x in each 8-row half of the pass
+#pragma unroll
+      for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int t = 16 * (it % p.passes) + 8 * nb + 2 * t4 + e;
+          if (t >= p.M) continue;
+          const float ca = v[4 * nb + e], cb = v[4 * nb + 2 + e];
+          __nv_bfloat16* crow = p.C + (long long)t * p.ldc;
+          if (p.mode == kGateUp) {
+            crow[row_a + g8] = __float2bfloat16_rn(ca / (1.f + __expf(-ca)) * cb);
+          } else if (p.mode == kRotary) {
+            const int half = p.head_dim >> 1;
+            const long long ti = (long long)t * half + (row_a % p.head_dim) + g8;
+            const float cs = p.rope_cos[ti], sn = p.rope_sin[ti];
+            crow[row_a + g8] = __float2bfloat16_rn(ca * cs - cb * sn);
+            crow[row_b + g8] = __float2bfloat16_rn(cb * cs + ca * sn);
+          } else {
+            crow[row_a + g8] = __float2bfloat16_rn(ca);
+            crow[row_b + g8] = __float2bfloat16_rn(cb);
+          }
+        }
+    }
+  }
+}
+
+// dims (64 columns, rows, K / 64 chunks); a box is 64 columns x box_rows rows x kChunks chunks.
+bool make_rows_map(CUtensorMap* map, const void* base, long long rows, int K, int box_rows) {
+  const cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(K / 64)};
+  const cuuint64_t strides[2] = {(cuuint64_t)K * 2, 128};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)kChunks};
+  return make_tmap_bf16_sw128(map, base, 3, dims, strides, box);
+}
+
+}  // namespace
+
+bool linear_skinny_supported(long long M, int N, int K, bool dual, int head_dim, bool rotary) {
+  if (M < 1 || M > kSkinnyMaxRows || K % 64 != 0 || K < 64) return false;
+  if (rotary) return !dual && head_dim % 16 == 0 && head_dim >= 16 && N % head_dim == 0;
+  return dual ? N % 8 == 0 : N % 16 == 0;
+}
+
+cudaError_t launch_linear_skinny(const void* A, const void* B0, const void* B1, void* C, long long M, int N, int K,
+                                 int* dev_status, cudaStream_t stream, const float* rope_cos, const float* rope_sin,
+                                 int head_dim) {
+  CUtensorMap mx, ma, mb;
+  if (!make_rows_map(&mx, A, M, K, 16) || !make_rows_map(&ma, B0, N, K, 8) ||
+      !make_rows_map(&mb, B1 ? B1 : B0, N, K, 8))
+    return cudaErrorNotSupported;
+  SkinnyParams p;
+  p.C = reinterpret_cast<__nv_bfloat16*>(C);
+  p.ldc = N; p.M = (int)M; p.N = N; p.K = K;
+  p.mode = B1 ? kGateUp : (rope_cos ? kRotary : kPlain);
+  p.head_dim = head_dim;
+  p.items = p.mode == kGateUp ? N / 8 : N / 16;
+  p.passes = (int)((M + 15) / 16);
+  p.rope_cos = rope_cos; p.rope_sin = rope_sin;
+  p.dev_status = dev_status;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return cudaErrorUnknown;
+  const long long total = (long long)p.items * p.passes;
+  cudaError_t err = cudaFuncSetAttribute(linear_skinny_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSkSmem);
+  if (err != cudaSuccess) return err;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)(total < sms ? total : sms));
+  cfg.blockDim = dim3(kSkThreads);
+  cfg.dynamicSmemBytes = kSkSmem;
+  err = cudaLaunchKernelEx(&cfg, linear_skinny_kernel, mx, ma, mb, p);
+  if (err != cudaSuccess) return err;
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace diffqkv

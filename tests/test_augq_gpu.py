@@ -45,7 +45,7 @@ def _check(out, ref, what):
     assert rms <= 4e-3, f"{what}: rms err / rms ref = {rms:.3e}"
 
 
-@pytest.mark.parametrize("T", [1, 128, 300, 1000])
+@pytest.mark.parametrize("T", [1, 5, 16, 33, 64, 128, 300, 1000])
 @pytest.mark.parametrize("dims", [(256, 384, 384, 256), (128, 128, 128, 128), (512, 256, 640, 384)])
 def test_augq_small_shapes_every_row(api, oracle, T, dims):
     """Ragged row counts (tail tiles) and column counts that end in a half-filled 256-column tile."""

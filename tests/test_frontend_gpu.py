@@ -34,7 +34,7 @@ def _tables(oracle, pos, d, theta):
     return (torch.from_numpy(c.astype(np.float32)).cuda().contiguous(), torch.from_numpy(s.astype(np.float32)).cuda().contiguous())
 
 
-@pytest.mark.parametrize("T", [1, 200, 1000])
+@pytest.mark.parametrize("T", [1, 4, 16, 17, 50, 64, 65, 200, 1000])
 @pytest.mark.parametrize("heads,d", [(4, 128), (3, 128), (8, 64), (6, 64)])
 def test_projection_with_and_without_rotation(api, oracle, T, heads, d):
     """d_out = heads * d ends in a half-filled 256-column tile for odd head counts at d 128."""
@@ -53,6 +53,39 @@ def test_projection_with_and_without_rotation(api, oracle, T, heads, d):
     assert int(status.item()) == 0
     ref = oracle.rope(plain.reshape(T, heads, d), pos, theta).reshape(T, heads * d)
     _check(yr.float().cpu().numpy().astype(np.float64), ref, "rotated projection")
+
+
+@pytest.fixture
+def tensor_gemm(api):
+    """Switches the projections to the tensor-core GEMM for any row count and back."""
+    yield api.force_tensor_gemm
+    api.force_tensor_gemm(False)
+
+
+@pytest.mark.parametrize("T", [3, 16, 40])
+def test_few_rows_on_either_kernel(api, oracle, tensor_gemm, T):
+    """Up to 64 rows take the weight-streaming kernel, the tensor-core GEMM computes the same thing: both against the
+    oracle, for a K that is not a multiple of the 512-column stage and the three epilogues."""
+    d_in, heads, d, theta = 896, 6, 64, 500000.0
+    x = W.normal(61, (T, d_in))
+    w = W.normal(62, (heads * d, d_in), std=d_in ** -0.5)
+    pos = np.arange(T) * 7 + 3
+    cos, sin = _tables(oracle, pos, d, theta)
+    plain = oracle.linear(x, w)
+    ref_rot = oracle.rope(plain.reshape(T, heads, d), pos, theta).reshape(T, heads * d)
+    h = W.normal(63, (T, 256), std=1.0)
+    ws = [W.normal(64, (384, 256), std=256 ** -0.5), W.normal(65, (640, 384), std=384 ** -0.5),
+          W.normal(66, (640, 384), std=384 ** -0.5), W.normal(67, (256, 640), std=640 ** -0.5)]
+    ref_q = oracle.augq(h, *ws)
+    for on in (False, True):
+        tensor_gemm(on)
+        y = api.diffqkv_project(W.to_torch(x, "cuda"), W.to_torch(w, "cuda"))
+        yr = api.diffqkv_project(W.to_torch(x, "cuda"), W.to_torch(w, "cuda"), d, cos, sin)
+        q = api.diffqkv_augq(W.to_torch(h, "cuda"), *(W.to_torch(a, "cuda") for a in ws))
+        torch.cuda.synchronize()
+        _check(y.float().cpu().numpy().astype(np.float64), plain, f"plain, tensor_gemm={on}")
+        _check(yr.float().cpu().numpy().astype(np.float64), ref_rot, f"rotated, tensor_gemm={on}")
+        _check(q.float().cpu().numpy().astype(np.float64), ref_q, f"aug-Q, tensor_gemm={on}")
 
 
 def test_rotation_at_position_zero_is_the_plain_projection(api, oracle):
