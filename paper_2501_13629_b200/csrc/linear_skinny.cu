@@ -10,12 +10,17 @@
 //              rotary: channels c .. c + 7 of a head and their partners c + d/2 ..), times a pass of 16 rows of x.
 //              Items are dealt round-robin to one persistent block per SM, passes of an item back to back (the
 //              second pass finds the weight rows in L2).
-//   producer   one warp; a stage is 512 columns of K: two 8-row weight boxes (8 KB each) and a 16-row box of x
-//              (16 KB, from L2), TMA with 128-byte swizzle into a ring of 6 stages, bounded waits
+//   producer   one warp; a stage is 512 columns of K: two 8-row weight boxes (8 KB each) and a box of x (8 or 16 rows,
+//              from L2), TMA with 128-byte swizzle into a ring of 4 or 3 stages, bounded waits.  The weights do not
+//              depend on the grid before this one, so the first ring-full of weight boxes is requested before the
+//              grid-dependency wait and only the x boxes after it.
 //   consumers  8 warps; a stage has 32 steps of 16 columns, warp w takes steps w, w + 8, ...: ldmatrix of the weight
-//              rows (A, 16 x 16) and of the x rows (B, 16 columns x 16 rows), two mma.sync.m16n8k16 into fp32
-//              accumulators; at the end of an item the eight partial sums meet in shared memory and warp 0 applies
-//              the epilogue: rows g and g + 8 of the accumulator tile, i.e. the two groups, sit in the same thread.
+//              rows (A, 16 x 16) and of the x rows (B, 16 columns x 8 or 16 rows), mma.sync.m16n8k16 into fp32
+//              accumulators; at the end of an item the eight partial sums go to shared memory
+//   epilogue   one warp adds them and applies the epilogue (rows g and g + 8 of the accumulator tile, i.e. the two
+//              groups, sit in the same thread) while the consumers are already in the next item.
+// A block takes half an SM's shared memory: two blocks per SM stream side by side, and the blocks of the next grid in
+// the stream (programmatic launch) move in and request their weights while this grid's last blocks finish.
 // HBM-bound by design (2 flops per weight byte and row of x), hence mma.sync and not tcgen05.
 #include <cuda.h>
 
@@ -28,14 +33,13 @@ namespace {
 
 constexpr int kKC = 512;                  // columns of K per stage
 constexpr int kChunks = kKC / 64;         // 64-column chunks (128 bytes) per stage
-constexpr int kSkStages = 6;
 constexpr int kSkWarps = 8;               // consumer warps
-constexpr int kSkThreads = (kSkWarps + 1) * 32;
+constexpr int kSkThreads = (kSkWarps + 2) * 32;  // + producer warp + epilogue warp
 constexpr int kWBox = kChunks * 8 * 128;  // one 8-row weight box
-constexpr int kXBox = kChunks * 16 * 128; // the 16-row box of x
-constexpr int kStageBytes = 2 * kWBox + kXBox;
-constexpr int kRedBytes = 2 * kSkWarps * 32 * 8 * 4;
-constexpr int kSkSmem = 1024 + kSkStages * kStageBytes + kRedBytes + 256;
+constexpr int kRingBytes = 96 * 1024;     // 4 stages with 8 rows of x, 3 with 16
+constexpr int kRedBytes = kSkWarps * 32 * 8 * 4;
+constexpr int kSkSmem = 1024 + kRingBytes + kRedBytes + 256;
+constexpr int kBarThreads = (kSkWarps + 1) * 32;  // consumers + epilogue warp on the two named barriers
 
 enum { kPlain = 0, kGateUp = 1, kRotary = 2 };
 
@@ -62,20 +66,25 @@ __device__ __forceinline__ void item_rows(const SkinnyParams& p, int item, int& 
   }
 }
 
-__global__ void __launch_bounds__(kSkThreads, 1)
+template <int XROWS>  // rows of x per pass: 8 or 16
+__global__ void __launch_bounds__(kSkThreads, 2)
 linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_wa,
                      const __grid_constant__ CUtensorMap tmap_wb, const SkinnyParams p) {
+  constexpr int kXBox = kChunks * XROWS * 128;
+  constexpr int kStageBytes = 2 * kWBox + kXBox;
+  constexpr int kStages = kRingBytes / kStageBytes;
+  constexpr int NB = XROWS / 8;  // 8-row blocks of x = N blocks of the MMA
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  float* red = reinterpret_cast<float*>(smem + kSkStages * kStageBytes);  // [2][warp][lane][8]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSkStages * kStageBytes + kRedBytes);  // full[s], empty[s]
-  volatile int* abort_flag = reinterpret_cast<int*>(bars + 2 * kSkStages);
+  float* red = reinterpret_cast<float*>(smem + kRingBytes);  // [warp][lane][8]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kRingBytes + kRedBytes);  // full[s], empty[s]
+  volatile int* abort_flag = reinterpret_cast<int*>(bars + 2 * kStages);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t full0 = ptx::smem_u32(bars), empty0 = ptx::smem_u32(bars + kSkStages);
+  const uint32_t full0 = ptx::smem_u32(bars), empty0 = ptx::smem_u32(bars + kStages);
   if (tid == 0) {
     *abort_flag = 0;
-    for (int s = 0; s < kSkStages; ++s) {
+    for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(full0 + 8 * s, 1);
       ptx::mbar_init(empty0 + 8 * s, kSkWarps);
     }
@@ -86,7 +95,6 @@ linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   }
   __syncthreads();
   ptx::grid_launch_dependents();
-  ptx::grid_dependency_wait();  // x may be the output of the grid before this one
 
   const int total = p.items * p.passes;
   const int n_chunks = (p.K + kKC - 1) / kKC;  // stages per item (columns past K read as zero)
@@ -98,31 +106,92 @@ linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
       int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int it = blockIdx.x; it < total && ok; it += gridDim.x) {
+      // the (item, chunk) sequence of this block, walked twice: `w` requests weight boxes, `x` the boxes of x
+      struct Walk { int it, c; };
+      Walk w = {(int)blockIdx.x, 0}, x = w;
+      auto step = [&](Walk& k) { if (++k.c == n_chunks) { k.c = 0; k.it += gridDim.x; } };
+      auto load_w = [&](const Walk& k, int st) {
         int row_a, row_b;
-        item_rows(p, it / p.passes, row_a, row_b);
-        const int xrow = 16 * (it % p.passes);
-        for (int c = 0; c < n_chunks; ++c) {
-          if (issued >= kSkStages && !ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) {
-            report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
-            ok = false;
-            break;
-          }
-          const uint32_t bar = full0 + 8 * stage, dst = smem_u32 + stage * kStageBytes;
-          ptx::mbar_arrive_expect_tx(bar, kStageBytes);
-          ptx::tma_load_3d(dst, &tmap_wa, bar, 0, row_a, c * kChunks);
-          ptx::tma_load_3d(dst + kWBox, &tmap_wb, bar, 0, row_b, c * kChunks);
-          ptx::tma_load_3d(dst + 2 * kWBox, &tmap_x, bar, 0, xrow, c * kChunks);
-          ++issued;
-          if (++stage == kSkStages) { stage = 0; phase ^= 1; }
+        item_rows(p, k.it / p.passes, row_a, row_b);
+        const uint32_t bar = full0 + 8 * st, dst = smem_u32 + st * kStageBytes;
+        ptx::mbar_arrive_expect_tx(bar, kStageBytes);
+        ptx::tma_load_3d(dst, &tmap_wa, bar, 0, row_a, k.c * kChunks);
+        ptx::tma_load_3d(dst + kWBox, &tmap_wb, bar, 0, row_b, k.c * kChunks);
+      };
+      auto load_x = [&](const Walk& k, int st) {
+        ptx::tma_load_3d(smem_u32 + st * kStageBytes + 2 * kWBox, &tmap_x, full0 + 8 * st, 0, XROWS * (k.it % p.passes),
+                         k.c * kChunks);
+      };
+      int ahead = 0;  // stages whose weights are requested but whose x is not
+      for (; ahead < kStages && w.it < total; ++ahead, step(w)) load_w(w, ahead);
+      ptx::grid_dependency_wait();  // x may be the output of the grid before this one
+      for (int s = 0; s < ahead; ++s, step(x)) load_x(x, s);
+      issued = ahead;
+      stage = ahead % kStages;
+      phase = ahead == kStages ? 1 : 0;
+      for (; w.it < total; step(w), step(x)) {
+        if (!ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) {
+          report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+          ok = false;
+          break;
         }
+        load_w(w, stage);
+        load_x(x, stage);
+        ++issued;
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
       if (!ok) {  // give copies in flight a bounded chance to land before the block's shared memory is released
-        for (int s = 0; s < min(issued, kSkStages); ++s) {
-          const int uses = (issued - s + kSkStages - 1) / kSkStages;
+        for (int s = 0; s < min(issued, kStages); ++s) {
+          const int uses = (issued - s + kStages - 1) / kStages;
           ptx::mbar_wait(full0 + 8 * s, (uint32_t)(uses - 1) & 1u, nullptr);
         }
       }
+    }
+    return;
+  }
+  ptx::grid_dependency_wait();
+
+  if (warp == kSkWarps + 1) {
+    // ------------------------------------------------------------------ epilogue warp
+    const int g8 = lane >> 2, t4 = lane & 3;
+    for (int it = blockIdx.x; it < total; it += gridDim.x) {
+      asm volatile("bar.sync 1, %0;" ::"n"(kBarThreads) : "memory");  // the item's partial sums are in place
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = 0.f;
+#pragma unroll
+      for (int w = 0; w < kSkWarps; ++w) {
+        const float4* src = reinterpret_cast<const float4*>(red + (w * 32 + lane) * 8);
+        const float4 lo = src[0], hi = src[1];
+        v[0] += lo.x; v[1] += lo.y; v[2] += lo.z; v[3] += lo.w;
+        v[4] += hi.x; v[5] += hi.y; v[6] += hi.z; v[7] += hi.w;
+      }
+      asm volatile("bar.arrive 2, %0;" ::"n"(kBarThreads) : "memory");  // the buffer may be written again
+      if (*abort_flag) continue;
+      int row_a, row_b;
+      item_rows(p, it / p.passes, row_a, row_b);
+      // thread: weight rows g8 of either group, rows 2 t4 and 2 t4 + 1 of x in each 8-row block of the pass
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int t = XROWS * (it % p.passes) + 8 * nb + 2 * t4 + e;
+          if (t >= p.M) continue;
+          const float ca = v[4 * nb + e], cb = v[4 * nb + 2 + e];
+          __nv_bfloat16* crow = p.C + (long long)t * p.ldc;
+          if (p.mode == kGateUp) {
+            crow[row_a + g8] = __float2bfloat16_rn(ca / (1.f + __expf(-ca)) * cb);
+          } else if (p.mode == kRotary) {
+            const int half = p.head_dim >> 1;
+            const long long ti = (long long)t * half + (row_a % p.head_dim) + g8;
+            const float cs = p.rope_cos[ti], sn = p.rope_sin[ti];
+            crow[row_a + g8] = __float2bfloat16_rn(ca * cs - cb * sn);
+            crow[row_b + g8] = __float2bfloat16_rn(cb * cs + ca * sn);
+          } else {
+            crow[row_a + g8] = __float2bfloat16_rn(ca);
+            crow[row_b + g8] = __float2bfloat16_rn(cb);
+          }
+        }
     }
     return;
   }
@@ -130,9 +199,10 @@ linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
   // -------------------------------------------------------------------- consumers
   const int mi = lane >> 3, rr = lane & 7;
   // A (weights): matrices (rows 0-7, k 0-7), (rows 8-15, k 0-7), (rows 0-7, k 8-15), (rows 8-15, k 8-15); rows 8-15
-  // are the second box.  B (x): matrices (rows 0-7, k 0-7), (rows 0-7, k 8-15), (rows 8-15, k 0-7), (rows 8-15, k 8-15).
+  // are the second box.  B (x): matrices (rows 0-7, k 0-7), (rows 0-7, k 8-15), (rows 8-15, k 0-7), (rows 8-15, k 8-15);
+  // with 8 rows of x the last two repeat the first two and are not used.
   const uint32_t a_base = (mi & 1) * kWBox + rr * 128, a_half = mi >> 1;
-  const int xr = (mi >> 1) * 8 + rr;
+  const int xr = (NB == 2 ? (mi >> 1) * 8 : 0) + rr;
   const uint32_t b_base = 2 * kWBox + xr * 128, b_half = mi & 1;
   int stage = 0, n_item = 0;
   uint32_t phase = 0;
@@ -156,59 +226,23 @@ linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           const uint32_t chunk = s >> 2, unit = (s & 3) * 2;
           uint32_t a[4], b[4];
           ptx::ldmatrix_x4(st + a_base + chunk * 1024 + (((unit + a_half) ^ rr) << 4), a);
-          ptx::ldmatrix_x4(st + b_base + chunk * 2048 + (((unit + b_half) ^ rr) << 4), b);
+          ptx::ldmatrix_x4(st + b_base + chunk * (XROWS * 128) + (((unit + b_half) ^ rr) << 4), b);
           ptx::mma_bf16_16816(acc[0], a, b[0], b[1]);
-          ptx::mma_bf16_16816(acc[1], a, b[2], b[3]);
+          if (NB == 2) ptx::mma_bf16_16816(acc[1], a, b[2], b[3]);
         }
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(empty0 + 8 * stage);
-      if (++stage == kSkStages) { stage = 0; phase ^= 1; }
+      if (++stage == kStages) { stage = 0; phase ^= 1; }
     }
-    // ---- the eight partial sums meet; warp 0 finishes the item
-    float* buf = red + (n_item & 1) * (kSkWarps * 32 * 8);
-    float4* mine = reinterpret_cast<float4*>(buf + (warp * 32 + lane) * 8);
+    // ---- the eight partial sums go to the epilogue warp
+    if (n_item > 0) asm volatile("bar.sync 2, %0;" ::"n"(kBarThreads) : "memory");  // it has read the previous ones
+    float4* mine = reinterpret_cast<float4*>(red + (warp * 32 + lane) * 8);
     mine[0] = make_float4(acc[0][0], acc[0][1], acc[0][2], acc[0][3]);
     mine[1] = make_float4(acc[1][0], acc[1][1], acc[1][2], acc[1][3]);
-    asm volatile("bar.sync 1, %0;" ::"n"(kSkWarps * 32) : "memory");
-    if (warp == 0 && !dead) {
-      float v[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) v[e] = 0.f;
-#pragma unroll
-      for (int w = 0; w < kSkWarps; ++w) {
-        const float4* src = reinterpret_cast<const float4*>(buf + (w * 32 + lane) * 8);
-        const float4 lo = src[0], hi = src[1];
-        v[0] += lo.x; v[1] += lo.y; v[2] += lo.z; v[3] += lo.w;
-        v[4] += hi.x; v[5] += hi.y; v[6] += hi.z; v[7] += hi.w;
-      }
-      int row_a, row_b;
-      item_rows(p, it / p.passes, row_a, row_b);
-      const int g8 = lane >> 2, t4 = lane & 3;
-      // thread: weight rows g8 of either group, rows 2 t4 and 2 t4 + 1 of x in each 8-row half of the pass
-#pragma unroll
-      for (int nb = 0; nb < 2; ++nb)
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int t = 16 * (it % p.passes) + 8 * nb + 2 * t4 + e;
-          if (t >= p.M) continue;
-          const float ca = v[4 * nb + e], cb = v[4 * nb + 2 + e];
-          __nv_bfloat16* crow = p.C + (long long)t * p.ldc;
-          if (p.mode == kGateUp) {
-            crow[row_a + g8] = __float2bfloat16_rn(ca / (1.f + __expf(-ca)) * cb);
-          } else if (p.mode == kRotary) {
-            const int half = p.head_dim >> 1;
-            const long long ti = (long long)t * half + (row_a % p.head_dim) + g8;
-            const float cs = p.rope_cos[ti], sn = p.rope_sin[ti];
-            crow[row_a + g8] = __float2bfloat16_rn(ca * cs - cb * sn);
-            crow[row_b + g8] = __float2bfloat16_rn(cb * cs + ca * sn);
-          } else {
-            crow[row_a + g8] = __float2bfloat16_rn(ca);
-            crow[row_b + g8] = __float2bfloat16_rn(cb);
-          }
-        }
-    }
+    asm volatile("bar.arrive 1, %0;" ::"n"(kBarThreads) : "memory");
   }
+  if (n_item > 0) asm volatile("bar.sync 2, %0;" ::"n"(kBarThreads) : "memory");  // pairs with the last arrival
 }
 
 // dims (64 columns, rows, K / 64 chunks); a box is 64 columns x box_rows rows x kChunks chunks.
@@ -230,8 +264,9 @@ bool linear_skinny_supported(long long M, int N, int K, bool dual, int head_dim,
 cudaError_t launch_linear_skinny(const void* A, const void* B0, const void* B1, void* C, long long M, int N, int K,
                                  int* dev_status, cudaStream_t stream, const float* rope_cos, const float* rope_sin,
                                  int head_dim) {
+  const int xrows = M <= 8 ? 8 : 16;
   CUtensorMap mx, ma, mb;
-  if (!make_rows_map(&mx, A, M, K, 16) || !make_rows_map(&ma, B0, N, K, 8) ||
+  if (!make_rows_map(&mx, A, M, K, xrows) || !make_rows_map(&ma, B0, N, K, 8) ||
       !make_rows_map(&mb, B1 ? B1 : B0, N, K, 8))
     return cudaErrorNotSupported;
   SkinnyParams p;
@@ -240,7 +275,7 @@ cudaError_t launch_linear_skinny(const void* A, const void* B0, const void* B1, 
   p.mode = B1 ? kGateUp : (rope_cos ? kRotary : kPlain);
   p.head_dim = head_dim;
   p.items = p.mode == kGateUp ? N / 8 : N / 16;
-  p.passes = (int)((M + 15) / 16);
+  p.passes = (int)((M + xrows - 1) / xrows);
   p.rope_cos = rope_cos; p.rope_sin = rope_sin;
   p.dev_status = dev_status;
   int dev = 0, sms = 0;
@@ -248,7 +283,8 @@ cudaError_t launch_linear_skinny(const void* A, const void* B0, const void* B1, 
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return cudaErrorUnknown;
   const long long total = (long long)p.items * p.passes;
-  cudaError_t err = cudaFuncSetAttribute(linear_skinny_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSkSmem);
+  auto kernel = xrows == 8 ? linear_skinny_kernel<8> : linear_skinny_kernel<16>;
+  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSkSmem);
   if (err != cudaSuccess) return err;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -257,10 +293,10 @@ cudaError_t launch_linear_skinny(const void* A, const void* B0, const void* B1, 
   cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cfg.gridDim = dim3((unsigned)(total < sms ? total : sms));
+  cfg.gridDim = dim3((unsigned)(total < 2 * sms ? total : 2 * sms));  // two blocks per SM
   cfg.blockDim = dim3(kSkThreads);
   cfg.dynamicSmemBytes = kSkSmem;
-  err = cudaLaunchKernelEx(&cfg, linear_skinny_kernel, mx, ma, mb, p);
+  err = cudaLaunchKernelEx(&cfg, kernel, mx, ma, mb, p);
   if (err != cudaSuccess) return err;
   count_launch();
   return cudaGetLastError();
