@@ -330,6 +330,46 @@ def time_prefill(api, W, device, peaks, steps):
     return res
 
 
+def time_augq_decode(api, W, device, steps):
+    """The augmented-Q projection of one decode step (config 4's widths, one row per sequence): three launches that
+    stream the 92 MB of weights; four weight sets are rotated so that none is found in L2."""
+    import torch
+    cfg = W.CFG4
+    d_q0 = cfg.n_q * cfg.d_qk
+    g = torch.Generator(device=device)
+    g.manual_seed(cfg.seed + 7)
+
+    def rn(*shape, std=1.0):
+        return (torch.randn(shape, generator=g, device=device) * std).to(torch.bfloat16)
+
+    sets = [(rn(d_q0, cfg.d_model, std=cfg.d_model ** -0.5), rn(cfg.d_aug, d_q0, std=d_q0 ** -0.5),
+             rn(cfg.d_aug, d_q0, std=d_q0 ** -0.5), rn(d_q0, cfg.d_aug, std=cfg.d_aug ** -0.5)) for _ in range(4)]
+    wbytes = float(sum(w.numel() * 2 for w in sets[0]))
+    res = {"weight_bytes": wbytes, "rows": {}}
+    for T in (4, 16, 64):
+        h = rn(T, cfg.d_model, std=cfg.h_std)
+        ws = torch.empty(max(api.diffqkv_augq_workspace_bytes(T, d_q0, cfg.d_aug), 256), dtype=torch.uint8, device=device)
+        q = torch.empty(T, d_q0, dtype=torch.bfloat16, device=device)
+        i = [0]
+
+        def step():
+            api.diffqkv_augq(h, *sets[i[0] % 4], workspace=ws, q_out=q)
+            i[0] += 1
+
+        for _ in range(10):
+            step()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            step()
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / steps
+        res["rows"][str(T)] = {"us_per_step": ms * 1e3, "weights_GB/s": wbytes / ms / 1e6}
+    return res
+
+
 def time_sigma_table(api, W, device, steps):
     """The paper's own efficiency experiment in shape: SIGMA-1.5B attention heads (32 query, 4 K, 16 V heads, head
     dimension 64) against the standard model's 16 K / 16 V heads at prefix lengths 2k, 4k, 16k and 32k (batch 8,
@@ -518,6 +558,8 @@ def run_ours(args):
             del c5
             torch.cuda.empty_cache()
             others[W.CFG4.name] = time_prefill(api, W, device, peaks, max(5, min(args.steps, 20)))
+            torch.cuda.empty_cache()
+            others["augq_at_decode"] = time_augq_decode(api, W, device, 200)
             torch.cuda.empty_cache()
             others["sigma1p5b_vs_std_heads"] = time_sigma_table(api, W, device, max(20, min(args.steps, 300)))
             torch.cuda.empty_cache()
