@@ -494,6 +494,11 @@ def run_ours(args):
 
     cfg = W.CFG3
     host = W.make_decode_inputs(cfg)
+    if args.workload == "augq_decode":  # the projection chain at decode row counts alone (the command profilers wrap)
+        if rank == 0:
+            print(json.dumps({"workload": "cfg4 widths, 4 / 16 / 64 rows",
+                              **time_augq_decode(api, W, device, max(1, min(args.steps, 200)))}))
+        return
     if args.workload == "topk":  # selective V fetching on the headline workload alone (the command profilers wrap)
         if rank == 0:
             print(json.dumps({"workload": cfg.name + " top-100 / top-1024",
@@ -669,9 +674,10 @@ def main():
     ap.add_argument("--quick", action="store_true", help="headline workload only")
     ap.add_argument("--budget-s", type=float, default=150.0,
                     help="--impl reference: seconds of oracle time the whole run may take (sizes the per-step sample)")
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "topk"],
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "topk", "augq_decode"],
                     help="decode = the headline line (default); prefill = only the config 4 timings; "
-                         "topk = only selective V fetching on the headline workload")
+                         "topk = only selective V fetching on the headline workload; augq_decode = only the projection "
+                         "chain at decode row counts")
     ap.add_argument("--profile", action="store_true",
                     help="only the timed loop of the headline workload (the command profilers wrap)")
     args = ap.parse_args()
