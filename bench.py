@@ -385,6 +385,71 @@ def time_augq_decode(api, W, device, steps):
     return res
 
 
+def time_decode_step(api, W, device, host, steps):
+    """One decode step of the whole attention block on the headline shape (config 3: batch 4, 32/4/8 heads, d 128,
+    32768 cached tokens; hidden 2048 and the aug-Q widths of config 4): q = rope(aug-Q(h)), k = rope(h W_K^T),
+    v = h W_V^T, append k and v as token 32767, attention over the 32768 tokens.  Weights and caches are rotated
+    out of L2; every product runs in this library's kernels."""
+    import dataclasses
+    import torch
+    cfg, c4 = host.cfg, W.CFG4
+    case = DecodeCase(api, cfg, device, host_inputs=host)
+    d_q0 = cfg.n_q * cfg.d_qk
+    g = torch.Generator(device=device)
+    g.manual_seed(cfg.seed + 11)
+
+    def rn(*shape, std=1.0):
+        return (torch.randn(shape, generator=g, device=device) * std).to(torch.bfloat16)
+
+    sets = [(rn(d_q0, c4.d_model, std=c4.d_model ** -0.5), rn(c4.d_aug, d_q0, std=d_q0 ** -0.5),
+             rn(c4.d_aug, d_q0, std=d_q0 ** -0.5), rn(d_q0, c4.d_aug, std=c4.d_aug ** -0.5),
+             rn(cfg.n_k * cfg.d_qk, c4.d_model, std=c4.d_model ** -0.5),
+             rn(cfg.n_v * cfg.d_v, c4.d_model, std=c4.d_model ** -0.5)) for _ in range(4)]
+    T = cfg.batch
+    h = rn(T, c4.d_model, std=c4.h_std)
+    pos = torch.full((T,), cfg.kv_len - 1, device=device, dtype=torch.float64)
+    inv = torch.pow(torch.tensor(50000.0, dtype=torch.float64, device=device),
+                    -2.0 * torch.arange(cfg.d_qk // 2, device=device, dtype=torch.float64) / cfg.d_qk)
+    ang = pos[:, None] * inv[None, :]
+    cos, sin = torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()
+    ws = torch.empty(max(api.diffqkv_augq_workspace_bytes(T, d_q0, c4.d_aug), 256), dtype=torch.uint8, device=device)
+    q = torch.empty(T, d_q0, dtype=torch.bfloat16, device=device)
+    k_new = torch.empty(T, cfg.n_k * cfg.d_qk, dtype=torch.bfloat16, device=device)
+    v_new = torch.empty(T, cfg.n_v * cfg.d_v, dtype=torch.bfloat16, device=device)
+    before = torch.from_numpy(case.seqlens_host - 1).to(device)  # the new token becomes the last cached one
+    appends = [dataclasses.replace(c, seqlens=before) for c in case.caches]
+    i = [0]
+
+    def step():
+        w_q, w_g, w_u, w_d, w_k, w_v = sets[i[0] % 4]
+        r = i[0] % case.rotate
+        i[0] += 1
+        api.diffqkv_augq_rope(h, w_q, w_g, w_u, w_d, cfg.d_qk, cos, sin, workspace=ws, q_out=q, dev_status=case.status)
+        api.diffqkv_project(h, w_k, cfg.d_qk, cos, sin, out=k_new, dev_status=case.status)
+        api.diffqkv_project(h, w_v, out=v_new, dev_status=case.status)
+        api.diffqkv_cache_append(k_new.view(T, 1, cfg.n_k, cfg.d_qk), v_new.view(T, 1, cfg.n_v, cfg.d_v), appends[r],
+                                 dev_status=case.status)
+        api.diffqkv_decode(q.view(T, cfg.n_q, cfg.d_qk), case.caches[r], cfg.n_k, cfg.n_v, cfg.scale,
+                           workspace=case.workspace, out=case.out, dev_status=case.status)
+
+    for _ in range(10):
+        step()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = api.launch_count()
+    a.record()
+    for _ in range(steps):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    assert int(case.status.item()) == 0, "device status reported an error"
+    ms = a.elapsed_time(b) / steps
+    wbytes = float(sum(w.numel() * 2 for w in sets[0]))
+    return {"us_per_step": ms * 1e3, "kernels_per_step": (api.launch_count() - l0) // steps,
+            "weight_bytes": wbytes, "kv_bytes": case.bytes, "GB/s": (wbytes + case.bytes) / ms / 1e6,
+            "tokens_per_s_per_layer": cfg.batch / (ms * 1e-3)}
+
+
 def time_sigma_table(api, W, device, steps):
     """The paper's own efficiency experiment in shape: SIGMA-1.5B attention heads (32 query, 4 K, 16 V heads, head
     dimension 64) against the standard model's 16 K / 16 V heads at prefix lengths 2k, 4k, 16k and 32k (batch 8,
@@ -580,6 +645,7 @@ def run_ours(args):
             others[W.CFG4.name] = time_prefill(api, W, device, peaks, max(5, min(args.steps, 20)))
             torch.cuda.empty_cache()
             others["augq_at_decode"] = time_augq_decode(api, W, device, 200)
+            others["decode_step_cfg3"] = time_decode_step(api, W, device, host, 200)
             torch.cuda.empty_cache()
             others["sigma1p5b_vs_std_heads"] = time_sigma_table(api, W, device, max(20, min(args.steps, 300)))
             torch.cuda.empty_cache()
