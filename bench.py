@@ -387,8 +387,8 @@ def time_augq_decode(api, W, device, steps):
 
 def time_decode_step(api, W, device, host, steps):
     """One decode step of the whole attention block on the headline shape (config 3: batch 4, 32/4/8 heads, d 128,
-    32768 cached tokens; hidden 2048 and the aug-Q widths of config 4): q = rope(aug-Q(h)), k = rope(h W_K^T),
-    v = h W_V^T, append k and v as token 32767, attention over the 32768 tokens.  Weights and caches are rotated
+    32768 cached tokens; hidden 2048 and the aug-Q widths of config 4): diffqkv_decode_frontend (q = rope(aug-Q(h)),
+    k = rope(h W_K^T) and v = h W_V^T written into the cache as token 32767), then diffqkv_decode over the 32768 tokens.  Weights and caches are rotated
     out of L2; every product runs in this library's kernels."""
     import dataclasses
     import torch
@@ -412,10 +412,8 @@ def time_decode_step(api, W, device, host, steps):
                     -2.0 * torch.arange(cfg.d_qk // 2, device=device, dtype=torch.float64) / cfg.d_qk)
     ang = pos[:, None] * inv[None, :]
     cos, sin = torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()
-    ws = torch.empty(max(api.diffqkv_augq_workspace_bytes(T, d_q0, c4.d_aug), 256), dtype=torch.uint8, device=device)
+    ws = torch.empty(1 << 22, dtype=torch.uint8, device=device)  # far more than the few rows need
     q = torch.empty(T, d_q0, dtype=torch.bfloat16, device=device)
-    k_new = torch.empty(T, cfg.n_k * cfg.d_qk, dtype=torch.bfloat16, device=device)
-    v_new = torch.empty(T, cfg.n_v * cfg.d_v, dtype=torch.bfloat16, device=device)
     before = torch.from_numpy(case.seqlens_host - 1).to(device)  # the new token becomes the last cached one
     appends = [dataclasses.replace(c, seqlens=before) for c in case.caches]
     i = [0]
@@ -424,11 +422,8 @@ def time_decode_step(api, W, device, host, steps):
         w_q, w_g, w_u, w_d, w_k, w_v = sets[i[0] % 4]
         r = i[0] % case.rotate
         i[0] += 1
-        api.diffqkv_augq_rope(h, w_q, w_g, w_u, w_d, cfg.d_qk, cos, sin, workspace=ws, q_out=q, dev_status=case.status)
-        api.diffqkv_project(h, w_k, cfg.d_qk, cos, sin, out=k_new, dev_status=case.status)
-        api.diffqkv_project(h, w_v, out=v_new, dev_status=case.status)
-        api.diffqkv_cache_append(k_new.view(T, 1, cfg.n_k, cfg.d_qk), v_new.view(T, 1, cfg.n_v, cfg.d_v), appends[r],
-                                 dev_status=case.status)
+        api.diffqkv_decode_frontend(h, w_q, w_g, w_u, w_d, w_k, w_v, appends[r], cfg.n_q, cfg.d_qk, cfg.d_v, cos, sin,
+                                    workspace=ws, q_out=q.view(T, cfg.n_q, cfg.d_qk), dev_status=case.status)
         api.diffqkv_decode(q.view(T, cfg.n_q, cfg.d_qk), case.caches[r], cfg.n_k, cfg.n_v, cfg.scale,
                            workspace=case.workspace, out=case.out, dev_status=case.status)
 

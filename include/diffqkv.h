@@ -236,6 +236,32 @@ diffqkv_status diffqkv_cache_append(const void *k_new, const void *v_new, int32_
                                     const diffqkv_shape *shape, int32_t *dev_status, void *stream);
 
 /*
+ * diffqkv_decode_frontend -- everything one decode step computes from the hidden states before it attends
+ * (appendix attention listing: q_proj and the augmented-Q chain, k_proj, v_proj, rotary embedding, cache update), for
+ * one new token per sequence:
+ *     q_out[b] = rope(aug-Q(h[b]))                      as diffqkv_augq_rope with T = batch rows
+ *     K cache row at position seqlens[b]  = rope(h[b] W_K^T)     V cache row at seqlens[b] = h[b] W_V^T
+ *   h [batch, d_model] bf16; W_Q [n_q d_qk, d_model], W_gate, W_up [d_aug, n_q d_qk], W_down [n_q d_qk, d_aug],
+ *   W_K [n_k d_qk, d_model], W_V [n_v d_v, d_model], all bf16 in the nn.Linear layout
+ *   cos, sin   [batch, d_qk / 2] fp32 tables of the new tokens' positions, or both NULL for no rotation
+ *   cache      bf16 pools; seqlens[b] = tokens already cached; seqlens is not modified (the caller adds 1 and calls
+ *              diffqkv_decode with q_out); positions at or past max_seqlen and page ids outside the pool are
+ *              reported as DIFFQKV_ERR_INDEX in *dev_status and skipped
+ *   workspace  diffqkv_decode_frontend_workspace_bytes(shape, d_aug) bytes, 256-byte aligned
+ *   q_out      [batch, n_q, d_qk] bf16
+ * With at most 64 sequences this is three launches (the products of h share one, which writes k and v straight into
+ * the cache); with more it is the separate steps of diffqkv_augq_rope, diffqkv_project and diffqkv_cache_append.
+ * d_model, d_aug and n_q d_qk must be multiples of 128, n_k d_qk and n_v d_v multiples of 16 (of 128 beyond 64
+ * sequences), d_qk 64 or 128 when rotating.
+ */
+size_t diffqkv_decode_frontend_workspace_bytes(const diffqkv_shape *shape, int32_t d_aug);
+diffqkv_status diffqkv_decode_frontend(const void *h, const void *W_Q, const void *W_gate, const void *W_up,
+                                       const void *W_down, const void *W_K, const void *W_V, int32_t d_model,
+                                       int32_t d_aug, const float *cos, const float *sin, const diffqkv_cache *cache,
+                                       const diffqkv_shape *shape, void *workspace, size_t workspace_bytes,
+                                       void *q_out, int32_t *dev_status, void *stream);
+
+/*
  * diffqkv_decode_topk -- decode with selective V cache fetching (paper Section "Selective V Cache Fetching"; its
  * table uses the 100 highest scores): every query head scores all cached tokens of its K head, keeps the `topk`
  * highest scores (equal scores: the earlier token), takes the softmax over the kept scores only (the paper does

@@ -31,7 +31,8 @@ EXPORTS = (
     "diffqkv_status_string", "diffqkv_launch_count", "diffqkv_profile_split_events", "diffqkv_decode_static",
     "diffqkv_set_max_blocks", "diffqkv_topk_general_only", "diffqkv_last_decode_kernel",
     "diffqkv_last_prefill_kernel", "diffqkv_force_tensor_gemm", "diffqkv_augq_rope", "diffqkv_project", "diffqkv_cache_append",
-    "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes",
+    "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes", "diffqkv_decode_frontend",
+    "diffqkv_decode_frontend_workspace_bytes",
 )
 
 
@@ -95,6 +96,12 @@ _lib.diffqkv_decode_topk.argtypes = [C.c_void_p, C.POINTER(CacheStruct), C.POINT
 _lib.diffqkv_status_string.restype = C.c_char_p
 _lib.diffqkv_status_string.argtypes = [C.c_int]
 _lib.diffqkv_launch_count.restype = C.c_int64
+_lib.diffqkv_decode_frontend_workspace_bytes.restype = C.c_size_t
+_lib.diffqkv_decode_frontend_workspace_bytes.argtypes = [C.POINTER(ShapeStruct), C.c_int32]
+_lib.diffqkv_decode_frontend.restype = C.c_int32
+_lib.diffqkv_decode_frontend.argtypes = [C.c_void_p] * 7 + [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                         C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_void_p, C.c_size_t,
+                                         C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.diffqkv_force_tensor_gemm.restype = None
 _lib.diffqkv_force_tensor_gemm.argtypes = [C.c_int32]
 _lib.diffqkv_last_prefill_kernel.restype = C.c_int32
@@ -369,6 +376,36 @@ def diffqkv_project(x: torch.Tensor, W: torch.Tensor, head_dim: int = 0, cos: Op
     if st != OK:
         raise DiffQKVError(st, "diffqkv_project")
     return out
+
+
+def diffqkv_decode_frontend(h: torch.Tensor, W_Q: torch.Tensor, W_gate: torch.Tensor, W_up: torch.Tensor,
+                            W_down: torch.Tensor, W_K: torch.Tensor, W_V: torch.Tensor, cache: KVCache, n_q: int,
+                            d_qk: int, d_v: int, cos: Optional[torch.Tensor] = None,
+                            sin: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                            q_out: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                            stream: Optional[torch.cuda.Stream] = None):
+    """One decode step's projections: returns q [batch, n_q, d_qk] = rope(aug-Q(h)) and writes the new token's
+    k = rope(h W_K^T), v = h W_V^T into the cache at position seqlens[b] (seqlens is left as it is)."""
+    batch, d_model = h.shape
+    d_aug = W_gate.shape[0]
+    n_k, n_v = W_K.shape[0] // d_qk, W_V.shape[0] // d_v
+    assert W_Q.shape[0] == n_q * d_qk
+    if cos is not None:
+        assert cos.dtype == torch.float32 and sin.dtype == torch.float32 and cos.is_contiguous() and sin.is_contiguous()
+        assert tuple(cos.shape) == (batch, d_qk // 2) and tuple(sin.shape) == (batch, d_qk // 2)
+    shape = make_shape(batch, n_q, n_k, n_v, d_qk, d_v, h.dtype, h.dtype, 1.0)
+    if workspace is None:
+        nbytes = int(_lib.diffqkv_decode_frontend_workspace_bytes(C.byref(shape), d_aug))
+        workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=h.device)
+    if q_out is None:
+        q_out = torch.empty((batch, n_q, d_qk), dtype=torch.bfloat16, device=h.device)
+    cs = cache.c_struct()
+    st = _lib.diffqkv_decode_frontend(_p(h), _p(W_Q), _p(W_gate), _p(W_up), _p(W_down), _p(W_K), _p(W_V), d_model, d_aug,
+                                      _p(cos), _p(sin), C.byref(cs), C.byref(shape), _p(workspace), workspace.numel(),
+                                      _p(q_out), _p(dev_status), _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_decode_frontend")
+    return q_out
 
 
 def diffqkv_cache_append(k_new: torch.Tensor, v_new: torch.Tensor, cache: KVCache,

@@ -290,6 +290,41 @@ diffqkv_status diffqkv_augq_rope(const void* h, const void* W_Q, const void* W_g
   return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
 
+size_t diffqkv_decode_frontend_workspace_bytes(const diffqkv_shape* shape, int32_t d_aug) {
+  if (!shape || check_shape(shape) != DIFFQKV_OK || d_aug <= 0) return 0;
+  return decode_frontend_workspace_bytes(*shape, d_aug);
+}
+
+diffqkv_status diffqkv_decode_frontend(const void* h, const void* W_Q, const void* W_gate, const void* W_up,
+                                       const void* W_down, const void* W_K, const void* W_V, int32_t d_model,
+                                       int32_t d_aug, const float* cos, const float* sin, const diffqkv_cache* cache,
+                                       const diffqkv_shape* shape, void* workspace, size_t workspace_bytes, void* q_out,
+                                       int32_t* dev_status, void* stream) {
+  diffqkv_status st = check_shape(shape);
+  if (st != DIFFQKV_OK) return st;
+  if (!h || !W_Q || !W_gate || !W_up || !W_down || !W_K || !W_V || !q_out) return DIFFQKV_ERR_INVALID_ARG;
+  if (d_model <= 0 || d_aug <= 0) return DIFFQKV_ERR_INVALID_ARG;
+  if (shape->dtype != DIFFQKV_BF16) return DIFFQKV_ERR_UNSUPPORTED;
+  st = check_cache(cache, shape);
+  if (st != DIFFQKV_OK) return st;
+  const int d_q0 = shape->n_q * shape->d_qk;
+  if (d_model % 128 != 0 || d_aug % 128 != 0 || d_q0 % 128 != 0) return DIFFQKV_ERR_UNSUPPORTED;
+  if ((shape->n_k * shape->d_qk) % 16 != 0 || (shape->n_v * shape->d_v) % 16 != 0) return DIFFQKV_ERR_UNSUPPORTED;
+  const diffqkv_status rs = check_rope(cos, sin, shape->d_qk, d_q0);
+  if (rs != DIFFQKV_OK) return rs;
+  const void* ptrs[8] = {h, W_Q, W_gate, W_up, W_down, W_K, W_V, q_out};
+  for (const void* ptr : ptrs)
+    if (!aligned16(ptr)) return DIFFQKV_ERR_ALIGNMENT;
+  if (shape->batch == 0) return DIFFQKV_OK;
+  if (!workspace || workspace_bytes < decode_frontend_workspace_bytes(*shape, d_aug)) return DIFFQKV_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DIFFQKV_ERR_ALIGNMENT;
+  const cudaError_t err = launch_decode_frontend(h, W_Q, W_gate, W_up, W_down, W_K, W_V, d_model, d_aug, cos, sin,
+                                                 *cache, view_of(cache), *shape, workspace, q_out, dev_status,
+                                                 static_cast<cudaStream_t>(stream));
+  if (err == cudaErrorNotSupported) return DIFFQKV_ERR_UNSUPPORTED;
+  return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
+}
+
 diffqkv_status diffqkv_augq(const void* h, const void* W_Q, const void* W_gate, const void* W_up, const void* W_down,
                             int64_t T, int32_t d_model, int32_t d_q0, int32_t d_aug, int32_t d_out, void* workspace,
                             size_t workspace_bytes, void* q_out, int32_t* dev_status, void* stream) {

@@ -342,6 +342,46 @@ cudaError_t launch_augq(const void* h, const void* W_Q, const void* W_gate, cons
   return launch_gemm(a, W_down, nullptr, q_out, T, d_out, d_aug, dev_status, stream, rope_cos, rope_sin, head_dim);
 }
 
+size_t decode_frontend_workspace_bytes(const diffqkv_shape& s, int d_aug) {
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  return augq_workspace_bytes(s.batch, s.n_q * s.d_qk, d_aug) + up((size_t)s.batch * s.n_k * s.d_qk * 2) +
+         up((size_t)s.batch * s.n_v * s.d_v * 2);
+}
+
+cudaError_t launch_decode_frontend(const void* h, const void* W_Q, const void* W_gate, const void* W_up,
+                                   const void* W_down, const void* W_K, const void* W_V, int d_model, int d_aug,
+                                   const float* rope_cos, const float* rope_sin, const diffqkv_cache& c,
+                                   const CacheView& view, const diffqkv_shape& s, void* workspace, void* q_out,
+                                   int* dev_status, cudaStream_t stream) {
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  const long long T = s.batch;
+  const int d_q0 = s.n_q * s.d_qk, kw = s.n_k * s.d_qk, vw = s.n_v * s.d_v;
+  char* ws = reinterpret_cast<char*>(workspace);
+  void* x = ws;
+  void* a = ws + up((size_t)T * d_q0 * 2);
+  if (!g_force_tensor_gemm && T <= kSkinnyMaxRows) {
+    // three launches: {x = h W_Q^T, k and v into the cache}, a = silu(x W_gate^T) * (x W_up^T), q = rope(a W_down^T)
+    cudaError_t err = launch_qkv_skinny(h, W_Q, x, d_q0, W_K, W_V, T, d_model, rope_cos, rope_sin, view, s.n_k, s.n_v,
+                                        s.d_qk, s.d_v, dev_status, stream);
+    if (err != cudaSuccess) return err;
+    err = launch_gemm(x, W_gate, W_up, a, T, d_aug, d_q0, dev_status, stream);
+    if (err != cudaSuccess) return err;
+    return launch_gemm(a, W_down, nullptr, q_out, T, d_q0, d_aug, dev_status, stream, rope_cos, rope_sin, s.d_qk);
+  }
+  // many rows: the separate steps (tensor-core products, then the cache update)
+  if (kw % 128 != 0 || vw % 128 != 0) return cudaErrorNotSupported;
+  char* k_new = ws + augq_workspace_bytes(T, d_q0, d_aug);
+  char* v_new = k_new + up((size_t)T * kw * 2);
+  cudaError_t err = launch_augq(h, W_Q, W_gate, W_up, W_down, T, d_model, d_q0, d_aug, d_q0, workspace, q_out,
+                                dev_status, stream, rope_cos, rope_sin, s.d_qk);
+  if (err != cudaSuccess) return err;
+  err = launch_gemm(h, W_K, nullptr, k_new, T, kw, d_model, dev_status, stream, rope_cos, rope_sin, s.d_qk);
+  if (err != cudaSuccess) return err;
+  err = launch_gemm(h, W_V, nullptr, v_new, T, vw, d_model, dev_status, stream);
+  if (err != cudaSuccess) return err;
+  return launch_cache_append(k_new, v_new, 1, c, s, dev_status, stream);
+}
+
 // y[T, d_out] = x[T, d_in] . W[d_out, d_in]^T, optionally rotated per head (the K and V projections).
 cudaError_t launch_project(const void* x, const void* W, long long T, int d_in, int d_out, void* y, int* dev_status,
                            cudaStream_t stream, const float* rope_cos, const float* rope_sin, int head_dim) {

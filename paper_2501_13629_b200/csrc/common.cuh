@@ -65,6 +65,17 @@ void count_launch(int n = 1);
 // the rotate-half rotary embedding per head of head_dim channels.
 constexpr int kSkinnyMaxRows = 64;
 void set_force_tensor_gemm(int on);
+cudaError_t launch_qkv_skinny(const void* h, const void* W_Q, void* x, int d_q0, const void* W_K, const void* W_V,
+                              long long M, int K, const float* rope_cos, const float* rope_sin, const CacheView& cache,
+                              int n_k, int n_v, int d_qk, int d_v, int* dev_status, cudaStream_t stream);
+// Everything a decode step computes from the hidden states h [batch, d_model]: q_out = rope(aug-Q(h)), and the new
+// token's k = rope(h W_K^T), v = h W_V^T written into the cache at position seqlens[b] (augq.cu).
+size_t decode_frontend_workspace_bytes(const diffqkv_shape& s, int d_aug);
+cudaError_t launch_decode_frontend(const void* h, const void* W_Q, const void* W_gate, const void* W_up,
+                                   const void* W_down, const void* W_K, const void* W_V, int d_model, int d_aug,
+                                   const float* rope_cos, const float* rope_sin, const diffqkv_cache& c,
+                                   const CacheView& view, const diffqkv_shape& s, void* workspace, void* q_out,
+                                   int* dev_status, cudaStream_t stream);
 bool linear_skinny_supported(long long M, int N, int K, bool dual, int head_dim, bool rotary);
 cudaError_t launch_linear_skinny(const void* A, const void* B0, const void* B1, void* C, long long M, int N, int K,
                                  int* dev_status, cudaStream_t stream, const float* rope_cos, const float* rope_sin,

@@ -43,33 +43,80 @@ constexpr int kBarThreads = (kSkWarps + 1) * 32;  // consumers + epilogue warp o
 
 enum { kPlain = 0, kGateUp = 1, kRotary = 2 };
 
-struct SkinnyParams {
+enum { kToMatrix = 0, kToKCache = 1, kToVCache = 2 };
+
+// A launch covers up to three weight matrices that share x (and so K): a segment is a run of items on one of them.
+struct Segment {
+  int first_item, mode, head_dim;
+  int map_a, map_b;  // which of the four weight maps the two 8-row boxes come from
+  int dest;          // kToMatrix: row t of C; otherwise the cache row of sequence t at position seqlens[t]
   __nv_bfloat16* C;
-  int ldc, M, N, K;
-  int mode, head_dim;
-  int items, passes;  // items of 16 weight rows; passes of 16 rows of x
+  int ldc;
+};
+
+struct SkinnyParams {
+  Segment seg[3];
+  int n_seg;
+  int M, K;
+  int items, passes;  // items of 16 weight rows over all segments; passes of 8 or 16 rows of x
   const float* rope_cos;
   const float* rope_sin;
+  CacheView cache;    // for the cache destinations
+  int d_qk, d_v;
   int* dev_status;
 };
 
-__device__ __forceinline__ void item_rows(const SkinnyParams& p, int item, int& row_a, int& row_b) {
-  if (p.mode == kGateUp) {
-    row_a = row_b = 8 * item;
-  } else if (p.mode == kRotary) {
-    const int half = p.head_dim >> 1, per_head = half >> 3;
-    row_a = (item / per_head) * p.head_dim + 8 * (item % per_head);
+// Segment of an item and the first weight rows of its two boxes.
+__device__ __forceinline__ const Segment& item_rows(const SkinnyParams& p, int item, int& row_a, int& row_b) {
+  int si = 0;
+  if (p.n_seg > 1 && item >= p.seg[1].first_item) si = 1;
+  if (p.n_seg > 2 && item >= p.seg[2].first_item) si = 2;
+  const Segment& sg = p.seg[si];
+  const int local = item - sg.first_item;
+  if (sg.mode == kGateUp) {
+    row_a = row_b = 8 * local;
+  } else if (sg.mode == kRotary) {
+    const int half = sg.head_dim >> 1, per_head = half >> 3;
+    row_a = (local / per_head) * sg.head_dim + 8 * (local % per_head);
     row_b = row_a + half;
   } else {
-    row_a = 16 * item;
+    row_a = 16 * local;
     row_b = row_a + 8;
   }
+  return sg;
+}
+
+// Where output channel `col` of row t goes: into C, or into the cache row of sequence t at position seqlens[t]
+// (one new token per sequence; positions at or past max_seqlen and page ids outside the pool are reported and skipped).
+__device__ __forceinline__ __nv_bfloat16* dest_of(const SkinnyParams& p, const Segment& sg, int t, int col) {
+  if (sg.dest == kToMatrix) return sg.C + (long long)t * sg.ldc + col;
+  const CacheView& c = p.cache;
+  const int pos = c.seqlens[t];
+  if (pos < 0 || pos >= c.max_seqlen) {
+    report(p.dev_status, DIFFQKV_ERR_INDEX);
+    return nullptr;
+  }
+  long long blk = t, slot = pos;
+  if (c.page_table) {
+    blk = c.page_table[(long long)t * c.max_pages_per_seq + pos / c.page_size];
+    slot = pos % c.page_size;
+    if (blk < 0 || blk >= c.num_blocks) {
+      report(p.dev_status, DIFFQKV_ERR_INDEX);
+      return nullptr;
+    }
+  }
+  if (sg.dest == kToKCache)
+    return reinterpret_cast<__nv_bfloat16*>(const_cast<void*>(c.k)) + blk * c.k_sb + (long long)(col / p.d_qk) * c.k_sh +
+           slot * c.k_st + col % p.d_qk;
+  return reinterpret_cast<__nv_bfloat16*>(const_cast<void*>(c.v)) + blk * c.v_sb + (long long)(col / p.d_v) * c.v_sh +
+         slot * c.v_st + col % p.d_v;
 }
 
 template <int XROWS>  // rows of x per pass: 8 or 16
 __global__ void __launch_bounds__(kSkThreads, 2)
-linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_wa,
-                     const __grid_constant__ CUtensorMap tmap_wb, const SkinnyParams p) {
+linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w0,
+                     const __grid_constant__ CUtensorMap tmap_w1, const __grid_constant__ CUtensorMap tmap_w2,
+                     const __grid_constant__ CUtensorMap tmap_w3, const SkinnyParams p) {
   constexpr int kXBox = kChunks * XROWS * 128;
   constexpr int kStageBytes = 2 * kWBox + kXBox;
   constexpr int kStages = kRingBytes / kStageBytes;
@@ -90,8 +137,10 @@ linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
     }
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmap_x);
-    ptx::prefetch_tmap(&tmap_wa);
-    ptx::prefetch_tmap(&tmap_wb);
+    ptx::prefetch_tmap(&tmap_w0);
+    ptx::prefetch_tmap(&tmap_w1);
+    ptx::prefetch_tmap(&tmap_w2);
+    ptx::prefetch_tmap(&tmap_w3);
   }
   __syncthreads();
   ptx::grid_launch_dependents();
@@ -110,13 +159,14 @@ linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
       struct Walk { int it, c; };
       Walk w = {(int)blockIdx.x, 0}, x = w;
       auto step = [&](Walk& k) { if (++k.c == n_chunks) { k.c = 0; k.it += gridDim.x; } };
+      const CUtensorMap* wmaps[4] = {&tmap_w0, &tmap_w1, &tmap_w2, &tmap_w3};
       auto load_w = [&](const Walk& k, int st) {
         int row_a, row_b;
-        item_rows(p, k.it / p.passes, row_a, row_b);
+        const Segment& sg = item_rows(p, k.it / p.passes, row_a, row_b);
         const uint32_t bar = full0 + 8 * st, dst = smem_u32 + st * kStageBytes;
         ptx::mbar_arrive_expect_tx(bar, kStageBytes);
-        ptx::tma_load_3d(dst, &tmap_wa, bar, 0, row_a, k.c * kChunks);
-        ptx::tma_load_3d(dst + kWBox, &tmap_wb, bar, 0, row_b, k.c * kChunks);
+        ptx::tma_load_3d(dst, wmaps[sg.map_a], bar, 0, row_a, k.c * kChunks);
+        ptx::tma_load_3d(dst + kWBox, wmaps[sg.map_b], bar, 0, row_b, k.c * kChunks);
       };
       auto load_x = [&](const Walk& k, int st) {
         ptx::tma_load_3d(smem_u32 + st * kStageBytes + 2 * kWBox, &tmap_x, full0 + 8 * st, 0, XROWS * (k.it % p.passes),
@@ -169,7 +219,7 @@ linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
       asm volatile("bar.arrive 2, %0;" ::"n"(kBarThreads) : "memory");  // the buffer may be written again
       if (*abort_flag) continue;
       int row_a, row_b;
-      item_rows(p, it / p.passes, row_a, row_b);
+      const Segment& sg = item_rows(p, it / p.passes, row_a, row_b);
       // thread: weight rows g8 of either group, rows 2 t4 and 2 t4 + 1 of x in each 8-row block of the pass
 #pragma unroll
       for (int nb = 0; nb < NB; ++nb)
@@ -178,18 +228,22 @@ linear_skinny_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
           const int t = XROWS * (it % p.passes) + 8 * nb + 2 * t4 + e;
           if (t >= p.M) continue;
           const float ca = v[4 * nb + e], cb = v[4 * nb + 2 + e];
-          __nv_bfloat16* crow = p.C + (long long)t * p.ldc;
-          if (p.mode == kGateUp) {
-            crow[row_a + g8] = __float2bfloat16_rn(ca / (1.f + __expf(-ca)) * cb);
-          } else if (p.mode == kRotary) {
-            const int half = p.head_dim >> 1;
-            const long long ti = (long long)t * half + (row_a % p.head_dim) + g8;
+          __nv_bfloat16* da = dest_of(p, sg, t, row_a + g8);
+          if (!da) continue;
+          if (sg.mode == kGateUp) {
+            *da = __float2bfloat16_rn(ca / (1.f + __expf(-ca)) * cb);
+            continue;
+          }
+          __nv_bfloat16* db = dest_of(p, sg, t, row_b + g8);
+          if (sg.mode == kRotary) {
+            const int half = sg.head_dim >> 1;
+            const long long ti = (long long)t * half + (row_a % sg.head_dim) + g8;
             const float cs = p.rope_cos[ti], sn = p.rope_sin[ti];
-            crow[row_a + g8] = __float2bfloat16_rn(ca * cs - cb * sn);
-            crow[row_b + g8] = __float2bfloat16_rn(cb * cs + ca * sn);
+            *da = __float2bfloat16_rn(ca * cs - cb * sn);
+            *db = __float2bfloat16_rn(cb * cs + ca * sn);
           } else {
-            crow[row_a + g8] = __float2bfloat16_rn(ca);
-            crow[row_b + g8] = __float2bfloat16_rn(cb);
+            *da = __float2bfloat16_rn(ca);
+            *db = __float2bfloat16_rn(cb);
           }
         }
     }
@@ -261,27 +315,15 @@ bool linear_skinny_supported(long long M, int N, int K, bool dual, int head_dim,
   return dual ? N % 8 == 0 : N % 16 == 0;
 }
 
-cudaError_t launch_linear_skinny(const void* A, const void* B0, const void* B1, void* C, long long M, int N, int K,
-                                 int* dev_status, cudaStream_t stream, const float* rope_cos, const float* rope_sin,
-                                 int head_dim) {
-  const int xrows = M <= 8 ? 8 : 16;
-  CUtensorMap mx, ma, mb;
-  if (!make_rows_map(&mx, A, M, K, xrows) || !make_rows_map(&ma, B0, N, K, 8) ||
-      !make_rows_map(&mb, B1 ? B1 : B0, N, K, 8))
-    return cudaErrorNotSupported;
-  SkinnyParams p;
-  p.C = reinterpret_cast<__nv_bfloat16*>(C);
-  p.ldc = N; p.M = (int)M; p.N = N; p.K = K;
-  p.mode = B1 ? kGateUp : (rope_cos ? kRotary : kPlain);
-  p.head_dim = head_dim;
-  p.items = p.mode == kGateUp ? N / 8 : N / 16;
-  p.passes = (int)((M + xrows - 1) / xrows);
-  p.rope_cos = rope_cos; p.rope_sin = rope_sin;
-  p.dev_status = dev_status;
+namespace {
+
+cudaError_t launch_segments(const CUtensorMap& mx, const CUtensorMap (&mw)[4], SkinnyParams& p, int xrows,
+                            cudaStream_t stream) {
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return cudaErrorUnknown;
+  p.passes = (p.M + xrows - 1) / xrows;
   const long long total = (long long)p.items * p.passes;
   auto kernel = xrows == 8 ? linear_skinny_kernel<8> : linear_skinny_kernel<16>;
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSkSmem);
@@ -296,10 +338,67 @@ cudaError_t launch_linear_skinny(const void* A, const void* B0, const void* B1, 
   cfg.gridDim = dim3((unsigned)(total < 2 * sms ? total : 2 * sms));  // two blocks per SM
   cfg.blockDim = dim3(kSkThreads);
   cfg.dynamicSmemBytes = kSkSmem;
-  err = cudaLaunchKernelEx(&cfg, kernel, mx, ma, mb, p);
+  err = cudaLaunchKernelEx(&cfg, kernel, mx, mw[0], mw[1], mw[2], mw[3], p);
   if (err != cudaSuccess) return err;
   count_launch();
   return cudaGetLastError();
+}
+
+Segment make_segment(int first_item, int mode, int head_dim, int map_a, int map_b, int dest, void* C, int ldc) {
+  Segment sg;
+  sg.first_item = first_item; sg.mode = mode; sg.head_dim = head_dim;
+  sg.map_a = map_a; sg.map_b = map_b; sg.dest = dest;
+  sg.C = reinterpret_cast<__nv_bfloat16*>(C); sg.ldc = ldc;
+  return sg;
+}
+
+}  // namespace
+
+cudaError_t launch_linear_skinny(const void* A, const void* B0, const void* B1, void* C, long long M, int N, int K,
+                                 int* dev_status, cudaStream_t stream, const float* rope_cos, const float* rope_sin,
+                                 int head_dim) {
+  const int xrows = M <= 8 ? 8 : 16;
+  CUtensorMap mx, mw[4];
+  if (!make_rows_map(&mx, A, M, K, xrows) || !make_rows_map(&mw[0], B0, N, K, 8) ||
+      !make_rows_map(&mw[1], B1 ? B1 : B0, N, K, 8))
+    return cudaErrorNotSupported;
+  mw[2] = mw[0];
+  mw[3] = mw[0];
+  SkinnyParams p = {};
+  const int mode = B1 ? kGateUp : (rope_cos ? kRotary : kPlain);
+  p.seg[0] = make_segment(0, mode, head_dim, 0, B1 ? 1 : 0, kToMatrix, C, N);
+  p.n_seg = 1;
+  p.M = (int)M; p.K = K;
+  p.items = mode == kGateUp ? N / 8 : N / 16;
+  p.rope_cos = rope_cos; p.rope_sin = rope_sin;
+  p.dev_status = dev_status;
+  return launch_segments(mx, mw, p, xrows, stream);
+}
+
+// One launch for everything a decode step computes from the hidden state h [M, K]: x = h W_Q^T into C (the first
+// product of the aug-Q chain), k = rope(h W_K^T) and v = h W_V^T straight into the cache rows of the new tokens.
+cudaError_t launch_qkv_skinny(const void* h, const void* W_Q, void* x, int d_q0, const void* W_K, const void* W_V,
+                              long long M, int K, const float* rope_cos, const float* rope_sin, const CacheView& cache,
+                              int n_k, int n_v, int d_qk, int d_v, int* dev_status, cudaStream_t stream) {
+  const int xrows = M <= 8 ? 8 : 16;
+  CUtensorMap mx, mw[4];
+  if (!make_rows_map(&mx, h, M, K, xrows) || !make_rows_map(&mw[0], W_Q, d_q0, K, 8) ||
+      !make_rows_map(&mw[1], W_K, (long long)n_k * d_qk, K, 8) || !make_rows_map(&mw[2], W_V, (long long)n_v * d_v, K, 8))
+    return cudaErrorNotSupported;
+  mw[3] = mw[0];
+  SkinnyParams p = {};
+  const int items_q = d_q0 / 16, items_k = n_k * d_qk / 16, items_v = n_v * d_v / 16;
+  p.seg[0] = make_segment(0, kPlain, 0, 0, 0, kToMatrix, x, d_q0);
+  p.seg[1] = make_segment(items_q, rope_cos ? kRotary : kPlain, d_qk, 1, 1, kToKCache, nullptr, 0);
+  p.seg[2] = make_segment(items_q + items_k, kPlain, 0, 2, 2, kToVCache, nullptr, 0);
+  p.n_seg = 3;
+  p.M = (int)M; p.K = K;
+  p.items = items_q + items_k + items_v;
+  p.rope_cos = rope_cos; p.rope_sin = rope_sin;
+  p.cache = cache;
+  p.d_qk = d_qk; p.d_v = d_v;
+  p.dev_status = dev_status;
+  return launch_segments(mx, mw, p, xrows, stream);
 }
 
 }  // namespace diffqkv

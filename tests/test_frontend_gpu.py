@@ -184,3 +184,65 @@ def test_decode_step_through_the_front_end(api, oracle):
     # and the front-end outputs themselves against the unrounded chain
     k_ref = oracle.rope(oracle.linear(h, w_k).reshape(batch, n_k, d), pos, theta)
     _check(k_new.float().cpu().numpy().astype(np.float64).reshape(batch, n_k, d), k_ref, "k_new")
+
+
+@pytest.mark.parametrize("batch,paged,rotate", [(2, 0, True), (5, 16, True), (16, 0, False), (33, 64, True), (70, 0, True)])
+def test_fused_decode_front_end_equals_the_separate_steps(api, oracle, tensor_gemm, batch, paged, rotate):
+    """diffqkv_decode_frontend writes the same cache rows and returns the same queries as diffqkv_project x 2 +
+    diffqkv_cache_append + diffqkv_augq_rope, bit for bit when both run on the same kernels (up to 64 sequences the
+    weight-streaming kernel, beyond that the tensor-core one), and the new K row matches the oracle's chain."""
+    n_q, n_k, n_v, d, d_model, d_aug, theta, S = 8, 2, 4, 128, 256, 384, 50000.0, 200
+    cfg = W.DecodeConfig("t", batch=batch, n_q=n_q, n_k=n_k, n_v=n_v, d_qk=d, d_v=d, kv_len=S, seed=181)
+    lens = (np.arange(batch) * 37 % (S - 1)).astype(np.int32)
+    inp = W.make_decode_inputs(cfg, seqlens=lens)
+    if paged:
+        inp = W.paginate(inp, paged, seed=5)
+    h = W.normal(182, (batch, d_model))
+    w_k = W.normal(183, (n_k * d, d_model), std=d_model ** -0.5)
+    w_v = W.normal(184, (n_v * d, d_model), std=d_model ** -0.5)
+    ws = [W.normal(185, (n_q * d, d_model), std=d_model ** -0.5), W.normal(186, (d_aug, n_q * d), std=(n_q * d) ** -0.5),
+          W.normal(187, (d_aug, n_q * d), std=(n_q * d) ** -0.5), W.normal(188, (n_q * d, d_aug), std=d_aug ** -0.5)]
+    pos = lens.astype(np.int64)
+    cos, sin = _tables(oracle, pos, d, theta) if rotate else (None, None)
+    dev = "cuda"
+    th, tw = W.to_torch(h, dev), [W.to_torch(w, dev) for w in ws]
+    tk, tv = W.to_torch(w_k, dev), W.to_torch(w_v, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    # separate steps
+    c1 = device_cache(api, inp)
+    k_new = (api.diffqkv_project(th, tk, d, cos, sin) if rotate else api.diffqkv_project(th, tk)).view(batch, 1, n_k, d)
+    v_new = api.diffqkv_project(th, tv).view(batch, 1, n_v, d)
+    api.diffqkv_cache_append(k_new, v_new, c1, dev_status=status)
+    q1 = (api.diffqkv_augq_rope(th, *tw, d, cos, sin) if rotate else api.diffqkv_augq(th, *tw)).view(batch, n_q, d)
+    # fused
+    c2 = device_cache(api, inp)
+    q2 = api.diffqkv_decode_frontend(th, *tw, tk, tv, c2, n_q, d, d, cos, sin, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(q1.view(torch.uint16), q2.view(torch.uint16))
+    assert torch.equal(c1.k.view(torch.uint16), c2.k.view(torch.uint16))
+    assert torch.equal(c1.v.view(torch.uint16), c2.v.view(torch.uint16))
+    k_ref = oracle.linear(h, w_k).reshape(batch, n_k, d)
+    if rotate:
+        k_ref = oracle.rope(k_ref, pos, theta)
+    _check(k_new.float().cpu().numpy().astype(np.float64).reshape(batch, n_k, d), k_ref, "k_new")
+    if batch <= 64:  # the same entry on the tensor-core kernels agrees within rounding
+        tensor_gemm(True)
+        c3 = device_cache(api, inp)
+        q3 = api.diffqkv_decode_frontend(th, *tw, tk, tv, c3, n_q, d, d, cos, sin, dev_status=status)
+        torch.cuda.synchronize()
+        assert (q3.float() - q2.float()).abs().max().item() <= 2e-2 * q2.float().abs().max().item()
+        assert (c3.k.float() - c2.k.float()).abs().max().item() <= 2e-2 * c2.k.float().abs().max().item()
+
+
+def test_fused_decode_front_end_reports_a_full_cache(api):
+    n_q, n_k, n_v, d, d_model, d_aug = 8, 2, 2, 128, 128, 128
+    z = lambda *s: torch.zeros(s, dtype=torch.bfloat16, device="cuda")  # noqa: E731
+    lens = torch.tensor([64, 10], dtype=torch.int32, device="cuda")  # sequence 0 is full
+    cache = api.KVCache(z(2, n_k, 64, d), z(2, n_v, 64, d), lens, 64)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.diffqkv_decode_frontend(z(2, d_model), z(n_q * d, d_model), z(d_aug, n_q * d), z(d_aug, n_q * d),
+                                z(n_q * d, d_aug), z(n_k * d, d_model), z(n_v * d, d_model), cache, n_q, d, d,
+                                dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 1 << api.ERR_INDEX
