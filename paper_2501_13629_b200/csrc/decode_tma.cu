@@ -535,6 +535,17 @@ combine_segments_kernel(const float* __restrict__ o_partial, const float* __rest
   const int n = (int)(last - first + 1);
   const float* lp = lse_partial + (first + wlin) * U + col;  // partial c at lp[c * U]
   const float* op = o_partial + ((first + wlin) * U + col) * d_v;  // partial c at op[c * U * d_v]
+  // The first partials of this warp's share (channels 0 .. 127) are requested together with the log-sum-exps, so
+  // that the step costs one trip to L2 and not two: it is all that is left on the stream once the split kernel ends.
+  constexpr int kEarly = 4;
+  float4 early[kEarly];
+  const int ch_e = lane * 4;
+#pragma unroll
+  for (int i = 0; i < kEarly; ++i) {
+    const int c = warp + 4 * i;
+    early[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < n && ch_e < d_v) early[i] = *reinterpret_cast<const float4*>(op + (long long)c * U * d_v + ch_e);
+  }
   float M = -INFINITY;
   for (int c = lane; c < n; c += 32) M = fmaxf(M, lp[(long long)c * U]);
 #pragma unroll
@@ -547,8 +558,18 @@ combine_segments_kernel(const float* __restrict__ o_partial, const float* __rest
     const int ch = ch0 + lane * 4;
     const bool in = ch < d_v;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    int c = warp;
+    if (ch0 == 0) {
+#pragma unroll
+      for (int i = 0; i < kEarly; ++i, c += 4)
+        if (c < n) {
+          const float wgt = exp2f(lp[(long long)c * U] - M);
+          const float4 v = early[i];
+          a.x = fmaf(wgt, v.x, a.x); a.y = fmaf(wgt, v.y, a.y); a.z = fmaf(wgt, v.z, a.z); a.w = fmaf(wgt, v.w, a.w);
+        }
+    }
 #pragma unroll 4
-    for (int c = warp; c < n; c += 4) {
+    for (; c < n; c += 4) {
       const float wgt = exp2f(lp[(long long)c * U] - M);
       if (in) {
         const float4 v = *reinterpret_cast<const float4*>(op + (long long)c * U * d_v + ch);
