@@ -119,6 +119,21 @@ diffqkv_status diffqkv_decode(const void *q, const diffqkv_cache *cache, const d
                               float *lse, int32_t *dev_status, void *stream);
 
 /*
+ * diffqkv_decode_host -- diffqkv_decode for a query that sits in host memory and a result that is wanted there (the
+ * paper has no counterpart; the KV cache is decode state and stays on the device).  On `stream`, in order: copy
+ * q_host -> q_dev, diffqkv_decode(q_dev ... out_dev), copy out_dev -> out_host.  Nothing is synchronised: the result
+ * is in out_host once the stream has run the last copy.
+ *   q_host, out_host  HOST pointers ([batch, n_q, d_qk] shape.dtype and [batch, n_q, d_v] shape.out_dtype);
+ *                     page-locked memory keeps the copies asynchronous
+ *   q_dev, out_dev    device staging buffers of the same sizes, provided by the caller (the library allocates nothing)
+ *   everything else as in diffqkv_decode
+ */
+diffqkv_status diffqkv_decode_host(const void *q_host, void *q_dev, const diffqkv_cache *cache,
+                                   const diffqkv_shape *shape, int32_t num_splits, void *workspace,
+                                   size_t workspace_bytes, void *out_dev, void *out_host, float *lse,
+                                   int32_t *dev_status, void *stream);
+
+/*
  * diffqkv_decode_static -- diffqkv_decode for callers that cannot provide or allocate a workspace.
  * (The paper has no counterpart; this is a deployment convenience of this library.)
  * Some hosts cannot call cudaMalloc when they decode: all device memory already belongs to their own

@@ -32,7 +32,7 @@ EXPORTS = (
     "diffqkv_set_max_blocks", "diffqkv_topk_general_only", "diffqkv_last_decode_kernel",
     "diffqkv_last_prefill_kernel", "diffqkv_force_tensor_gemm", "diffqkv_augq_rope", "diffqkv_project", "diffqkv_cache_append",
     "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes", "diffqkv_decode_frontend",
-    "diffqkv_decode_frontend_workspace_bytes",
+    "diffqkv_decode_frontend_workspace_bytes", "diffqkv_decode_host",
 )
 
 
@@ -102,6 +102,9 @@ _lib.diffqkv_decode_frontend.restype = C.c_int32
 _lib.diffqkv_decode_frontend.argtypes = [C.c_void_p] * 7 + [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                          C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_void_p, C.c_size_t,
                                          C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.diffqkv_decode_host.restype = C.c_int32
+_lib.diffqkv_decode_host.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_int32,
+                                     C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.diffqkv_force_tensor_gemm.restype = None
 _lib.diffqkv_force_tensor_gemm.argtypes = [C.c_int32]
 _lib.diffqkv_last_prefill_kernel.restype = C.c_int32
@@ -250,6 +253,48 @@ def diffqkv_decode(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: f
     """q [batch, n_q, d_qk] against the cache; returns out [batch, n_q, d_v] (enqueued on the stream)."""
     return _decode("diffqkv_decode", q, cache, n_k, n_v, scale, num_splits, workspace, out, lse, dev_status,
                    out_dtype, stream)
+
+
+def diffqkv_decode_host(q_host: torch.Tensor, q_dev: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: float,
+                        workspace: torch.Tensor, out_dev: torch.Tensor, out_host: torch.Tensor, num_splits: int = 0,
+                        lse: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                        stream: Optional[torch.cuda.Stream] = None):
+    """diffqkv_decode with the query in (pinned) host memory and the result copied back to (pinned) host memory, all on
+    the stream and in one library call; q_dev / out_dev are the device staging buffers.  Returns out_host, which
+    is valid once the stream has been synchronised."""
+    batch, n_q, d_qk = q_host.shape
+    assert not q_host.is_cuda and not out_host.is_cuda and q_dev.is_cuda and out_dev.is_cuda
+    shape = make_shape(batch, n_q, n_k, n_v, d_qk, cache.v.shape[-1], q_host.dtype, out_host.dtype, scale)
+    cs = cache.c_struct()
+    st = _lib.diffqkv_decode_host(_p(q_host), _p(q_dev), C.byref(cs), C.byref(shape), int(num_splits), _p(workspace),
+                                  workspace.numel(), _p(out_dev), _p(out_host), _p(lse), _p(dev_status),
+                                  _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_decode_host")
+    return out_host
+
+
+def bind_decode_host(q_host: torch.Tensor, q_dev: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: float,
+                     workspace: torch.Tensor, out_dev: torch.Tensor, out_host: torch.Tensor, num_splits: int = 0,
+                     lse: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None):
+    """diffqkv_decode_host with its argument structs built once: returns a function of no arguments that makes the
+    library call on the current stream (what a C caller that keeps its diffqkv_shape / diffqkv_cache around does).
+    The tensors must stay alive and unmoved while the function is in use."""
+    batch, n_q, d_qk = q_host.shape
+    assert not q_host.is_cuda and not out_host.is_cuda and q_dev.is_cuda and out_dev.is_cuda
+    shape = make_shape(batch, n_q, n_k, n_v, d_qk, cache.v.shape[-1], q_host.dtype, out_host.dtype, scale)
+    cs = cache.c_struct()
+    args = (_p(q_host), _p(q_dev), C.byref(cs), C.byref(shape), int(num_splits), _p(workspace), workspace.numel(),
+            _p(out_dev), _p(out_host), _p(lse), _p(dev_status))
+    keep = (shape, cs, q_host, q_dev, cache, workspace, out_dev, out_host, lse, dev_status)
+
+    def call():
+        st = _lib.diffqkv_decode_host(*args, C.c_void_p(torch.cuda.current_stream().cuda_stream))
+        if st != OK:
+            raise DiffQKVError(st, "diffqkv_decode_host")
+        return keep[7]
+
+    return call
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

@@ -192,6 +192,26 @@ diffqkv_status diffqkv_decode(const void* q, const diffqkv_cache* cache, const d
                      static_cast<cudaStream_t>(stream));
 }
 
+diffqkv_status diffqkv_decode_host(const void* q_host, void* q_dev, const diffqkv_cache* cache,
+                                   const diffqkv_shape* shape, int32_t num_splits, void* workspace,
+                                   size_t workspace_bytes, void* out_dev, void* out_host, float* lse,
+                                   int32_t* dev_status, void* stream) {
+  const diffqkv_status st = check_shape(shape);
+  if (st != DIFFQKV_OK) return st;
+  if (!q_host || !q_dev || !out_dev || !out_host) return DIFFQKV_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t rows = (size_t)shape->batch * shape->n_q;
+  const size_t q_bytes = rows * shape->d_qk * (shape->dtype == DIFFQKV_BF16 ? 2 : 4);
+  const size_t out_bytes = rows * shape->d_v * (shape->out_dtype == DIFFQKV_BF16 ? 2 : 4);
+  if (q_bytes && cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return DIFFQKV_ERR_CUDA;
+  const diffqkv_status ds =
+      decode_impl(q_dev, cache, shape, num_splits, workspace, workspace_bytes, out_dev, lse, dev_status, s);
+  if (ds != DIFFQKV_OK) return ds;
+  if (out_bytes && cudaMemcpyAsync(out_host, out_dev, out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return DIFFQKV_ERR_CUDA;
+  return DIFFQKV_OK;
+}
+
 diffqkv_status gqa_decode(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape, int32_t num_splits,
                           void* workspace, size_t workspace_bytes, void* out, float* lse, int32_t* dev_status,
                           void* stream) {

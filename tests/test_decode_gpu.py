@@ -288,3 +288,29 @@ def test_config5_full_size_sampled_rows(api, oracle):
     sel = (pairs[:, 0], pairs[:, 1])
     check_bf16(got[sel], ref[sel], "cfg5 full size")
     check_lse(lse.cpu().numpy().astype(np.float64)[sel], lse_ref[sel], 2e-2, "cfg5 full size")
+
+
+def test_decode_from_and_to_host_memory(api, oracle):
+    """diffqkv_decode_host: q in pinned host memory, the result back in pinned host memory, same numbers as
+    diffqkv_decode on device buffers (bitwise) and within tolerance of the oracle."""
+    inp = W.make_decode_inputs(SMALL)
+    cfg = inp.cfg
+    cache = device_cache(api, inp)
+    q_dev_in = W.to_torch(inp.q, "cuda")
+    ref_out = api.diffqkv_decode(q_dev_in, cache, cfg.n_k, cfg.n_v, cfg.scale, out_dtype=torch.float32)
+    q_host = W.to_torch(inp.q).pin_memory()
+    out_host = torch.empty(ref_out.shape, dtype=torch.float32).pin_memory()
+    q_dev, out_dev = torch.empty_like(q_dev_in), torch.empty_like(ref_out)
+    shape = api.make_shape(cfg.batch, cfg.n_q, cfg.n_k, cfg.n_v, cfg.d_qk, cfg.d_v, q_dev.dtype, torch.float32, cfg.scale)
+    ws = torch.empty(max(api.diffqkv_decode_workspace_bytes(shape, int(inp.max_seqlen), 0), 256), dtype=torch.uint8,
+                     device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for _ in range(2):
+        out_host.fill_(float("nan"))
+        api.diffqkv_decode_host(q_host, q_dev, cache, cfg.n_k, cfg.n_v, cfg.scale, ws, out_dev, out_host,
+                                dev_status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(out_host, ref_out.cpu())
+    ref, _ = run_oracle(oracle, inp)
+    check_bf16(out_host.numpy().astype(np.float64), ref, "decode from host memory")
