@@ -671,7 +671,7 @@ bool pick_variant(int d_qk, int d_v, int kpu, int vpu, Variant* v) {
   DIFFQKV_CASE(128, 128, 2, 1) DIFFQKV_CASE(128, 128, 4, 1)
   DIFFQKV_CASE(64, 64, 1, 1) DIFFQKV_CASE(64, 64, 1, 2) DIFFQKV_CASE(64, 64, 1, 4)
   DIFFQKV_CASE(64, 64, 2, 1) DIFFQKV_CASE(64, 64, 4, 1)
-  DIFFQKV_CASE(64, 128, 1, 1) DIFFQKV_CASE(64, 128, 1, 2)
+  DIFFQKV_CASE(64, 128, 1, 1) DIFFQKV_CASE(64, 128, 1, 2) DIFFQKV_CASE(64, 128, 1, 4)
   DIFFQKV_CASE(64, 64, 2, 2) DIFFQKV_CASE(64, 64, 4, 4) DIFFQKV_CASE(64, 64, 2, 4) DIFFQKV_CASE(64, 64, 4, 2)
 #undef DIFFQKV_CASE
   return false;

@@ -71,6 +71,24 @@ def test_mixed_head_dims(api, oracle):
     check_bf16(out, ref)
 
 
+@pytest.mark.parametrize("heads", [(32, 4, 16), (16, 2, 4), (8, 4, 4)])
+def test_half_width_keys_take_the_tma_kernel(api, oracle, heads):
+    """d_k = d_v / 2 (the paper's other axis of K compression) with SIGMA-1.5B's 4 K / 16 V heads and two smaller
+    shapes: the persistent TMA kernel, not the generic fallback."""
+    n_q, n_k, n_v = heads
+    cfg = dataclasses.replace(SMALL, n_q=n_q, n_k=n_k, n_v=n_v, d_qk=64, d_v=128, kv_len=1500, seed=44)
+    inp = W.make_decode_inputs(cfg, seqlens=np.array([1500, 333, 64], dtype=np.int32))
+    ref, lse_ref = run_oracle(oracle, inp)
+    out, lse, st = run_decode(api, inp)
+    assert st == 0 and api.last_decode_kernel() == 2
+    check_bf16(out, ref, str(heads))
+    check_lse(lse, lse_ref, 2e-2)
+    pg = W.paginate(inp, 16, seed=3)
+    out_p, lse_p, st = run_decode(api, pg)
+    assert st == 0 and api.last_decode_kernel() == 2
+    assert np.array_equal(out_p, out) and np.array_equal(lse_p, lse)
+
+
 @pytest.mark.parametrize("lens", [[0, 0, 0], [0, 5, 700], [63, 64, 65], [127, 128, 129], [1, 2, 3]])
 def test_ragged_and_empty_lengths(api, oracle, lens):
     inp = W.make_decode_inputs(SMALL, seqlens=np.array(lens, dtype=np.int32))
