@@ -85,6 +85,7 @@ void profile_after_split(cudaStream_t stream);  // records the benchmark hook's 
 // TMA decode path (decode_tma.cu): persistent blocks over a flat (sequence, unit, tile) list.
 struct TmaPlan {
   int U, kpu, vpu;   // query heads, K heads and V heads per unit
+  int k_shift, v_shift;  // 2^shift neighbouring units read the same K (V) head (more than 8 query heads per head)
   int box_tok;       // tokens per TMA box
   int stages, grid, smem;
   long long slots;   // partial-result slots: grid + batch * units

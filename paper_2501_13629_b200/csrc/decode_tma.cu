@@ -46,6 +46,7 @@ struct TmaParams {
   int page_size, max_pages_per_seq, num_blocks, max_seqlen;
   int batch, n_q, n_units, U;
   int hk_per_unit, hv_per_unit;  // KPU, VPU
+  int k_shift, v_shift;          // units that share their K (V) head with 2^shift - 1 neighbours: head = (u * KPU) >> shift
   int box_tok;                   // tokens per TMA box (64, or the page size when smaller)
   int stages;
   float scale_log2;
@@ -90,7 +91,8 @@ struct Walker {
   }
 };
 
-template <int D_QK, int D_V, int KPU, int VPU>
+// SHARED: neighbouring units read the same K or V head (see k_shift / v_shift); the plain case keeps its own code.
+template <int D_QK, int D_V, int KPU, int VPU, bool SHARED = false>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                   const TmaParams p) {
@@ -212,8 +214,13 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
           blk = 0;
         }
         const uint32_t dst = ptx::smem_u32(stage_base + (size_t)stage * STAGE_BYTES) + my_off;
-        if (my_is_k) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, 0, w.u * KPU + my_tile, blk);
-        else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, 0, w.u * VPU + (my_tile - KPU), blk);
+        if (SHARED) {
+          if (my_is_k) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, 0, ((w.u * KPU) >> p.k_shift) + my_tile, blk);
+          else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, 0, ((w.u * VPU) >> p.v_shift) + (my_tile - KPU), blk);
+        } else {
+          if (my_is_k) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, 0, w.u * KPU + my_tile, blk);
+          else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, 0, w.u * VPU + (my_tile - KPU), blk);
+        }
       }
       ++issued;
       if (++stage == p.stages) { stage = 0; phase ^= 1; }
@@ -655,13 +662,16 @@ DeviceInfo device_info() {
 using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const TmaParams);
 struct Variant {
   KernelFn fn;
+  KernelFn fn_shared;  // the SHARED instantiation, where one exists (a shared pool has one head per unit)
   int stage_bytes;
   int d_v;
 };
 
 template <int D_QK, int D_V, int KPU, int VPU>
 Variant variant() {
-  return Variant{decode_tma_kernel<D_QK, D_V, KPU, VPU>, kTT * 2 * (KPU * D_QK + VPU * D_V), D_V};
+  KernelFn shared = nullptr;
+  if constexpr (KPU == 1 || VPU == 1) shared = decode_tma_kernel<D_QK, D_V, KPU, VPU, true>;
+  return Variant{decode_tma_kernel<D_QK, D_V, KPU, VPU>, shared, kTT * 2 * (KPU * D_QK + VPU * D_V), D_V};
 }
 
 bool pick_variant(int d_qk, int d_v, int kpu, int vpu, Variant* v) {
@@ -683,10 +693,29 @@ bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPla
   if (s.dtype != DIFFQKV_BF16) return false;
   const int mn = s.n_k < s.n_v ? s.n_k : s.n_v;
   if (s.n_k % mn != 0 || s.n_v % mn != 0) return false;
-  int U = s.n_q / mn, kpu = s.n_k / mn, vpu = s.n_v / mn;
-  if (U > kHeadsPerMma || s.batch > kMaxBatchTma || s.batch < 1) return false;
+  int U = s.n_q / mn, kpu = s.n_k / mn, vpu = s.n_v / mn, k_shift = 0, v_shift = 0;
+  if (U > kHeadsPerMma) {
+    // More query heads per unit than one MMA takes: cut the unit into sub-units of kHeadsPerMma query heads.  A
+    // sub-unit needs its share of the unit's K and V heads, at least one each; neighbouring sub-units that share a
+    // head stream it again (mostly out of L2: they run at the same time on other SMs).
+    if (U % kHeadsPerMma != 0) return false;
+    const int sub = U / kHeadsPerMma;
+    auto share = [&](int& per_unit, int* shift) {  // heads per sub-unit, and how many sub-units share one (2^shift)
+      if (per_unit >= sub) { if (per_unit % sub != 0) return false; per_unit /= sub; return true; }
+      int sh = 0;
+      while ((per_unit << sh) < sub) ++sh;
+      if ((per_unit << sh) != sub) return false;  // powers of two only
+      *shift = sh;
+      per_unit = 1;
+      return true;
+    };
+    if (!share(kpu, &k_shift) || !share(vpu, &v_shift)) return false;
+    U = kHeadsPerMma;
+  }
+  if (s.batch > kMaxBatchTma || s.batch < 1) return false;
   Variant v;
   if (!pick_variant(s.d_qk, s.d_v, kpu, vpu, &v)) return false;
+  if ((k_shift || v_shift) && !v.fn_shared) return false;
   // Small units make small tiles (16-24 KB per 64 tokens at d = 64), and the fixed cost per tile then shows.  Several
   // neighbouring units can share a tile: m units are one unit of m*U query heads with m*KPU K heads and m*VPU V
   // heads (the head maps are contiguous blocks, so nothing else changes).  Merge while the tile stays within 64 KB.
@@ -718,6 +747,7 @@ bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPla
   if (grid > tiles_max) grid = tiles_max;
   if (grid < 1) grid = 1;
   plan->U = U; plan->kpu = kpu; plan->vpu = vpu; plan->box_tok = box_tok; plan->stages = stages;
+  plan->k_shift = k_shift; plan->v_shift = v_shift;
   plan->grid = (int)grid;
   plan->smem = fixed + stages * v.stage_bytes;
   plan->slots = grid + (long long)s.batch * (s.n_q / U);
@@ -753,6 +783,7 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
   p.num_blocks = c.num_blocks; p.max_seqlen = c.max_seqlen;
   p.batch = s.batch; p.n_q = s.n_q; p.n_units = s.n_q / plan.U; p.U = plan.U;
   p.hk_per_unit = plan.kpu; p.hv_per_unit = plan.vpu;
+  p.k_shift = plan.k_shift; p.v_shift = plan.v_shift;
   p.box_tok = plan.box_tok; p.stages = plan.stages;
   p.scale_log2 = s.scale * kLog2e;
   char* ws = reinterpret_cast<char*>(workspace);
@@ -764,7 +795,9 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
   p.out = out; p.lse = lse; p.out_is_f32 = s.out_dtype == DIFFQKV_F32;
   p.dev_status = dev_status;
 
-  cudaError_t err = cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem);
+  const KernelFn fn = (plan.k_shift || plan.v_shift) ? v.fn_shared : v.fn;
+  if (!fn) return cudaErrorNotSupported;
+  cudaError_t err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem);
   if (err != cudaSuccess) return err;
   // both kernels may start before their predecessor in the stream has finished; each waits on the device
   // before it touches anything the predecessor may still be producing
@@ -778,7 +811,7 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
   cfg.gridDim = dim3((unsigned)plan.grid);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = (size_t)plan.smem;
-  err = cudaLaunchKernelEx(&cfg, v.fn, mk, mv, p);
+  err = cudaLaunchKernelEx(&cfg, fn, mk, mv, p);
   if (err != cudaSuccess) return err;
   count_launch();
   profile_after_split(stream);

@@ -71,6 +71,23 @@ def test_mixed_head_dims(api, oracle):
     check_bf16(out, ref)
 
 
+@pytest.mark.parametrize("heads", [(32, 1, 2), (32, 2, 4), (32, 2, 2), (16, 1, 1), (64, 4, 8), (64, 2, 16)])
+@pytest.mark.parametrize("d", [64, 128])
+def test_more_than_eight_query_heads_per_kv_head(api, oracle, heads, d):
+    """Multi-query-like shapes: the TMA kernel cuts a unit of 16 to 32 query heads into sub-units of 8 that share
+    their K (and V) head; parity with the oracle, contiguous and paged."""
+    n_q, n_k, n_v = heads
+    cfg = dataclasses.replace(SMALL, batch=2, n_q=n_q, n_k=n_k, n_v=n_v, d_qk=d, d_v=d, kv_len=900, seed=45)
+    inp = W.make_decode_inputs(cfg, seqlens=np.array([900, 130], dtype=np.int32))
+    ref, lse_ref = run_oracle(oracle, inp)
+    out, lse, st = run_decode(api, inp)
+    assert st == 0 and api.last_decode_kernel() == 2
+    check_bf16(out, ref, str(heads))
+    check_lse(lse, lse_ref, 2e-2)
+    out_p, lse_p, st = run_decode(api, W.paginate(inp, 64, seed=4))
+    assert st == 0 and np.array_equal(out_p, out) and np.array_equal(lse_p, lse)
+
+
 @pytest.mark.parametrize("heads", [(32, 4, 16), (16, 2, 4), (8, 4, 4)])
 def test_half_width_keys_take_the_tma_kernel(api, oracle, heads):
     """d_k = d_v / 2 (the paper's other axis of K compression) with SIGMA-1.5B's 4 K / 16 V heads and two smaller
