@@ -16,7 +16,8 @@
 //                 reads its 128 scores into registers (tcgen05.ld), takes the row maximum (a running reference
 //                 maximum is only raised when exceeded by 2^8; then O is rescaled in TMEM), computes
 //                 P = 2^(S scale - m), sums it in fp32 and writes it as packed bf16 over the first 64 score columns
-//                 (tcgen05.st), where the second product reads it.
+//                 (tcgen05.st), where the second product reads it; the first 64 tokens of P are announced on a
+//                 barrier of their own, so that half of the second product runs under the rest of the exponentials.
 //   fp32 scores, softmax statistics and output accumulation; P is rounded to bf16 for the second product.
 //   The kernel is a template on the head dimension (128 or 64 channels for Q/K and V alike): with 64 the tiles are
 //   half as wide, the first product takes four K steps instead of eight and O takes 64 TMEM columns per M-tile.
@@ -85,13 +86,14 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   unsigned char* k_s = q_s + 2 * kQBytes;         // ring of K tiles
   unsigned char* v_s = k_s + kKSlots * kTBytes;   // ring of V tiles
   uint64_t* bars = reinterpret_cast<uint64_t*>(v_s + kVSlots * kTBytes);
-  // q_full, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2], drain
+  // q_full, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2], drain, p_half[2]
   const uint32_t q_full = ptx::smem_u32(bars);
   const uint32_t k_full0 = q_full + 8, k_empty0 = k_full0 + 8 * kKSlots;
   const uint32_t v_full0 = k_empty0 + 8 * kKSlots, v_empty0 = v_full0 + 8 * kVSlots;
   const uint32_t s_full0 = v_empty0 + 8 * kVSlots, p_full0 = s_full0 + 16, o_done0 = p_full0 + 16;
   const uint32_t drain = o_done0 + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 + 2 * kKSlots + 2 * kVSlots + 6);
+  const uint32_t p_half0 = drain + 8;  // the first 64 tokens of P_t are in place
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 + 2 * kKSlots + 2 * kVSlots + 6 + 2);
   volatile int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -109,6 +111,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     for (int t = 0; t < 2; ++t) {
       ptx::mbar_init(s_full0 + 8 * t, 1);
       ptx::mbar_init(p_full0 + 8 * t, 4);
+      ptx::mbar_init(p_half0 + 8 * t, 4);
       ptx::mbar_init(o_done0 + 8 * t, 1);
     }
     ptx::mbar_init(drain, 1);
@@ -218,14 +221,23 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         }
         tc::commit(s_full0 + 8 * t);
       };
-      auto issue_pv = [&](int t, int slot, bool first) {  // O_t += P_t . V
+      // O_t += P_t . V in two halves of 64 tokens: the first is issued while the softmax warps still work on the
+      // second half of P_t
+      auto issue_pv = [&](int t, int slot, bool first, int half) {
         const uint32_t va = v_lo + slot * (kTBytes >> 4);
         const uint32_t d = tmem_base + 256 + t * kD, pa = tmem_base + t * 128;
-        if (first) tc::mma_ts_halves<false>(d, pa, va, hi, idesc_pv);
-        else tc::mma_ts_halves<true>(d, pa, va, hi, idesc_pv);
+        constexpr int kSteps = kKT / 32;  // K steps of 16 tokens per half
+        if (half == 0) {
+          if (first) tc::mma_ts_halves<false>(d, pa, va, hi, idesc_pv);
+          else tc::mma_ts_halves<true>(d, pa, va, hi, idesc_pv);
 #pragma unroll
-        for (int k = 1; k < kKT / 16; ++k) tc::mma_ts_halves<true>(d, pa + k * 8, va + ((k * 16 * 128) >> 4), hi, idesc_pv);
-        tc::commit(o_done0 + 8 * t);
+          for (int k = 1; k < kSteps; ++k) tc::mma_ts_halves<true>(d, pa + k * 8, va + ((k * 16 * 128) >> 4), hi, idesc_pv);
+        } else {
+#pragma unroll
+          for (int k = kSteps; k < 2 * kSteps; ++k)
+            tc::mma_ts_halves<true>(d, pa + k * 8, va + ((k * 16 * 128) >> 4), hi, idesc_pv);
+          tc::commit(o_done0 + 8 * t);
+        }
       };
       ok = ptx::mbar_wait(q_full, 0, abort_flag);
       if (ok && nkv_max > 0) ok = ptx::mbar_wait(k_full0, 0, abort_flag);
@@ -241,12 +253,15 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
           if (j < nkv[t]) {
-            if (!ptx::mbar_wait(p_full0 + 8 * t, j & 1, abort_flag) || !ptx::mbar_wait(v_full0 + 8 * vs, vph, abort_flag)) {
+            if (!ptx::mbar_wait(p_half0 + 8 * t, j & 1, abort_flag) || !ptx::mbar_wait(v_full0 + 8 * vs, vph, abort_flag)) {
               ok = false;
               break;
             }
             tc::fence_after_sync();
-            issue_pv(t, vs, j == 0);
+            issue_pv(t, vs, j == 0, 0);
+            if (!ptx::mbar_wait(p_full0 + 8 * t, j & 1, abort_flag)) { ok = false; break; }
+            tc::fence_after_sync();
+            issue_pv(t, vs, j == 0, 1);
           }
           if (t == 1) tc::commit(v_empty0 + 8 * vs);  // every MMA that reads V tile j has been issued
           if (j + 1 < nkv[t]) {  // P_t of tile j has been consumed by then (same pipe, in order): S_t may be overwritten
@@ -323,7 +338,23 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         }
         l *= alpha;
         const float neg_m = -m_ref;
-        // ---- P = 2^(S scale - m_ref) as packed bf16 over the first 64 score columns; fp32 row sum
+        if (j == nkv_max - 1 && (kv_len & (kKT - 1)) != 0) {
+          // ragged last tile: V rows past the sequence end hold whatever followed in memory; zero them before any
+          // product reads the tile (0 * NaN would poison it).  Both M-tiles may do this; they write the same zeros.
+          const int vslot = j % kVSlots;
+          if (!wait_warp(v_full0 + 8 * vslot, (j / kVSlots) & 1, abort_flag)) { ok = false; break; }
+          if (r >= kv_len - k0) {
+#pragma unroll
+            for (int half = 0; half < kHalves; ++half) {
+              uint4* dst = reinterpret_cast<uint4*>(v_s + vslot * kTBytes + half * (kKT * 128) + r * 128);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) dst[e] = make_uint4(0, 0, 0, 0);
+            }
+          }
+          ptx::fence_proxy_async();
+        }
+        // ---- P = 2^(S scale - m_ref) as packed bf16 over the first 64 score columns; fp32 row sum.  The first 64
+        // tokens are announced on their own, so that their half of the product runs during the second half's work.
         float l0 = 0.f, l1 = 0.f;
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
@@ -337,23 +368,14 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             l1 += p1;
           }
           tc::st_32x32b_x32(s_taddr + c * 32, w);
+          if (c == 0) {
+            tc::wait_st();
+            tc::fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(p_half0 + 8 * t);
+          }
         }
         l += l0 + l1;
-        if (j == nkv_max - 1 && (kv_len & (kKT - 1)) != 0) {
-          // ragged last tile: V rows past the sequence end hold whatever followed in memory; zero them
-          // (0 * NaN would poison the product).  Both M-tiles may do this; they write the same zeros.
-          const int vslot = j % kVSlots;
-          if (!wait_warp(v_full0 + 8 * vslot, (j / kVSlots) & 1, abort_flag)) { ok = false; break; }
-          if (r >= kv_len - k0) {
-#pragma unroll
-            for (int half = 0; half < kHalves; ++half) {
-              uint4* dst = reinterpret_cast<uint4*>(v_s + vslot * kTBytes + half * (kKT * 128) + r * 128);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) dst[e] = make_uint4(0, 0, 0, 0);
-            }
-          }
-          ptx::fence_proxy_async();
-        }
         tc::wait_st();
         tc::fence_before_sync();
         __syncwarp();
