@@ -635,8 +635,13 @@ __device__ __noinline__ bool block_select_sparse(const float* row, const float* 
   if (!(mx < INFINITY && mn > -INFINITY)) return false;
   const unsigned key_min = order_key(mn), key_max = order_key(mx);
   unsigned pre = 0, dummy = 0;
-  radix_kth_shared(keys, nblk, key_min, key_max != key_min ? 32 - __clz(key_max - key_min) : 0, k, 2, sc, &pre, &dummy);
-  const unsigned cut_key = key_min + pre;  // at most the k-th largest block maximum
+  // With fewer blocks than kept scores the maxima bound nothing: every finite score is a candidate (the key just
+  // above that of -inf, which is what positions past the row's end hold in the staging area).
+  unsigned cut_key = order_key(-INFINITY) + 1u;
+  if (k < nblk) {
+    radix_kth_shared(keys, nblk, key_min, key_max != key_min ? 32 - __clz(key_max - key_min) : 0, k, 2, sc, &pre, &dummy);
+    cut_key = key_min + pre;  // at most the k-th largest block maximum
+  }
 
   // ---- the blocks that can hold a kept score, in order
   const int per = (nblk + kAttendThreads - 1) / kAttendThreads;
@@ -690,7 +695,9 @@ __device__ __noinline__ bool block_select_sparse(const float* row, const float* 
   for (int i = f_lo; i < f_hi; ++i) cnt += (unsigned)foff[i];
   unsigned ncand = 0;
   at = block_scan(cnt, &ncand, sc);
-  if (ncand > (unsigned)kSparseCand) return false;
+  // fewer candidates than kept scores can only mean scores of -inf among the k largest: leave those rows to the
+  // selection over all scores
+  if (ncand > (unsigned)kSparseCand || ncand < (unsigned)k) return false;
 #pragma unroll 1
   for (int i = f_lo; i < f_hi; ++i) {
     const unsigned c = (unsigned)foff[i];
@@ -745,8 +752,10 @@ __device__ __noinline__ bool block_select_sparse(const float* row, const float* 
     const bool g = key > thr, q = key == thr;
     if (g || (q && eq_before < need_eq)) {
       const unsigned pos = gt_before + min(eq_before, need_eq);
-      out.pos[pos] = cpos[i];
-      out.val[pos] = cval[i];
+      if (pos < (unsigned)kMaxTopk) {  // always true for a consistent threshold; never write past the arrays
+        out.pos[pos] = cpos[i];
+        out.val[pos] = cval[i];
+      }
     }
     gt_before += g;
     eq_before += q;
@@ -796,8 +805,9 @@ topk_attend_kernel(const AttendParams p) {
   }
   const float* row = p.scores + (long long)blockIdx.x * p.lpad;
   int k = min(p.topk, len);
-  // worth trying when the bound from the block maxima cuts deep: at least two blocks per kept score
-  const bool sparse = !p.general_only && 32LL * k <= len &&
+  // worth trying when the bound from the block maxima cuts deep (at least two blocks per kept score), or when the row
+  // is short enough for all of it to fit the candidate buffer
+  const bool sparse = !p.general_only && (32LL * k <= len || len <= kSparseCand) &&
                       block_select_sparse(row, p.bmax + (long long)blockIdx.x * (p.lpad / 16), len, k, sel, sc,
                                           cand_key, cpos, flag_id, foff, stage);
   if (sparse) {
