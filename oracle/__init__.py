@@ -149,6 +149,26 @@ def decode_topk(q: np.ndarray, cache: Cache, n_q: int, n_k: int, n_v: int, d_qk:
     return out, lse, sel, margin
 
 
+def decode_kup(q: np.ndarray, W_kup: np.ndarray, cache: Cache, n_q: int, n_k: int, n_v: int, d_v: int, scale: float):
+    """Decode over keys cached at width d_k < d_q: every cached key goes through the linear layer W_kup[hk]
+    ([n_k, d_q, d_k]) before its inner product with the query.  q [batch, n_q, d_q]; returns (out, lse)."""
+    dt = _dtype_code(q)
+    assert _dtype_code(W_kup) == dt and _dtype_code(cache.k) == dt
+    q, W_kup = np.ascontiguousarray(q), np.ascontiguousarray(W_kup)
+    batch, _, d_q = q.shape
+    assert W_kup.shape[:2] == (n_k, d_q)
+    d_k = W_kup.shape[2]
+    out = np.zeros((batch, n_q, d_v), dtype=np.float64)
+    lse = np.zeros((batch, n_q), dtype=np.float64)
+    cs = cache.c_struct()
+    lib().oracle_decode_kup.restype = C.c_int
+    rc = lib().oracle_decode_kup(_ptr(q), _ptr(W_kup), C.byref(cs), batch, n_q, n_k, n_v, d_q, d_k, d_v, dt,
+                                 C.c_double(scale), _ptr(out), _ptr(lse))
+    if rc != 0:
+        raise ValueError("n_k and n_v must divide n_q")
+    return out, lse
+
+
 def decode_splits(q: np.ndarray, cache: Cache, n_q: int, n_k: int, n_v: int, d_qk: int, d_v: int,
                   scale: float, cuts: Sequence[int]):
     """Per-split normalised outputs and lse for token ranges [cuts[s], cuts[s+1])."""

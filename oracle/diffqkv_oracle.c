@@ -36,6 +36,10 @@
  * oracle_linear and oracle_rope (the projections and the rotary embedding around the cache update) are pinned
  * by a library matmul, by closed forms and by the relative-position identity; that the rotary embedding uses the
  * rotate-half pairing is a reading (the listing only names the call): "parity unpinned" for that choice.
+ * oracle_decode_kup (keys cached at half width, widened by a feed-forward layer before the inner product) is pinned
+ * by its reduction to oracle_decode when the layer is the identity, by a numpy restatement on small shapes, and by
+ * the identity <q, W k> = <W^T q, k> against oracle_decode on folded queries; that the layer is linear, bias-free
+ * and per K head is a reading: "parity unpinned" for that choice.
  * The choice of SiLU as act_fn is a reading of the paper, not pinned by it:
  * for oracle_augq the activation choice is "parity unpinned" (the rest of the
  * chain is pinned by closed forms).
@@ -205,6 +209,58 @@ int oracle_decode_topk(const void *q, const oracle_cache *c, int batch, int n_q,
     }
     lse[w] = m + log(l);
     free(st);
+  }
+  return 0;
+}
+
+/* Decode with keys cached at a smaller width than the queries (Section 2: when the Q and K head dimensions
+ * differ, "Attend" first transforms K to the query width through another feed-forward layer; Observation 2:
+ * d_k = d_v / 2 with that trainable layer).  The layer is read as linear, without bias or activation, with one
+ * weight matrix per K head (the paper does not print it): W_kup [n_k, d_q, d_k].  In the paper's order, for query
+ * head h with K head hk and every cached token j:
+ *     k'_j = W_kup[hk] k_j            (width d_k -> d_q)
+ *     s_j  = scale * <q_h, k'_j>
+ * then softmax over j and the weighted V sum as everywhere else.
+ *   q [batch, n_q, d_q]; the K pool holds rows of d_k channels; W_kup, q and the pools share the storage dtype.
+ * Returns 0, or -1 when n_k or n_v does not divide n_q. */
+int oracle_decode_kup(const void *q, const void *W_kup, const oracle_cache *c, int batch, int n_q, int n_k, int n_v,
+                      int d_q, int d_k, int d_v, int dtype, double scale, double *out, double *lse) {
+  if (n_k <= 0 || n_v <= 0 || n_q % n_k || n_q % n_v) return -1;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t w = 0; w < (int64_t)batch * n_q; ++w) {
+    int b = (int)(w / n_q), h = (int)(w % n_q);
+    int hk = (int)(((int64_t)h * n_k) / n_q);
+    int hv = (int)(((int64_t)h * n_v) / n_q);
+    int64_t len = c->seqlens[b];
+    double *o = out + w * d_v;
+    for (int ch = 0; ch < d_v; ++ch) o[ch] = 0.0;
+    if (len <= 0) { lse[w] = -INFINITY; continue; }
+    double *s = (double *)malloc(sizeof(double) * (size_t)len);
+    double *kw = (double *)malloc(sizeof(double) * (size_t)d_q);
+    double m = -INFINITY;
+    for (int64_t j = 0; j < len; ++j) {
+      int64_t row = cache_row(c, 0, b, j, hk);
+      for (int a = 0; a < d_q; ++a) { /* the feed-forward layer on the cached key */
+        double acc = 0.0;
+        for (int ch = 0; ch < d_k; ++ch)
+          acc += load_elt(W_kup, ((int64_t)hk * d_q + a) * d_k + ch, dtype) * load_elt(c->k_cache, row + ch, dtype);
+        kw[a] = acc;
+      }
+      double acc = 0.0;
+      for (int a = 0; a < d_q; ++a) acc += load_elt(q, w * d_q + a, dtype) * kw[a];
+      s[j] = acc * scale;
+      if (s[j] > m) m = s[j];
+    }
+    double l = 0.0;
+    for (int64_t j = 0; j < len; ++j) { s[j] = exp(s[j] - m); l += s[j]; }
+    for (int64_t j = 0; j < len; ++j) {
+      int64_t row = cache_row(c, 1, b, j, hv);
+      for (int ch = 0; ch < d_v; ++ch) o[ch] += s[j] * load_elt(c->v_cache, row + ch, dtype);
+    }
+    for (int ch = 0; ch < d_v; ++ch) o[ch] /= l;
+    lse[w] = m + log(l);
+    free(kw);
+    free(s);
   }
   return 0;
 }

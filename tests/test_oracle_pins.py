@@ -364,6 +364,62 @@ def test_augq_matches_library_matmul(oracle, dtype):
     assert np.array_equal(oracle.augq(h, wq, wg, wu, wd, rows=rows), out[rows])
 
 
+# --------------------------------------------------------------------------- half-width keys (K feed-forward + Attend)
+def _kup_case(seed, b, n_q, n_k, n_v, S, d_q, d_k, d_v, dtype="f32"):
+    q = _rand(seed, (b, n_q, d_q), dtype)
+    k = _rand(seed + 1, (b, n_k, S, d_k), dtype)
+    v = _rand(seed + 2, (b, n_v, S, d_v), dtype)
+    w = W.normal(seed + 3, (n_k, d_q, d_k), std=d_k ** -0.5, dtype=dtype)
+    return q, k, v, w
+
+
+def test_kup_with_identity_layer_is_plain_decode(oracle):
+    """W = I (d_q = d_k) leaves the keys as they are: the function must reduce to oracle_decode exactly."""
+    b, n_q, n_k, n_v, S, d = 2, 8, 2, 4, 33, 16
+    q, k, v, _ = _kup_case(301, b, n_q, n_k, n_v, S, d, d, d)
+    w = np.broadcast_to(np.eye(d, dtype=np.float32), (n_k, d, d)).copy()
+    cache = _contig_cache(oracle, k, v, [S, 7])
+    out, lse = oracle.decode_kup(q, w, cache, n_q, n_k, n_v, d, 0.41)
+    ref, lse_ref = oracle.decode(q, cache, n_q, n_k, n_v, d, d, 0.41)
+    assert np.array_equal(out, ref) and np.array_equal(lse, lse_ref)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_kup_matches_numpy_restatement(oracle, dtype):
+    """Widen every key with numpy's matmul, then textbook softmax attention per head (per-head weights, so a
+    transposed or head-shared W would fail; d_q != d_k != d_v so swapped dimensions fail)."""
+    b, n_q, n_k, n_v, S, d_q, d_k, d_v = 2, 8, 2, 4, 29, 12, 6, 10
+    q, k, v, w = _kup_case(311, b, n_q, n_k, n_v, S, d_q, d_k, d_v, dtype)
+    lens = [S, 11]
+    out, lse = oracle.decode_kup(q, w, _contig_cache(oracle, k, v, lens), n_q, n_k, n_v, d_v, 0.3)
+    qf, kf, vf, wf = (W.as_f64(a) for a in (q, k, v, w))
+    for bi in range(b):
+        for h in range(n_q):
+            hk, hv, L = h // (n_q // n_k), h // (n_q // n_v), lens[bi]
+            kw = kf[bi, hk, :L] @ wf[hk].T  # [L, d_q]
+            s = 0.3 * (kw @ qf[bi, h])
+            p = np.exp(s - s.max())
+            assert np.allclose(out[bi, h], (p / p.sum()) @ vf[bi, hv, :L], rtol=0, atol=1e-13)
+            assert abs(lse[bi, h] - (s.max() + math.log(p.sum()))) < 1e-12
+
+
+def test_kup_fold_identity_justifies_scoring_the_half_width_cache(oracle):
+    """<q, W k> = <W^T q, k>: decoding with the layer equals plain decode over the narrow cache with the folded
+    queries q' = W[hk]^T q (here folded in float64 and fed as fp32-exact small integers so that both sides see
+    the same stored values)."""
+    b, n_q, n_k, n_v, S, d_q, d_k, d_v = 1, 4, 2, 2, 21, 8, 4, 8
+    g = np.random.Generator(np.random.Philox(key=321))
+    q = g.integers(-3, 4, size=(b, n_q, d_q)).astype(np.float32)
+    w = g.integers(-2, 3, size=(n_k, d_q, d_k)).astype(np.float32)
+    k = g.integers(-3, 4, size=(b, n_k, S, d_k)).astype(np.float32) / 4
+    v = _rand(322, (b, n_v, S, d_v))
+    cache = _contig_cache(oracle, k, v, [S])
+    out, lse = oracle.decode_kup(q, w, cache, n_q, n_k, n_v, d_v, 0.125)
+    folded = np.stack([[w[h // (n_q // n_k)].T @ q[bi, h] for h in range(n_q)] for bi in range(b)]).astype(np.float32)
+    ref, lse_ref = oracle.decode(folded, cache, n_q, n_k, n_v, d_k, d_v, 0.125)
+    assert np.allclose(out, ref, rtol=0, atol=1e-13) and np.allclose(lse, lse_ref, rtol=0, atol=1e-13)
+
+
 # --------------------------------------------------------------------------- selective V fetching
 def test_topk_keeps_everything_when_k_covers_the_sequence(oracle):
     n_q, n_k, n_v, d, S = 8, 2, 4, 16, 40
