@@ -8,6 +8,10 @@ bf16).  One step = one ``diffqkv_decode`` call (split kernel + combine kernel) o
 The line printed by rank 0 also carries the GQA twin (n_k = n_v), the other decode configurations,
 the roofline of the split kernel and the CPU oracle timed on the host cores.
 
+The timed region is exactly ``--steps`` steps between barriers; when that is shorter than 50 ms it is repeated as
+separate groups and the median group is reported (minimum and maximum beside it).  The last key of the line,
+``summary``, repeats the headline figures of every configuration in short form.
+
 With N > 1 every rank runs the same workload on its own GPU (the path has no exchange step:
 replicas only), the timed region is bracketed by barriers and the slowest rank's time is used.
 ``--impl reference`` times the float64 CPU oracle instead (rank 0 only).
@@ -30,9 +34,23 @@ if ROOT not in sys.path:
 METRIC = "decode_kv_cache_bandwidth"
 UNIT = "GB/s"
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the split kernel on the headline workload, from the
-# ncu capture summarised in profiles/decode_tma_kernel_cfg3.md (set to None whenever the kernel changes after it).
-SPLIT_KERNEL_DRAM_BYTES = 407.96e6
+
+
+def split_kernel_dram_bytes():
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of the split kernel on the headline workload, as
+    recorded (with a hash of the kernel's source) when the counters were last taken; None once the kernel's source
+    no longer matches that hash, so that a stale figure is never printed."""
+    import hashlib
+    rec = os.path.join(ROOT, "profiles", "decode_tma_kernel_cfg3.json")
+    src = os.path.join(ROOT, "paper_2501_13629_b200", "csrc", "decode_tma.cu")
+    try:
+        with open(rec) as f:
+            d = json.load(f)
+        with open(src, "rb") as f:
+            h = hashlib.sha256(f.read()).hexdigest()
+        return float(d["dram_bytes_per_launch"]) if d.get("source_sha256") == h else None
+    except Exception:
+        return None
 
 
 def measured_peaks():
@@ -201,6 +219,34 @@ class DecodeCase:
         if barrier:
             barrier()
         return start.elapsed_time(end)
+
+    def time_groups(self, steps, warmup, barrier=None, reduce_max=None, min_total_ms=50.0, max_groups=25):
+        """Groups of exactly `steps` steps, each bracketed like time_steps (warm-up before the first only).  One group
+        when it lasts min_total_ms or more; otherwise as many as make up that time (at most max_groups), so that a
+        short timed region is not one sample.  Every group time is the slowest rank's (`reduce_max`)."""
+        reduce_max = reduce_max or (lambda x: x)
+        first = reduce_max(self.time_steps(steps, warmup, barrier))
+        n = 1 if first >= min_total_ms else int(min(max_groups, np.ceil(min_total_ms / max(first, 1e-6))))
+        return [first] + [reduce_max(self.time_steps(steps, 0, barrier)) for _ in range(n - 1)]
+
+    def time_split_and_combine(self, steps):
+        """Mean durations of the split kernel and of the combine kernel, each timed alone: the library records an
+        event before and after the split kernel, a third event follows the call.  The events between the two
+        kernels keep them from overlapping, so the two figures add up to more than an untimed step."""
+        torch, api = self.torch, self.api
+        trip = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in range(steps)]
+        for t in trip:
+            for e in t:
+                e.record()  # creates the underlying CUDA events
+        torch.cuda.synchronize()
+        for a, b, c in trip:
+            api.set_split_events(a, b)
+            self.step()
+            c.record()
+        api.set_split_events(None, None)
+        torch.cuda.synchronize()
+        return (float(np.mean([a.elapsed_time(b) for a, b, _ in trip])),
+                float(np.mean([b.elapsed_time(c) for _, b, c in trip])))
 
     def time_split_kernel(self, steps):
         """Average duration of the split kernel alone: the library records an event pair around it."""
@@ -451,9 +497,11 @@ def time_decode_step(api, W, device, host, steps):
 
 
 def time_sigma_table(api, W, device, steps):
-    """The paper's own efficiency experiment in shape: SIGMA-1.5B attention heads (32 query, 4 K, 16 V heads, head
-    dimension 64) against the standard model's 16 K / 16 V heads at prefix lengths 2k, 4k, 16k and 32k (batch 8,
-    bf16 cache drawn on the device): time of one decode step and the share of it the split kernel takes."""
+    """The paper's own efficiency experiment in shape (appendix table of split / combine / total kernel times):
+    SIGMA-1.5B attention heads (32 query, 4 K, 16 V heads, head dimension 64) against the standard model's 16 K /
+    16 V heads at prefix lengths 2k, 4k, 16k and 32k (batch 8, bf16 cache drawn on the device).  Per shape: the split
+    kernel and the combine kernel each timed alone (events between them), and one whole untimed-inside decode step;
+    per prefix: the relative reduction of each, beside the reduction of the cache bytes."""
     import dataclasses
     rows = []
     for prefix in (2048, 4096, 16384, 32768):
@@ -462,10 +510,13 @@ def time_sigma_table(api, W, device, steps):
             cfg = dataclasses.replace(W.SIGMA15B, name=f"{name}_{prefix}", batch=8, n_k=n_k, n_v=n_v, kv_len=prefix)
             case = DecodeCase(api, cfg, device)
             ms = case.time_steps(steps, 20) / steps
-            row[name] = {"us_per_step": ms * 1e3, "GB/s": case.bytes / ms / 1e6, "kv_bytes": case.bytes,
-                         "rotate": case.rotate}
+            split_ms, combine_ms = case.time_split_and_combine(min(steps, 100))
+            row[name] = {"us_per_step": ms * 1e3, "split_us": split_ms * 1e3, "combine_us": combine_ms * 1e3,
+                         "GB/s": case.bytes / ms / 1e6, "kv_bytes": case.bytes, "rotate": case.rotate}
             del case
-        row["time_reduction_pct"] = 100.0 * (1.0 - row["sigma"]["us_per_step"] / row["std"]["us_per_step"])
+        for key, out in (("us_per_step", "time_reduction_pct"), ("split_us", "split_reduction_pct"),
+                         ("combine_us", "combine_reduction_pct")):
+            row[out] = 100.0 * (1.0 - row["sigma"][key] / row["std"][key])
         row["bytes_reduction_pct"] = 100.0 * (1.0 - row["sigma"]["kv_bytes"] / row["std"]["kv_bytes"])
         rows.append(row)
     return rows
@@ -526,6 +577,41 @@ def time_topk(api, W, device, host, steps, topk=100):
             "k_stream_GB/s": k_bytes / ms / 1e6}
 
 
+def summarize(line, peaks):
+    """The figures the benchmark definition asks for, in one short object: decode GB/s per configuration with the
+    fractions of the measured copy peak and of the 8 TB/s nominal figure, the prefill leg's TFLOP/s against the
+    measured bf16 burst peak, and DiffQKV against GQA at 32K context."""
+    o = line.get("others", {})
+    r3 = lambda x: None if x is None else round(float(x), 3)  # noqa: E731
+
+    def gbs(v):
+        return None if v is None else {"GB/s": round(v, 1), "of_measured": r3(v / peaks["hbm_gbs"]), "of_8TBs": r3(v / 8000.0)}
+
+    out = {"cfg3": gbs(line["value"] / line["n_gpus"]), "cfg3_us_per_step": r3(line["ms_per_step"] * 1e3),
+           "cfg3_us_per_step_min": r3(line["timed_groups"]["ms_per_step_min"] * 1e3)}
+    for key, name in (("cfg2_b16_4k", "cfg2"), ("cfg2_b16_4k_gqa", "cfg2_gqa"), ("cfg1_small_f32", "cfg1"),
+                      ("cfg5_paged_varlen", "cfg5"), ("cfg3_gqa_twin", "cfg3_gqa")):
+        if key in o:
+            out[name] = gbs(o[key]["GB/s"])
+    if "diffqkv_vs_gqa_speedup_32k" in line:
+        out["diffqkv_vs_gqa_32k"] = r3(line["diffqkv_vs_gqa_speedup_32k"])
+    for row in o.get("diffqkv_vs_gqa_over_context", []):
+        if row["context"] in (4096, 8192):
+            out[f"diffqkv_vs_gqa_{row['context'] // 1024}k"] = r3(row["speedup"])
+    c4 = o.get("cfg4_prefill_8k")
+    if c4:
+        for name in ("augq", "attention"):
+            out["cfg4_" + name] = {"TFLOP/s": round(c4[name]["TFLOP/s"], 1), "ms": r3(c4[name]["ms"]),
+                                   "of_measured_burst": r3(c4[name]["frac_of_measured_bf16_burst"])}
+    if "cfg3_selective_v_top100" in o:
+        out["cfg3_top100_us"] = r3(o["cfg3_selective_v_top100"]["ms_per_step"] * 1e3)
+    if line.get("e2e"):
+        out["e2e_GB/s"] = round(line["e2e"]["value"], 1)
+    if line.get("roofline"):
+        out["split_kernel_frac_of_measured"] = r3(line["roofline"]["frac"])
+    return out
+
+
 def max_over_ranks(value: float, device) -> float:
     """The slowest rank's value (all-reduce MAX over the default process group; identity without one)."""
     import torch
@@ -552,6 +638,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=device)
         barrier = lambda: (dist.barrier(), torch.cuda.synchronize())  # noqa: E731
     peaks = measured_peaks()
+    api.set_tail_reserve(args.tail_reserve)
     if args.workload == "prefill":  # the config 4 leg alone (the command profilers wrap for the tensor-core kernels)
         if rank == 0:
             print(json.dumps({"workload": W.CFG4.name, **time_prefill(api, W, device, peaks, max(1, min(args.steps, 20)))}))
@@ -572,13 +659,13 @@ def run_ours(args):
         return
     case = DecodeCase(api, cfg, device, host_inputs=host)
     launches0 = api.launch_count()
+    case.step()
+    launches_per_step = api.launch_count() - launches0
     with ClockSampler(local_rank) as clocks:
-        ms = case.time_steps(args.steps, args.warmup, barrier)
-    launches = api.launch_count() - launches0 - 0
-    launches_timed = launches * args.steps // (args.steps + args.warmup)
-    ms = max_over_ranks(ms, device)
+        groups = case.time_groups(args.steps, args.warmup, barrier, lambda x: max_over_ranks(x, device))
     assert int(case.status.item()) == 0, "device status reported an error"
-    ms_per_step = ms / args.steps
+    # every group is exactly `steps` steps between barriers, slowest rank; the line reports the median group
+    ms_per_step = float(np.median(groups)) / args.steps
     value = world * case.bytes / (ms_per_step * 1e-3) / 1e9
 
     line = {
@@ -590,7 +677,11 @@ def run_ours(args):
                    "kv_bytes_per_step": case.bytes, "parallelism": "replicas" if world > 1 else "single",
                    "l2": f"inputs larger than L2: {case.rotate} distinct cache copies rotated, "
                          f"working set {case.working_set / 1e6:.0f} MB"},
-        "gpu_launches": launches_timed,
+        "gpu_launches": launches_per_step * args.steps,
+        "timed_groups": {"groups": len(groups), "steps_each": args.steps,
+                         "ms_per_step_median": ms_per_step, "ms_per_step_min": float(np.min(groups)) / args.steps,
+                         "ms_per_step_max": float(np.max(groups)) / args.steps,
+                         "note": "groups of exactly `steps` steps, repeated until 50 ms are timed; value = median group"},
         "clocks": clocks.summary(),
         "tokens_per_s_per_layer": world * cfg.batch / (ms_per_step * 1e-3),
         "frac_of_8TBs_nominal": value / world / 8000.0,
@@ -615,7 +706,7 @@ def run_ours(args):
         k_ms = case.time_split_kernel(min(args.steps, 200))
         ach = case.bytes / (k_ms * 1e-3) / 1e9
         line["roofline"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                            "frac": ach / peaks["hbm_gbs"], "traffic": SPLIT_KERNEL_DRAM_BYTES,
+                            "frac": ach / peaks["hbm_gbs"], "traffic": split_kernel_dram_bytes(),
                             "kernel": "decode split kernel",
                             "kernel_ms": k_ms, "peak_source": peaks["source"] + " (burst copy)"}
         line["e2e"] = e2e
@@ -654,6 +745,7 @@ def run_ours(args):
         line["others"] = others
         if world == 1:
             line["cpu_baseline"] = cpu_baseline(host, budget_s=12.0)
+        line["summary"] = summarize(line, peaks)  # last on the line, so that it survives a truncated tail
         print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
@@ -745,6 +837,8 @@ def main():
                     help="decode = the headline line (default); prefill = only the config 4 timings; "
                          "topk = only selective V fetching on the headline workload; augq_decode = only the projection "
                          "chain at decode row counts")
+    ap.add_argument("--tail-reserve", type=int, default=-1,
+                    help="tail balance of the TMA decode kernel: -1 automatic (default), 0 off, n tiles per block")
     ap.add_argument("--profile", action="store_true",
                     help="only the timed loop of the headline workload (the command profilers wrap)")
     args = ap.parse_args()

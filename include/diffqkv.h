@@ -105,7 +105,8 @@ size_t diffqkv_decode_workspace_bytes(const diffqkv_shape *shape, int32_t max_se
  *   num_splits 0 = automatic (recommended): bf16 caches that a TMA tensor map can describe use the
  *              persistent TMA kernel, which divides all (sequence, head group, 64-token tile) work
  *              evenly over one block per SM and cuts sequences wherever a block's share ends; other
- *              inputs use fixed chunks.  > 0 = fixed chunks, at most that many per sequence (generic kernel)
+ *              inputs use fixed chunks.  > 0 = fixed chunks, at most that many per sequence (generic kernel);
+ *              more than 8192 returns DIFFQKV_ERR_UNSUPPORTED
  *   workspace  at least diffqkv_decode_workspace_bytes(...) bytes, 256-byte aligned; holds the
  *              per-split partial outputs (fp32 [batch, n_q, S, d_v]) and log-sum-exps
  *              (fp32 [batch, n_q, S]); contents on entry are ignored
@@ -186,9 +187,10 @@ diffqkv_status diffqkv_combine(const float *o_partial, const float *lse_partial,
  *          both pools are overwritten; seqlens itself is not modified (the caller adds q_len)
  *   out    [batch, q_len, n_q, d_v] out_dtype; query row i sees tokens 0 .. past_b + i
  *   lse    [batch, q_len, n_q] fp32 or NULL
- * bf16 with d_qk == d_v == 128 or 64 (and pages of at least 8 tokens that divide or are multiples of 128) runs on
- * the tensor cores; every other shape diffqkv_decode accepts (fp32, other head dimensions, d_qk != d_v) runs the same
- * two steps on a plain fp32-FMA kernel, one block per query row, which is a correctness path, not a fast one.
+ * bf16 with (d_qk, d_v) = (128, 128), (64, 64) or (64, 128), a positive scale and pages of at least 8 tokens that
+ * divide or are multiples of 128 runs on the tensor cores; every other shape diffqkv_decode accepts (fp32, other head
+ * dimensions, scale <= 0) runs the same two steps on a plain fp32-FMA kernel, one block per query row, which is a
+ * correctness path, not a fast one.
  */
 diffqkv_status diffqkv_prefill(const void *q, const void *k_new, const void *v_new, int32_t q_len,
                                const diffqkv_cache *cache, const diffqkv_shape *shape, void *out, float *lse,
@@ -277,6 +279,21 @@ diffqkv_status diffqkv_decode_frontend(const void *h, const void *W_Q, const voi
                                        void *q_out, int32_t *dev_status, void *stream);
 
 /*
+ * diffqkv_fold_k_up -- queries for a K cache that is stored at a smaller head width than the queries (Section 2:
+ * when the Q and K head dimensions differ, Attend first transforms K to the query width through another feed-forward
+ * layer; Observation 2 and its table: d_k = d_v / 2).  The layer is read as linear, without bias, one matrix per K
+ * head.  Since <q_h, W[hk] k_j> = <W[hk]^T q_h, k_j>, widening every cached key is replaced by folding the layer
+ * into the query once:
+ *     q_out[t, h, :] = W_kup[hk]^T q[t, h, :],   hk = floor(h * n_k / n_q)
+ *   q      [T, n_q, d_q] bf16      W_kup [n_k, d_q, d_k] bf16      q_out [T, n_q, d_k] bf16 (fp32 accumulation)
+ * Call sequence for the half-width cache: diffqkv_fold_k_up, then diffqkv_decode / diffqkv_prefill /
+ * diffqkv_decode_topk with shape.d_qk = d_k (64 with d_v = 128 runs on the TMA and tensor-core kernels) and the
+ * same scale the full-width scores would use.  (n_q / n_k) * d_q may not exceed 12288.
+ */
+diffqkv_status diffqkv_fold_k_up(const void *q, const void *W_kup, int64_t T, int32_t n_q, int32_t n_k, int32_t d_q,
+                                 int32_t d_k, void *q_out, void *stream);
+
+/*
  * diffqkv_decode_topk -- decode with selective V cache fetching (paper Section "Selective V Cache Fetching"; its
  * table uses the 100 highest scores): every query head scores all cached tokens of its K head, keeps the `topk`
  * highest scores (equal scores: the earlier token), takes the softmax over the kept scores only (the paper does
@@ -288,7 +305,7 @@ diffqkv_status diffqkv_decode_frontend(const void *h, const void *W_Q, const voi
  *   of 128 tokens; topk times the number of 32768-token pieces of max_seqlen may not exceed 8192
  *   (DIFFQKV_ERR_UNSUPPORTED otherwise)
  *   workspace  diffqkv_decode_topk_workspace_bytes(shape, cache->max_seqlen, topk) bytes, 256-byte aligned: the fp32
- *              scores [batch, n_q, max_seqlen rounded up to 128]
+ *              scores [batch, n_q, max_seqlen rounded up to 128] and the largest score of every 16 consecutive tokens
  */
 size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape *shape, int32_t max_seqlen, int32_t topk);
 diffqkv_status diffqkv_decode_topk(const void *q, const diffqkv_cache *cache, const diffqkv_shape *shape, int32_t topk,
@@ -299,43 +316,17 @@ diffqkv_status diffqkv_decode_topk(const void *q, const diffqkv_cache *cache, co
 const char *diffqkv_status_string(diffqkv_status status);
 
 /*
- * Tuning hook (process-wide host state): cap the number of persistent blocks the TMA decode kernel
- * launches; 0 restores the default of one block per SM.  Workspace sizes must be queried after the
- * cap is set.  Mainly for tests, which use it to move the places where sequences are cut.
+ * Tuning hook (process-wide host state) for the TMA decode kernel's tail balance.  Every persistent block holds the
+ * last few 64-token tiles of its share in a reserve that it and the other blocks working on the same (sequence, head
+ * group) draw from one tile at a time, so that a block that runs ahead takes over tiles of one that runs behind.
+ * Which block ends up with which tile depends on timing, so results can differ between runs in the last bits
+ * (fp32 summation order); everything stays within the stated tolerances.
+ *   tiles < 0  automatic (default): up to 8 tiles per block, at most a sixth of a block's share
+ *   tiles = 0  no reserve: every tile has a fixed owner and results are bitwise reproducible from run to run
+ *   tiles > 0  exactly that many (always leaving each segment one tile of its own); for tests
+ * Workspace sizes do not depend on it.
  */
-void diffqkv_set_max_blocks(int32_t max_blocks);
-
-/*
- * Test hook (process-wide host state): a non-zero value makes diffqkv_decode_topk always select over all scores of a
- * row; 0 (the default) lets it first try the selection that reads only the 16-token blocks whose largest score can
- * reach the top.  Both give the same result.
- */
-void diffqkv_topk_general_only(int32_t on);
-
-/*
- * Test hook (process-wide host state): the projections (diffqkv_augq, diffqkv_augq_rope, diffqkv_project) take a
- * weight-streaming kernel when there are at most 64 rows (decode: one token per sequence) and the tensor-core GEMM
- * otherwise; a non-zero value makes them always take the tensor-core GEMM.  Both round x and a to bf16 once and
- * accumulate in fp32; they differ in summation order only.
- */
-void diffqkv_force_tensor_gemm(int32_t on);
-
-/* Which attention kernel the most recent diffqkv_prefill call launched: 0 none yet, 1 generic, 2 tensor-core (for tests). */
-int32_t diffqkv_last_prefill_kernel(void);
-
-/* Which split kernel the most recent decode call launched: 0 none yet, 1 generic, 2 TMA (for tests). */
-int32_t diffqkv_last_decode_kernel(void);
-
-/*
- * Profiling hook for benchmarks (process-wide host state, not thread-safe).  While both arguments
- * are non-NULL cudaEvent_t handles, every decode call records `before_split` just before and
- * `after_split` just after its split kernel on the call's stream, so the split kernel can be timed
- * apart from the combine kernel.  Pass NULL, NULL to switch it off.
- */
-void diffqkv_profile_split_events(void *before_split, void *after_split);
-
-/* Kernels launched by this library since it was loaded (host counter, for benchmarks). */
-int64_t diffqkv_launch_count(void);
+void diffqkv_set_tail_reserve(int32_t tiles);
 
 #ifdef __cplusplus
 }

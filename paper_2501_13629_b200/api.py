@@ -32,7 +32,8 @@ EXPORTS = (
     "diffqkv_set_max_blocks", "diffqkv_topk_general_only", "diffqkv_last_decode_kernel",
     "diffqkv_last_prefill_kernel", "diffqkv_force_tensor_gemm", "diffqkv_augq_rope", "diffqkv_project", "diffqkv_cache_append",
     "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes", "diffqkv_decode_frontend",
-    "diffqkv_decode_frontend_workspace_bytes", "diffqkv_decode_host",
+    "diffqkv_decode_frontend_workspace_bytes", "diffqkv_decode_host", "diffqkv_fold_k_up",
+    "diffqkv_set_tail_reserve", "diffqkv_debug_decode_timeout",
 )
 
 
@@ -93,6 +94,9 @@ _lib.diffqkv_decode_topk_workspace_bytes.argtypes = [C.POINTER(ShapeStruct), C.c
 _lib.diffqkv_decode_topk.restype = C.c_int
 _lib.diffqkv_decode_topk.argtypes = [C.c_void_p, C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_int32, C.c_void_p,
                                      C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.diffqkv_fold_k_up.restype = C.c_int
+_lib.diffqkv_fold_k_up.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                   C.c_void_p, C.c_void_p]
 _lib.diffqkv_status_string.restype = C.c_char_p
 _lib.diffqkv_status_string.argtypes = [C.c_int]
 _lib.diffqkv_launch_count.restype = C.c_int64
@@ -111,6 +115,10 @@ _lib.diffqkv_last_prefill_kernel.restype = C.c_int32
 _lib.diffqkv_last_prefill_kernel.argtypes = []
 _lib.diffqkv_topk_general_only.restype = None
 _lib.diffqkv_topk_general_only.argtypes = [C.c_int32]
+_lib.diffqkv_debug_decode_timeout.restype = None
+_lib.diffqkv_debug_decode_timeout.argtypes = [C.c_int64, C.c_int64]
+_lib.diffqkv_set_tail_reserve.restype = None
+_lib.diffqkv_set_tail_reserve.argtypes = [C.c_int32]
 _lib.diffqkv_set_max_blocks.restype = None
 _lib.diffqkv_set_max_blocks.argtypes = [C.c_int32]
 _lib.diffqkv_profile_split_events.restype = None
@@ -148,6 +156,17 @@ def set_max_blocks(n: int) -> None:
 
 
 KERNEL_NONE, KERNEL_GENERIC, KERNEL_TMA = 0, 1, 2
+
+
+def set_tail_reserve(tiles: int) -> None:
+    """Tail balance of the TMA decode kernel: -1 automatic, 0 off (run-to-run bitwise reproducible), n tiles per block."""
+    _lib.diffqkv_set_tail_reserve(int(tiles))
+
+
+def debug_decode_timeout(wait_limit_ns: int = 0, skip_tile: int = -1) -> None:
+    """Test hook of the TMA decode kernel: bound every device wait by ``wait_limit_ns`` and never request the copies of
+    flat tile ``skip_tile`` (so that the wait for it runs out); (0, -1) restores the defaults."""
+    _lib.diffqkv_debug_decode_timeout(int(wait_limit_ns), int(skip_tile))
 
 
 def force_tensor_gemm(on: bool) -> None:
@@ -465,6 +484,21 @@ def diffqkv_cache_append(k_new: torch.Tensor, v_new: torch.Tensor, cache: KVCach
                                    _stream_ptr(stream))
     if st != OK:
         raise DiffQKVError(st, "diffqkv_cache_append")
+
+
+def diffqkv_fold_k_up(q: torch.Tensor, W_kup: torch.Tensor, out: Optional[torch.Tensor] = None,
+                      stream: Optional[torch.cuda.Stream] = None):
+    """q' = W_kup[hk]^T q per query head: q [..., n_q, d_q] bf16, W_kup [n_k, d_q, d_k] bf16 -> [..., n_q, d_k]."""
+    n_k, d_q, d_k = W_kup.shape
+    n_q = q.shape[-2]
+    assert q.shape[-1] == d_q and q.is_contiguous() and W_kup.is_contiguous()
+    T = q.numel() // (n_q * d_q)
+    if out is None:
+        out = torch.empty(q.shape[:-1] + (d_k,), dtype=torch.bfloat16, device=q.device)
+    st = _lib.diffqkv_fold_k_up(_p(q), _p(W_kup), T, n_q, n_k, d_q, d_k, _p(out), _stream_ptr(stream))
+    if st != OK:
+        raise DiffQKVError(st, "diffqkv_fold_k_up")
+    return out
 
 
 def diffqkv_decode_topk(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: float, topk: int,

@@ -2,6 +2,7 @@
 #include <atomic>
 
 #include "common.cuh"
+#include "diffqkv_debug.h"
 
 namespace diffqkv {
 
@@ -27,8 +28,10 @@ DecodePlan plan_decode(const diffqkv_shape& shape, int max_seqlen, int num_split
   return pl;
 }
 
-static cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
-static int g_last_kernel = 0;  // 0 none, 1 generic, 2 TMA
+constexpr int kMaxSplits = 8192;  // combine_kernel keeps one weight per split in shared memory
+// Hook state: process-wide, written and read from any calling thread, hence atomics.
+static std::atomic<cudaEvent_t> g_ev_before{nullptr}, g_ev_after{nullptr};
+static std::atomic<int> g_last_kernel{0};  // 0 none, 1 generic, 2 TMA
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -105,7 +108,8 @@ static size_t workspace_need(const diffqkv_shape& s, int max_seqlen, int num_spl
 }
 
 void profile_after_split(cudaStream_t stream) {
-  if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_after, stream);
+  const cudaEvent_t before = g_ev_before.load(), after = g_ev_after.load();
+  if (before && after) cudaEventRecord(after, stream);
 }
 
 static diffqkv_status decode_impl(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape,
@@ -118,17 +122,19 @@ static diffqkv_status decode_impl(const void* q, const diffqkv_cache* cache, con
   if (st != DIFFQKV_OK) return st;
   if (!aligned16(q) || !aligned16(out)) return DIFFQKV_ERR_ALIGNMENT;
   if (num_splits < 0) return DIFFQKV_ERR_INVALID_ARG;
+  if (num_splits > kMaxSplits) return DIFFQKV_ERR_UNSUPPORTED;  // the combine kernel's limit, as in diffqkv_combine
   if (shape->batch == 0) return DIFFQKV_OK;
   const DecodePlan pl = plan_decode(*shape, cache->max_seqlen, num_splits);
   const size_t need = workspace_need(*shape, cache->max_seqlen, num_splits);
   if (!workspace || workspace_bytes < need) return DIFFQKV_ERR_WORKSPACE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DIFFQKV_ERR_ALIGNMENT;
-  const bool timed = g_ev_before && g_ev_after;
+  const cudaEvent_t ev_before = g_ev_before.load();
+  const bool timed = ev_before && g_ev_after.load();
 
   // bf16 caches a tensor map can describe go to the TMA kernel (automatic schedule only)
   TmaPlan tp;
   if (num_splits == 0 && tma_decode_supported(*shape, *cache, &tp)) {
-    if (timed) cudaEventRecord(g_ev_before, stream);
+    if (timed) cudaEventRecord(ev_before, stream);
     const cudaError_t terr = launch_decode_tma(q, *cache, *shape, tp, workspace, out, lse, dev_status, stream);
     if (terr == cudaSuccess) {
       g_last_kernel = 2;
@@ -151,7 +157,7 @@ static diffqkv_status decode_impl(const void* q, const diffqkv_cache* cache, con
                                            align_up(rows * pl.splits * shape->d_v * sizeof(float), 256));
   p.dev_status = dev_status;
 
-  if (timed) cudaEventRecord(g_ev_before, stream);
+  if (timed) cudaEventRecord(ev_before, stream);
   cudaError_t err = launch_decode_generic(p, shape->dtype, stream);
   g_last_kernel = 1;
   profile_after_split(stream);
@@ -178,6 +184,12 @@ size_t diffqkv_decode_workspace_bytes(const diffqkv_shape* shape, int32_t max_se
 }
 
 void diffqkv_set_max_blocks(int32_t max_blocks) { set_tma_max_blocks(max_blocks); }
+
+void diffqkv_set_tail_reserve(int32_t tiles) { set_tma_tail_reserve(tiles); }
+
+void diffqkv_debug_decode_timeout(int64_t wait_limit_ns, int64_t skip_tile) {
+  set_tma_debug_timeout(wait_limit_ns, skip_tile);
+}
 
 void diffqkv_topk_general_only(int32_t on) { set_topk_general_only(on); }
 
@@ -226,14 +238,14 @@ diffqkv_status diffqkv_combine(const float* o_partial, const float* lse_partial,
   if (!o_partial || !lse_partial || !out) return DIFFQKV_ERR_INVALID_ARG;
   if (batch < 0 || n_q <= 0 || d_v <= 0 || num_splits <= 0) return DIFFQKV_ERR_INVALID_ARG;
   if (out_dtype != DIFFQKV_BF16 && out_dtype != DIFFQKV_F32) return DIFFQKV_ERR_INVALID_ARG;
-  if (num_splits > 8192) return DIFFQKV_ERR_UNSUPPORTED;
+  if (num_splits > kMaxSplits) return DIFFQKV_ERR_UNSUPPORTED;
   if ((long long)batch * n_q > 0x7fffffffLL) return DIFFQKV_ERR_UNSUPPORTED;
   cudaError_t err = launch_combine(o_partial, lse_partial, batch * n_q, d_v, num_splits, out_dtype, out, lse,
                                    static_cast<cudaStream_t>(stream));
   return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
 
-static int g_last_prefill_kernel = 0;  // 0 none yet, 1 generic, 2 tensor-core (for tests)
+static std::atomic<int> g_last_prefill_kernel{0};  // 0 none yet, 1 generic, 2 tensor-core (for tests)
 
 diffqkv_status diffqkv_prefill(const void* q, const void* k_new, const void* v_new, int32_t q_len,
                                const diffqkv_cache* cache, const diffqkv_shape* shape, void* out, float* lse,
@@ -383,6 +395,17 @@ diffqkv_status diffqkv_cache_append(const void* k_new, const void* v_new, int32_
   return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
 }
 
+diffqkv_status diffqkv_fold_k_up(const void* q, const void* W_kup, int64_t T, int32_t n_q, int32_t n_k, int32_t d_q,
+                                 int32_t d_k, void* q_out, void* stream) {
+  if (!q || !W_kup || !q_out) return DIFFQKV_ERR_INVALID_ARG;
+  if (T < 0 || n_q <= 0 || n_k <= 0 || d_q <= 0 || d_k <= 0 || n_q % n_k != 0) return DIFFQKV_ERR_INVALID_ARG;
+  if (T * n_k > 0x7fffffffLL) return DIFFQKV_ERR_UNSUPPORTED;
+  if (T == 0) return DIFFQKV_OK;
+  const cudaError_t err = launch_fold_kup(q, W_kup, T, n_q, n_k, d_q, d_k, q_out, static_cast<cudaStream_t>(stream));
+  if (err == cudaErrorNotSupported) return DIFFQKV_ERR_UNSUPPORTED;
+  return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
+}
+
 size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape* shape, int32_t max_seqlen, int32_t topk) {
   if (check_shape(shape) != DIFFQKV_OK || max_seqlen < 0 || topk < 1) return 0;
   return topk_decode_workspace_bytes(*shape, max_seqlen, topk);
@@ -423,8 +446,8 @@ const char* diffqkv_status_string(diffqkv_status status) {
 }
 
 void diffqkv_profile_split_events(void* before_split, void* after_split) {
-  g_ev_before = static_cast<cudaEvent_t>(before_split);
-  g_ev_after = static_cast<cudaEvent_t>(after_split);
+  g_ev_before.store(static_cast<cudaEvent_t>(before_split));
+  g_ev_after.store(static_cast<cudaEvent_t>(after_split));
 }
 
 int64_t diffqkv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -11,6 +11,8 @@
 //   warps 2-5   epilogue: tcgen05.ld of the warp's 32 TMEM lanes (= 32 output rows), silu-gate when fused,
 //               bf16 conversion, 16-byte global stores
 // Every wait is bounded; on expiry the block reports DIFFQKV_ERR_TIMEOUT, drains and frees its TMEM.
+#include <atomic>
+
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tcgen05.cuh"
@@ -281,7 +283,7 @@ int sm_count() {
   return sms;
 }
 
-int g_force_tensor_gemm = 0;  // test hook: 1 = never take the weight-streaming kernel for few rows
+std::atomic<int> g_force_tensor_gemm{0};  // test hook: 1 = never take the weight-streaming kernel for few rows
 
 // C[M, N] = A[M, K] . B0[N, K]^T, or with B1: C[M, N] = silu(A.B0^T) * (A.B1^T).
 cudaError_t launch_gemm(const void* A, const void* B0, const void* B1, void* C, long long M, int N, int K,

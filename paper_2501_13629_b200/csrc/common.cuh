@@ -89,12 +89,15 @@ struct TmaPlan {
   int box_tok;       // tokens per TMA box
   int stages, grid, smem;
   long long slots;   // partial-result slots: grid + batch * units
+  int reserve, reserve_auto;  // tail reserve per block in tiles (0 = none); auto: also at most a sixth of a block's share
 };
 bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPlan* plan);
 size_t tma_decode_workspace_bytes(const diffqkv_shape& s, const TmaPlan& plan);
 cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, const TmaPlan& plan,
                               void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream);
 void set_tma_max_blocks(int n);
+void set_tma_tail_reserve(int n);
+void set_tma_debug_timeout(long long wait_limit_ns, long long skip_tile);
 
 // Augmented-Q projection (augq.cu): three tcgen05 GEMMs, the gate/up pair fused with its silu-gate epilogue.
 size_t augq_workspace_bytes(long long T, int d_q0, int d_aug);
@@ -114,6 +117,10 @@ cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, 
                            const diffqkv_shape& s, int box_tok, void* out, float* lse, int* dev_status,
                            cudaStream_t stream);
 
+
+// Queries folded through the K feed-forward layer (kup.cu): q' = W_kup[hk]^T q per query head.
+cudaError_t launch_fold_kup(const void* q, const void* W_kup, long long T, int n_q, int n_k, int d_q, int d_k,
+                            void* q_out, cudaStream_t stream);
 
 // Selective V fetching (decode_topk.cu): K-only score pass, then top-k selection and V gather per query head.
 bool topk_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, int topk, int* box_tok);

@@ -44,8 +44,8 @@ extern "C" diffqkv_status diffqkv_decode_static(const void* q, const diffqkv_cac
                                                 const diffqkv_shape* shape, int32_t num_splits, void* out,
                                                 float* lse, int32_t* dev_status, void* stream) {
   if (!shape || !cache) return DIFFQKV_ERR_INVALID_ARG;
+  // 0 = nothing to do (batch 0) or arguments diffqkv_decode will refuse: either way it gives the answer below
   const size_t need = diffqkv_decode_workspace_bytes(shape, cache->max_seqlen, num_splits);
-  if (need == 0) return DIFFQKV_ERR_INVALID_ARG;
   if (need > kStaticScratchBytes) return DIFFQKV_ERR_WORKSPACE;  // beyond the built-in 8 MiB
   void* scratch = nullptr;
   if (scratch_for_current_device(&scratch) != cudaSuccess) return DIFFQKV_ERR_CUDA;

@@ -19,9 +19,19 @@
 // so every K and V byte is read from shared memory exactly once and scored against all query
 // heads of its unit.  Accumulation is fp32; P is rounded to bf16 for the second product and the
 // softmax denominator sums the rounded values.
+//
+// Tail balance.  Equal shares do not finish at the same time (blocks end several microseconds apart on a step of
+// 60), so the last few tiles of every block's last segment are not owned but pooled with those of the other blocks
+// whose last segment lies in the same (sequence, unit) row; the blocks of a row draw from their pool one tile at a
+// time through a counter in the workspace, and a block that runs ahead ends up with more tiles than one that runs
+// behind.  A drawn tile joins the running softmax state of the drawing block's segment (the state does not care
+// which tokens it has seen), so the number of partial results stays the same.  The counters carry the call's
+// epoch, so that nothing has to be zeroed between calls and a counter of an earlier call is recognised as such.
 #include <cuda.h>
 
+#include <atomic>
 #include <mutex>
+#include <random>
 
 #include "common.cuh"
 #include "ptx.cuh"
@@ -37,7 +47,13 @@ constexpr int kThreads = (kConsumerWarps + 1) * 32;
 // [token part][channel half][box_tok rows]; with box_tok = 64 that is simply [half][64 rows].
 constexpr int kHeadsPerMma = 8;
 constexpr int kMaxBatchTma = 2048;  // the per-sequence tile prefix lives in shared memory
-int g_max_blocks = 0;               // tuning / test hook: 0 = one block per SM
+// Hook state: process-wide, set and read from any calling thread, hence atomics.
+std::atomic<int> g_max_blocks{0};     // tuning / test hook: 0 = one block per SM
+std::atomic<int> g_tail_reserve{-1};  // tuning / test hook: -1 = automatic, 0 = no reserve, n = at most n tiles per block
+std::atomic<long long> g_wait_limit_ns{0};  // test hook: 0 = the default limit of every bounded wait
+std::atomic<long long> g_skip_tile{-1};     // test hook: flat tile whose copies are never issued (-1 = none)
+constexpr int kAutoReserve = 8;     // tiles a block holds back at most (automatic mode)
+constexpr int kEpochShift = 24;     // a reserve counter is (epoch << 24) | tiles taken
 
 struct TmaParams {
   const __nv_bfloat16* q;
@@ -53,6 +69,12 @@ struct TmaParams {
   float* o_partial;    // [slots][U][d_v] normalised partial outputs
   float* lse_partial;  // [slots][U] base-2 log-sum-exp of the scaled scores
   int* meta;           // [batch + 1] exclusive prefix of tiles per sequence
+  unsigned long long* steal;  // [grid] reserve counters, (epoch << 24) | tiles taken
+  unsigned long long epoch;   // of this call, below 2^40
+  int reserve;                // most tiles a block holds back for the tail (0 = none)
+  int reserve_auto;           // 1: and never more than a sixth of a block's share
+  unsigned long long wait_ns; // limit of every bounded wait
+  long long skip_tile;        // test hook: flat tile whose copies the producer does not issue (-1 = none)
   void* out;
   float* lse;
   int out_is_f32;
@@ -114,6 +136,7 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   volatile int* abort_flag = reinterpret_cast<int*>(bars + 2 * p.stages);         // set when a wait ran out
   int* prefix = const_cast<int*>(abort_flag) + 2;                                 // [batch + 1]
   int* lens_s = prefix + p.batch + 1;                                             // [batch] lengths, clamped
+  volatile int* ctrl = lens_s + p.batch;  // [stages] tail phase: valid tokens of the tile in the stage, 0 = no more tiles
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t full0 = ptx::smem_u32(bars), empty0 = ptx::smem_u32(bars + p.stages);
@@ -131,6 +154,9 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   // Everything above touches only this block's shared memory and the kernel parameters; from here on the
   // kernel reads what earlier work in the stream may still be producing (lengths, q, the cache).
   ptx::grid_dependency_wait();
+  // This block's reserve counter starts at zero tiles taken, under this call's epoch (ordered before every draw of
+  // this block by the barriers below; a draw of another block that comes earlier finds a stale epoch and moves on).
+  if (p.reserve > 0 && tid == 0) atomicExch(p.steal + blockIdx.x, p.epoch << kEpochShift);
   // One round of global loads for the lengths (a dependent round trip costs most of a microsecond here); the
   // prefix below comes out of shared memory.  The per-sequence reads further down go to global memory again
   // (by then first-level cache hits): measured, that streams config 5 about 4 % faster than reading lens_s.
@@ -167,6 +193,14 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   const long long g_begin = (total * blockIdx.x) / nblk;
   const long long g_end = (total * (blockIdx.x + 1)) / nblk;
 
+  // ---- the tail reserve: the last R tiles of this block's last segment (never all of the segment)
+  const int reserve = p.reserve_auto ? (int)min((long long)p.reserve, (total / nblk) / 6) : p.reserve;
+  Walker wl;  // the row (sequence, unit) of the last segment
+  wl.seek(g_end - 1, prefix, p.batch, p.n_units);
+  const long long row_lo = (long long)p.n_units * prefix[wl.b] + (long long)wl.u * wl.nt, row_hi = row_lo + wl.nt;
+  const int R = reserve > 0 ? min(reserve, (int)(g_end - max(g_begin, row_lo)) - 1) : 0;
+  const long long g_stat = g_end - R;  // tiles [g_begin, g_stat) are this block's own
+
   Walker w;
   w.seek(g_begin, prefix, p.batch, p.n_units);
 
@@ -192,20 +226,8 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
       if (lane >= boxes || tok >= len) return 0;
       return p.page_table[(long long)w.b * p.max_pages_per_seq + tok / p.page_size];
     };
-    int blk = fetch_blk();
-    for (; w.g < g_end; ++w.g) {
-      if (issued >= p.stages) {
-        if (!ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) {
-          report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
-          ok = false;
-          break;
-        }
-      }
-      const int tok0 = w.t * kTT;
-      const int parts_valid = min(parts, (len - tok0 + p.box_tok - 1) / p.box_tok);
-      const uint32_t bar = full0 + 8 * stage;
-      if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)parts_valid * tile_part_bytes);
-      __syncwarp();
+    // This lane's box of tile (unit u, tokens from tok0) of a sequence of `len` tokens into `stage`.
+    auto issue_box = [&](int u, int tok0, int parts_valid, int blk, uint32_t bar) {
       if (lane < boxes && my_part < parts_valid) {
         const int tok = tok0 + my_part * p.box_tok;
         const int slot = p.page_table ? tok % p.page_size : tok;
@@ -215,12 +237,30 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         }
         const uint32_t dst = ptx::smem_u32(stage_base + (size_t)stage * STAGE_BYTES) + my_off;
         if (SHARED) {
-          if (my_is_k) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, 0, ((w.u * KPU) >> p.k_shift) + my_tile, blk);
-          else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, 0, ((w.u * VPU) >> p.v_shift) + (my_tile - KPU), blk);
+          if (my_is_k) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, 0, ((u * KPU) >> p.k_shift) + my_tile, blk);
+          else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, 0, ((u * VPU) >> p.v_shift) + (my_tile - KPU), blk);
         } else {
-          if (my_is_k) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, 0, w.u * KPU + my_tile, blk);
-          else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, 0, w.u * VPU + (my_tile - KPU), blk);
+          if (my_is_k) ptx::tma_load_5d(dst, &tmap_k, bar, 0, slot, 0, u * KPU + my_tile, blk);
+          else ptx::tma_load_5d(dst, &tmap_v, bar, 0, slot, 0, u * VPU + (my_tile - KPU), blk);
         }
+      }
+    };
+    int blk = fetch_blk();
+    for (; w.g < g_stat; ++w.g) {
+      if (issued >= p.stages) {
+        if (!ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.wait_ns)) {
+          report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+          ok = false;
+          break;
+        }
+      }
+      const int tok0 = w.t * kTT;
+      const int parts_valid = min(parts, (len - tok0 + p.box_tok - 1) / p.box_tok);
+      const uint32_t bar = full0 + 8 * stage;
+      if (w.g != p.skip_tile) {  // (test hook: a tile that is never requested; its stage's barrier stays incomplete)
+        if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)parts_valid * tile_part_bytes);
+        __syncwarp();
+        issue_box(w.u, tok0, parts_valid, blk, bar);
       }
       ++issued;
       if (++stage == p.stages) { stage = 0; phase ^= 1; }
@@ -232,7 +272,86 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
           if (w.b < p.batch) len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
         }
       }
-      if (w.g + 1 < g_end) blk = fetch_blk();
+      if (w.g + 1 < g_stat) blk = fetch_blk();
+    }
+    if (reserve > 0 && ok) {
+      // ---- tail: the reserves of the blocks whose last segment lies in this block's last row form a pool that all
+      // of them draw from until it is empty, so that they finish within about a tile of each other whatever their
+      // speeds were.  Lane 0 draws, the warp follows.
+      const int len_l = min(max(p.seqlens[wl.b], 0), p.max_seqlen);
+      auto draw = [&](int k) -> unsigned long long {  // raw old value of block k's counter (lane 0 only)
+        return lane == 0 ? atomicAdd(p.steal + k, 1ull) : 0ull;
+      };
+      auto taken = [&](unsigned long long raw) -> uint32_t {  // tiles taken so far, huge when the counter is stale
+        return (raw >> kEpochShift) == p.epoch ? (uint32_t)(raw & ((1ull << kEpochShift) - 1)) : 0xffffffffu;
+      };
+      auto issue_reserve_tile = [&](long long g) -> bool {  // flat tile g of this row
+        if (issued >= p.stages && !ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.wait_ns)) {
+          report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+          return false;
+        }
+        const int tok0 = (int)(g - row_lo) * kTT;
+        const int parts_valid = min(parts, (len_l - tok0 + p.box_tok - 1) / p.box_tok);
+        const uint32_t bar = full0 + 8 * stage;
+        if (lane == 0) {
+          ctrl[stage] = min(kTT, len_l - tok0);
+          ptx::mbar_arrive_expect_tx(bar, (uint32_t)parts_valid * tile_part_bytes);
+        }
+        __syncwarp();
+        int blk_t = wl.b;
+        if (p.page_table && lane < boxes && my_part < parts_valid)
+          blk_t = p.page_table[(long long)wl.b * p.max_pages_per_seq + (tok0 + my_part * p.box_tok) / p.page_size];
+        issue_box(wl.u, tok0, parts_valid, blk_t, bar);
+        ++issued;
+        if (++stage == p.stages) { stage = 0; phase ^= 1; }
+        return true;
+      };
+      // The pool: the reserves of up to 32 consecutive blocks whose last segment is in this row (lane i <-> block
+      // k_first + i), numbered block after block; its counter is the slot of the pool's first block.
+      const int k_lo = (int)(((row_lo + 1) * nblk - 1) / total), k_hi = (int)(((row_hi + 1) * nblk - 1) / total) - 1;
+      const int k_first = k_lo + (((int)blockIdx.x - k_lo) & ~31);
+      const int kc = k_first + lane;
+      int Rc = 0;       // this lane's block: size of its reserve, first tile of it
+      long long sc = 0;
+      if (kc <= k_hi) {
+        const long long kb = (total * kc) / nblk, ke = (total * (kc + 1)) / nblk;
+        Rc = min(reserve, (int)(ke - max(kb, row_lo)) - 1);
+        sc = ke - Rc;
+      }
+      int incl = Rc;  // tiles of the pool up to and including this lane's block
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+      }
+      const uint32_t pool = (uint32_t)__shfl_sync(0xffffffffu, incl, 31);
+      auto tile_of = [&](uint32_t idx) -> long long {  // flat tile of pool entry idx < pool
+        const int src = __popc(__ballot_sync(0xffffffffu, (uint32_t)incl <= idx));
+        const long long s0 = __shfl_sync(0xffffffffu, sc, src);
+        const int before = __shfl_sync(0xffffffffu, incl - Rc, src);
+        return s0 + ((int)idx - before);
+      };
+      // One tile per draw; the next draw is in flight while the current tile is issued.
+      uint32_t cur = pool > 0 ? taken(__shfl_sync(0xffffffffu, draw(k_first), 0)) : 0u;
+      while (cur < pool) {
+        const unsigned long long next_raw = draw(k_first);
+        if (!issue_reserve_tile(tile_of(cur))) { ok = false; break; }
+        cur = taken(__shfl_sync(0xffffffffu, next_raw, 0));
+      }
+      if (ok) {  // tell the consumers that the segment is complete: a stage without data
+        if (issued >= p.stages && !ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.wait_ns)) {
+          report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
+          ok = false;
+        } else {
+          if (lane == 0) {
+            ctrl[stage] = 0;
+            ptx::mbar_arrive(full0 + 8 * stage);
+          }
+          __syncwarp();
+          ++issued;
+          if (++stage == p.stages) { stage = 0; phase ^= 1; }
+        }
+      }
     }
     // All loads of this block are on their way: let the combine kernel (launched with programmatic stream
     // serialisation) become resident now rather than earlier -- blocks that wait for this grid take issue
@@ -242,7 +361,7 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
       // Give copies already in flight a bounded chance to land before the block's shared memory is released.
       for (int s = 0; s < min(issued, p.stages); ++s) {
         const int uses = (issued - s + p.stages - 1) / p.stages;
-        ptx::mbar_wait(full0 + 8 * s, (uint32_t)(uses - 1) & 1u, nullptr);
+        ptx::mbar_wait(full0 + 8 * s, (uint32_t)(uses - 1) & 1u, nullptr, p.wait_ns);
       }
     }
     return;
@@ -259,10 +378,12 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   uint32_t phase = 0;
   bool dead = false;
 
-  while (w.g < g_end) {
-    // ---- one segment: tiles [w.t, w.t + seg_tiles) of (sequence w.b, unit w.u)
-    const int seg_tiles = (int)min((long long)(w.nt - w.t), g_end - w.g);
-    const bool whole = (w.t == 0 && seg_tiles == w.nt);
+  while (w.g < g_stat) {
+    // ---- one segment: tiles [w.t, w.t + seg_tiles) of (sequence w.b, unit w.u); the block's last segment goes
+    // on with whatever the producer draws from the reserves of this row, until it posts a stage without data
+    const int seg_tiles = (int)min((long long)(w.nt - w.t), g_stat - w.g);
+    const bool tail = reserve > 0 && w.g + seg_tiles == g_stat;
+    const bool whole = (w.t == 0 && seg_tiles + (tail ? R : 0) == w.nt);
     const int len = min(max(p.seqlens[w.b], 0), p.max_seqlen);
     const long long wlin = (long long)w.b * p.n_units + w.u;
 
@@ -291,14 +412,25 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[j][mt][e] = 0.f;
 
-    for (int it = 0; it < seg_tiles; ++it) {
+    for (int it = 0; it < seg_tiles || tail; ++it) {
       // A wait that runs out marks the block dead: the warp stops waiting and computing but keeps
       // walking, so that it still meets the other warps at the named barriers below.
-      if (!dead && !ptx::mbar_wait(full0 + 8 * stage, phase, abort_flag)) {
+      if (dead && it >= seg_tiles) break;
+      if (!dead && !ptx::mbar_wait(full0 + 8 * stage, phase, abort_flag, p.wait_ns)) {
         report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
         dead = true;
+        if (it >= seg_tiles) break;
       }
-      const int n_valid = dead ? 0 : min(kTT, len - (w.t + it) * kTT);
+      int n_valid = dead ? 0 : min(kTT, len - (w.t + it) * kTT);
+      if (it >= seg_tiles) {  // a tile out of a reserve, or the end of the segment
+        n_valid = ctrl[stage];
+        if (n_valid == 0) {
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(empty0 + 8 * stage);
+          if (++stage == p.stages) { stage = 0; phase ^= 1; }
+          break;
+        }
+      }
       unsigned char* st = stage_base + (size_t)stage * STAGE_BYTES;
       const uint32_t st_u32 = ptx::smem_u32(st);
       if (row0 < n_valid) {
@@ -737,13 +869,14 @@ bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPla
   }
   const DeviceInfo di = device_info();
   if (di.sms <= 0) return false;
-  const int fixed = 1024 + kConsumerWarps * kHeadsPerMma * (s.d_v + 4 + 2) * 4 + 2 * 16 * 8 + (2 * s.batch + 1) * 4 + 64;
+  const int fixed = 1024 + kConsumerWarps * kHeadsPerMma * (s.d_v + 4 + 2) * 4 + 2 * 16 * 8 + (2 * s.batch + 1) * 4 + 64 + 8 * 4;
   int stages = (di.max_smem - fixed) / v.stage_bytes;
   if (stages > 8) stages = 8;
   if (stages < 2) return false;
   const long long tiles_max = (long long)s.batch * (s.n_q / U) * ((c.max_seqlen + kTT - 1) / kTT);
   long long grid = di.sms;
-  if (g_max_blocks > 0 && grid > g_max_blocks) grid = g_max_blocks;
+  const int max_blocks = g_max_blocks.load();
+  if (max_blocks > 0 && grid > max_blocks) grid = max_blocks;
   if (grid > tiles_max) grid = tiles_max;
   if (grid < 1) grid = 1;
   plan->U = U; plan->kpu = kpu; plan->vpu = vpu; plan->box_tok = box_tok; plan->stages = stages;
@@ -751,14 +884,33 @@ bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPla
   plan->grid = (int)grid;
   plan->smem = fixed + stages * v.stage_bytes;
   plan->slots = grid + (long long)s.batch * (s.n_q / U);
+  const int tail_reserve = g_tail_reserve.load();
+  plan->reserve = tail_reserve < 0 ? kAutoReserve : tail_reserve;
+  plan->reserve_auto = tail_reserve < 0;
   return true;
 }
 
 void set_tma_max_blocks(int n) { g_max_blocks = n > 0 ? n : 0; }
+void set_tma_tail_reserve(int n) { g_tail_reserve = n < 0 ? -1 : (n > 4096 ? 4096 : n); }
+void set_tma_debug_timeout(long long wait_limit_ns, long long skip_tile) {
+  g_wait_limit_ns = wait_limit_ns > 0 ? wait_limit_ns : 0;
+  g_skip_tile = skip_tile >= 0 ? skip_tile : -1;
+}
+
+// Every launch gets an epoch of its own (below 2^40), counted up from a random start, so that a reserve counter
+// left in a workspace by an earlier call, or whatever else the memory held, is not mistaken for this call's.
+static unsigned long long next_epoch() {
+  static std::atomic<unsigned long long> counter{[] {
+    std::random_device rd;
+    return ((unsigned long long)rd() << 20) ^ (unsigned long long)rd();
+  }()};
+  return counter.fetch_add(1, std::memory_order_relaxed) & ((1ull << 40) - 1);
+}
 
 size_t tma_decode_workspace_bytes(const diffqkv_shape& s, const TmaPlan& plan) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
-  return up((size_t)plan.slots * plan.U * s.d_v * 4) + up((size_t)plan.slots * plan.U * 4) + up((size_t)(s.batch + 1) * 4);
+  return up((size_t)plan.slots * plan.U * s.d_v * 4) + up((size_t)plan.slots * plan.U * 4) +
+         up((size_t)(s.batch + 1) * 4) + up((size_t)plan.grid * 8);
 }
 
 // Returns cudaErrorNotSupported when no tensor map can describe the cache (the caller then falls back to
@@ -792,6 +944,14 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
   p.lse_partial = reinterpret_cast<float*>(ws);
   ws += up((size_t)plan.slots * plan.U * 4);
   p.meta = reinterpret_cast<int*>(ws);
+  ws += up((size_t)(s.batch + 1) * 4);
+  p.steal = reinterpret_cast<unsigned long long*>(ws);
+  p.epoch = next_epoch();
+  p.reserve = plan.reserve;
+  p.reserve_auto = plan.reserve_auto;
+  const long long wait_ns = g_wait_limit_ns.load();
+  p.wait_ns = wait_ns > 0 ? (unsigned long long)wait_ns : ptx::kWaitLimitNs;
+  p.skip_tile = g_skip_tile.load();
   p.out = out; p.lse = lse; p.out_is_f32 = s.out_dtype == DIFFQKV_F32;
   p.dev_status = dev_status;
 

@@ -15,6 +15,8 @@
 // Both are launched with programmatic stream serialisation and wait on the device before touching their inputs.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tmap.cuh"
@@ -966,7 +968,7 @@ size_t topk_decode_workspace_bytes(const diffqkv_shape& s, int max_seqlen, int /
   return up256(rows * lpad * sizeof(float)) + up256(rows * (lpad / 16) * sizeof(float));
 }
 
-static int g_topk_general_only = 0;  // test hook
+static std::atomic<int> g_topk_general_only{0};  // test hook
 void set_topk_general_only(int on) { g_topk_general_only = on != 0; }
 
 cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, int topk, int box_tok,

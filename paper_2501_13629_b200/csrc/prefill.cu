@@ -73,18 +73,20 @@ __device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity, volatil
   return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity, abort_flag));
 }
 
-template <int kD>  // channels per head, 64 or 128
+template <int kDQK, int kD>  // channels per head of Q/K and of V: (128, 128), (64, 64) or (64, 128)
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, const PrefillParams p) {
-  constexpr int kHalves = kD / 64;          // 64-channel halves of a row
-  constexpr int kQBytes = kQT * kD * 2;     // a Q tile: [half][128 rows][128 B]
-  constexpr int kTBytes = kKT * kD * 2;     // a K tile or a V tile: [half][128 rows][128 B]
+  constexpr int kHalvesK = kDQK / 64, kHalves = kD / 64;  // 64-channel halves of a Q/K row and of a V row
+  constexpr int kHalvesMax = kHalvesK > kHalves ? kHalvesK : kHalves;
+  constexpr int kQBytes = kQT * kDQK * 2;   // a Q tile: [half][128 rows][128 B]
+  constexpr int kKBytes = kKT * kDQK * 2;   // a K tile: [half][128 rows][128 B]
+  constexpr int kTBytes = kKT * kD * 2;     // a V tile: [half][128 rows][128 B]
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* q_s = smem;                      // 2 M-tiles
   unsigned char* k_s = q_s + 2 * kQBytes;         // ring of K tiles
-  unsigned char* v_s = k_s + kKSlots * kTBytes;   // ring of V tiles
+  unsigned char* v_s = k_s + kKSlots * kKBytes;   // ring of V tiles
   uint64_t* bars = reinterpret_cast<uint64_t*>(v_s + kVSlots * kTBytes);
   // q_full, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2], drain, p_half[2]
   const uint32_t q_full = ptx::smem_u32(bars);
@@ -158,8 +160,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     }
     // One box per (token part, channel half) of a tile: lane x owns box x of every K tile and of every V tile.
     const int parts = kKT / p.box_tok;
-    const int boxes = kHalves * parts;
-    const int my_part = lane / kHalves, my_half = lane % kHalves;
+    const int boxes = kHalvesMax * parts;
+    const int my_part = lane / kHalvesMax, my_half = lane % kHalvesMax;
     const uint32_t my_off = my_half * (kKT * 128) + my_part * (p.box_tok * 128);
     int ks = 0, vs = 0, issued_k = 0, issued_v = 0;
     uint32_t kph = 0, vph = 0;
@@ -179,16 +181,19 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         }
       }
       const uint32_t tx = (uint32_t)parts_valid * p.box_tok * 128u * kHalves;
+      const uint32_t tx_k = (uint32_t)parts_valid * p.box_tok * 128u * kHalvesK;
       if (!wait_warp(k_empty0 + 8 * ks, kph ^ 1, abort_flag)) { ok = false; break; }
-      if (lane == 0) ptx::mbar_arrive_expect_tx(k_full0 + 8 * ks, tx);
+      if (lane == 0) ptx::mbar_arrive_expect_tx(k_full0 + 8 * ks, tx_k);
       __syncwarp();
-      if (mine) ptx::tma_load_5d(k_u32 + ks * kTBytes + my_off, &tmap_k, k_full0 + 8 * ks, 0, slot, my_half, hk, blk);
+      if (mine && my_half < kHalvesK)
+        ptx::tma_load_5d(k_u32 + ks * kKBytes + my_off, &tmap_k, k_full0 + 8 * ks, 0, slot, my_half, hk, blk);
       ++issued_k;
       if (++ks == kKSlots) { ks = 0; kph ^= 1; }
       if (!wait_warp(v_empty0 + 8 * vs, vph ^ 1, abort_flag)) { ok = false; break; }
       if (lane == 0) ptx::mbar_arrive_expect_tx(v_full0 + 8 * vs, tx);
       __syncwarp();
-      if (mine) ptx::tma_load_5d(v_u32 + vs * kTBytes + my_off, &tmap_v, v_full0 + 8 * vs, 0, slot, my_half, hv, blk);
+      if (mine && my_half < kHalves)
+        ptx::tma_load_5d(v_u32 + vs * kTBytes + my_off, &tmap_v, v_full0 + 8 * vs, 0, slot, my_half, hv, blk);
       ++issued_v;
       if (++vs == kVSlots) { vs = 0; vph ^= 1; }
     }
@@ -211,11 +216,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       const uint32_t q_lo = tc::smem_desc_lo(q_u32, 16), k_lo = tc::smem_desc_lo(k_u32, 16);
       const uint32_t v_lo = tc::smem_desc_lo(v_u32, kKT * 128);  // 64-channel chunks of V are one half tile apart
       auto issue_s = [&](int t, int slot) {  // S_t = Q_t . K^T
-        const uint32_t qa = q_lo + t * (kQBytes >> 4), ka = k_lo + slot * (kTBytes >> 4);
+        const uint32_t qa = q_lo + t * (kQBytes >> 4), ka = k_lo + slot * (kKBytes >> 4);
         const uint32_t d = tmem_base + t * 128;
         tc::mma_ss_halves<false>(d, qa, hi, ka, hi, idesc);
 #pragma unroll
-        for (int ks = 1; ks < kD / 16; ++ks) {
+        for (int ks = 1; ks < kDQK / 16; ++ks) {
           const uint32_t step = ((ks / 4) * (128 * 128) + (ks % 4) * 32) >> 4;
           tc::mma_ss_halves<true>(d, qa + step, hi, ka + step, hi, idesc);
         }
@@ -492,7 +497,12 @@ bool make_cache_map(CUtensorMap* map, const void* base, int d, long long tok_ext
 }  // namespace
 
 bool prefill_supported(const diffqkv_shape& s, const diffqkv_cache& c, int* box_tok) {
-  if (s.dtype != DIFFQKV_BF16 || s.d_qk != s.d_v || (s.d_qk != 64 && s.d_qk != 128)) return false;
+  if (s.dtype != DIFFQKV_BF16) return false;
+  const bool dims_ok = (s.d_qk == 128 && s.d_v == 128) || (s.d_qk == 64 && s.d_v == 64) || (s.d_qk == 64 && s.d_v == 128);
+  if (!dims_ok) return false;
+  // The kernel takes the row maximum of the raw scores and scales it afterwards, which keeps the order only for a
+  // positive scale; zero and negative scales go to the generic kernel.
+  if (!(s.scale > 0.f)) return false;
   int bt = kKT;
   if (c.page_table) {
     if (c.page_size >= kKT) { if (c.page_size % kKT != 0) return false; }
@@ -531,12 +541,9 @@ cudaError_t launch_cache_append(const void* k_new, const void* v_new, int q_len,
 cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, int q_len, const diffqkv_cache& c,
                            const diffqkv_shape& s, int box_tok, void* out, float* lse, int* dev_status,
                            cudaStream_t stream) {
-  // ---- step 1: cache update
-  cudaError_t err = launch_cache_append(k_new, v_new, q_len, c, s, dev_status, stream);
-  if (err != cudaSuccess) return err;
-
-  // ---- step 2: attention over the cache
-  const int d = s.d_qk;  // == d_v, 64 or 128
+  // Tensor maps first: when one cannot be built the caller runs both steps on the generic kernels, and nothing
+  // has been launched yet.
+  const int d = s.d_qk;
   CUtensorMap mq, mk, mv;
   {
     const cuuint64_t dims[5] = {64, (cuuint64_t)q_len, (cuuint64_t)(d / 64), (cuuint64_t)s.n_q, (cuuint64_t)s.batch};
@@ -548,9 +555,13 @@ cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, 
   const long long tok_extent = c.page_table ? c.page_size : c.max_seqlen;
   if (!make_cache_map(&mk, c.k_cache, d, tok_extent, s.n_k, c.num_blocks, c.k_stride_tok, c.k_stride_head,
                       c.k_stride_blk, box_tok) ||
-      !make_cache_map(&mv, c.v_cache, d, tok_extent, s.n_v, c.num_blocks, c.v_stride_tok, c.v_stride_head,
+      !make_cache_map(&mv, c.v_cache, s.d_v, tok_extent, s.n_v, c.num_blocks, c.v_stride_tok, c.v_stride_head,
                       c.v_stride_blk, box_tok))
     return cudaErrorNotSupported;
+  // ---- step 1: cache update
+  cudaError_t err = launch_cache_append(k_new, v_new, q_len, c, s, dev_status, stream);
+  if (err != cudaSuccess) return err;
+  // ---- step 2: attention over the cache
   PrefillParams p;
   p.seqlens = c.seqlens; p.page_table = c.page_table;
   p.page_size = c.page_size; p.max_pages_per_seq = c.max_pages_per_seq;
@@ -562,15 +573,12 @@ cudaError_t launch_prefill(const void* q, const void* k_new, const void* v_new, 
   p.out = out; p.out_is_f32 = s.out_dtype == DIFFQKV_F32; p.lse = lse; p.dev_status = dev_status;
   const long long grid = (long long)p.n_qpairs * s.batch * s.n_q;
   if (grid > 0x7fffffffLL) return cudaErrorNotSupported;
-  if (d == 128) {
-    err = cudaFuncSetAttribute(prefill_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrefillSmem);
-    if (err != cudaSuccess) return err;
-    prefill_attn_kernel<128><<<(unsigned)grid, kPrefillThreads, kPrefillSmem, stream>>>(mq, mk, mv, p);
-  } else {
-    err = cudaFuncSetAttribute(prefill_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrefillSmem);
-    if (err != cudaSuccess) return err;
-    prefill_attn_kernel<64><<<(unsigned)grid, kPrefillThreads, kPrefillSmem, stream>>>(mq, mk, mv, p);
-  }
+  using PrefillFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const PrefillParams);
+  const PrefillFn fn = s.d_v == 64 ? prefill_attn_kernel<64, 64>
+                                   : (d == 128 ? prefill_attn_kernel<128, 128> : prefill_attn_kernel<64, 128>);
+  err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrefillSmem);
+  if (err != cudaSuccess) return err;
+  fn<<<(unsigned)grid, kPrefillThreads, kPrefillSmem, stream>>>(mq, mk, mv, p);
   count_launch();
   return cudaGetLastError();
 }

@@ -71,3 +71,29 @@ def check_lse(lse, ref, tol, what=""):
     with np.errstate(invalid="ignore"):
         d = np.where(both_inf, 0.0, np.abs(lse - ref))
     assert np.all(np.isfinite(d)) and d.max() <= tol, f"{what}: lse err {d.max()}"
+
+
+def check_proj(out, ref, what="", c_abs=2e-2):
+    """Projection chains (bf16 operands and result, fp32 accumulation; the oracle rounds nothing).
+
+    Three checks: max |err| <= 1e-2 max |ref|; rms(err) <= 4e-3 rms(ref); and element-wise
+    |err| <= 2^-8 |ref| + c_abs * rms(ref row).  The last one follows from the arithmetic: an output element is a sum
+    of products whose operands were rounded to bf16 (relative error at most 2^-9 each, independent), so its error
+    scales with the typical magnitude of its row (about 2e-3 of the row's rms over the three rounded stages of the
+    aug-Q chain), not with the element itself, plus 2^-9 |ref| from rounding the result; c_abs = 2e-2 leaves ten
+    standard deviations, and an element of small magnitude that is simply wrong (by its row's rms) fails it.
+    `out` and `ref` are [rows, columns] (or reshaped to that)."""
+    out = np.asarray(out, dtype=np.float64).reshape(-1, out.shape[-1])
+    ref = np.asarray(ref, dtype=np.float64).reshape(out.shape)
+    err = np.abs(out - ref)
+    assert np.isfinite(out).all(), what
+    big = np.abs(ref).max()
+    assert err.max() <= 1e-2 * big, f"{what}: max err {err.max():.3e} vs max|ref| {big:.3e}"
+    rms_all = np.sqrt(np.mean(ref ** 2))
+    rms = np.sqrt(np.mean(err ** 2)) / max(rms_all, 1e-300)
+    assert rms <= 4e-3, f"{what}: rms err / rms ref = {rms:.3e}"
+    row_rms = np.sqrt(np.mean(ref ** 2, axis=1, keepdims=True))
+    bound = 2.0 ** -8 * np.abs(ref) + c_abs * row_rms
+    worst = (err / np.maximum(bound, 1e-300)).max()
+    assert worst <= 1.0, f"{what}: element-wise bound exceeded by {worst:.2f}x"
+    return float(worst)

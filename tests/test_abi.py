@@ -9,6 +9,7 @@ import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 HEADER = os.path.join(ROOT, "include", "diffqkv.h")
+HEADERS = [HEADER, os.path.join(ROOT, "include", "diffqkv_debug.h")]
 
 
 @pytest.fixture(scope="module")
@@ -20,14 +21,15 @@ def api():
 
 
 def _declared_functions():
-    text = open(HEADER).read()
+    text = "".join(open(h).read() for h in HEADERS)
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b((?:diffqkv|gqa)_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_header_compiles_as_plain_c(tmp_path):
     src = tmp_path / "t.c"
-    src.write_text('#include "diffqkv.h"\nint main(void){diffqkv_shape s; (void)s; return DIFFQKV_OK;}\n')
+    src.write_text('#include "diffqkv.h"\n#include "diffqkv_debug.h"\n'
+                   'int main(void){diffqkv_shape s; (void)s; return DIFFQKV_OK;}\n')
     subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.dirname(HEADER), "-c", str(src),
                            "-o", str(tmp_path / "t.o")])
 
@@ -35,7 +37,7 @@ def test_header_compiles_as_plain_c(tmp_path):
 def test_every_declared_symbol_is_exported(api):
     names = _declared_functions()
     assert "diffqkv_decode" in names and "gqa_decode" in names and "diffqkv_combine" in names
-    assert "diffqkv_prefill" in names
+    assert "diffqkv_prefill" in names and "diffqkv_debug_decode_timeout" in names and "diffqkv_fold_k_up" in names
     lib = C.CDLL(api.LIB_PATH)
     for n in names:
         assert hasattr(lib, n), n

@@ -73,7 +73,7 @@ def test_mixed_head_dims(api, oracle):
 
 @pytest.mark.parametrize("heads", [(32, 1, 2), (32, 2, 4), (32, 2, 2), (16, 1, 1), (64, 4, 8), (64, 2, 16)])
 @pytest.mark.parametrize("d", [64, 128])
-def test_more_than_eight_query_heads_per_kv_head(api, oracle, heads, d):
+def test_more_than_eight_query_heads_per_kv_head(api, oracle, fixed_owners, heads, d):
     """Multi-query-like shapes: the TMA kernel cuts a unit of 16 to 32 query heads into sub-units of 8 that share
     their K (and V) head; parity with the oracle, contiguous and paged."""
     n_q, n_k, n_v = heads
@@ -89,7 +89,7 @@ def test_more_than_eight_query_heads_per_kv_head(api, oracle, heads, d):
 
 
 @pytest.mark.parametrize("heads", [(32, 4, 16), (16, 2, 4), (8, 4, 4)])
-def test_half_width_keys_take_the_tma_kernel(api, oracle, heads):
+def test_half_width_keys_take_the_tma_kernel(api, oracle, fixed_owners, heads):
     """d_k = d_v / 2 (the paper's other axis of K compression) with SIGMA-1.5B's 4 K / 16 V heads and two smaller
     shapes: the persistent TMA kernel, not the generic fallback."""
     n_q, n_k, n_v = heads
@@ -190,6 +190,22 @@ def test_paged_varlen_config5_shape_reduced(api, oracle):
 
 
 @pytest.fixture
+def fixed_owners(api):
+    """No tail reserve: every tile has a fixed owner, so results are bitwise reproducible (what the tests that
+    compare two runs bit for bit need); the default is restored afterwards."""
+    api.set_tail_reserve(0)
+    yield
+    api.set_tail_reserve(-1)
+
+
+@pytest.fixture
+def tail_reserve(api):
+    """Sets the tail reserve of the TMA kernel and always restores the automatic choice."""
+    yield api.set_tail_reserve
+    api.set_tail_reserve(-1)
+
+
+@pytest.fixture
 def blocks(api):
     """Sets the persistent-block cap of the TMA kernel and always restores the default."""
     yield api.set_max_blocks
@@ -229,7 +245,7 @@ def test_tma_block_partition_invariance(api, oracle, blocks, heads, d):
 
 
 @pytest.mark.parametrize("page_size", [16, 32, 64, 128])
-def test_tma_paged_equals_contiguous_bitwise(api, oracle, blocks, page_size):
+def test_tma_paged_equals_contiguous_bitwise(api, oracle, blocks, fixed_owners, page_size):
     inp = W.make_decode_inputs(dataclasses.replace(SMALL, kv_len=1024), seqlens=np.array([1024, 500, 17], np.int32))
     ref, _ = run_oracle(oracle, inp)
     for nb in (0, 5):
@@ -242,6 +258,74 @@ def test_tma_paged_equals_contiguous_bitwise(api, oracle, blocks, page_size):
             out, lse, st = run_decode(api, pg)
             assert st == 0 and api.last_decode_kernel() == api.KERNEL_TMA
             assert np.array_equal(out, base) and np.array_equal(lse, lse0)
+
+
+@pytest.mark.parametrize("heads,d_qk,d_v", [((16, 2, 4), 128, 128), ((32, 4, 16), 64, 64), ((8, 4, 1), 128, 128),
+                                            ((32, 1, 2), 128, 128), ((16, 2, 4), 64, 128)])
+def test_tail_reserve_invariance(api, oracle, blocks, tail_reserve, heads, d_qk, d_v):
+    """Tiles drawn from the reserves (the block's own and those of the other blocks of the row) give the same
+    attention as fixed owners: against the oracle and against each other up to fp32 reassociation, for several block
+    counts (which move the cuts), reserves from one tile to the whole segment, ragged and empty sequences, NaN bit
+    patterns behind every sequence end, contiguous and paged."""
+    n_q, n_k, n_v = heads
+    cfg = dataclasses.replace(SMALL, batch=5, n_q=n_q, n_k=n_k, n_v=n_v, d_qk=d_qk, d_v=d_v, kv_len=3000, seed=91)
+    lens = np.array([3000, 64, 0, 1777, 1], dtype=np.int32)
+    inp = W.make_decode_inputs(cfg, seqlens=lens)
+    for b, n in enumerate(lens):
+        inp.k[b, :, n:] = 0x7FC0  # bf16 NaN
+        inp.v[b, :, n:] = 0x7FC0
+    ref, lse_ref = run_oracle(oracle, inp)
+    outs = []
+    for paged in (0, 16):
+        case = W.paginate(inp, paged, seed=7) if paged else inp
+        for nb in (0, 7, 40):
+            blocks(nb)
+            for reserve in (0, 1, 3, 4096, -1):
+                tail_reserve(reserve)
+                out, lse, st = run_decode(api, case)
+                what = f"{heads} d={d_qk}/{d_v} paged={paged} blocks={nb} reserve={reserve}"
+                assert st == 0 and api.last_decode_kernel() == api.KERNEL_TMA, what
+                check_bf16(out, ref, what)
+                check_lse(lse, lse_ref, 2e-2, what)
+                assert np.all(out[2] == 0) and np.all(np.isneginf(lse[2])), what
+                outs.append(out)
+    for o in outs[1:]:
+        assert np.abs(o - outs[0]).max() <= 5e-3
+
+
+def test_tail_reserve_full_size_every_tile_drawn(api, oracle, tail_reserve):
+    """The headline shape with every tile but one per segment handed out through the counters: a stress of the
+    draw protocol at 148 blocks (the automatic reserve runs in test_full_size_bf16_and_gqa_twin)."""
+    inp = W.make_decode_inputs(W.CFG3)
+    ref, lse_ref = run_oracle(oracle, inp)
+    for reserve in (4096, 20):
+        tail_reserve(reserve)
+        for _ in range(3):
+            out, lse, st = run_decode(api, inp)
+            assert st == 0
+            check_bf16(out, ref, f"cfg3 reserve={reserve}")
+            check_lse(lse, lse_ref, 2e-2)
+
+
+def test_a_device_wait_that_runs_out_is_reported_and_leaves_the_context_usable(api, oracle, fixed_owners):
+    """The failure path of the bounded waits, reached without breaking anything: with the wait limit at 2 ms the
+    producer of block 0 never requests its first tile (no copy in flight, no completion count), the consumers' wait
+    for it runs out, the block reports DIFFQKV_ERR_TIMEOUT, drains and returns.  The same stream then runs an
+    ordinary call whose result equals, bit for bit, that of a call made before the failure."""
+    inp = W.make_decode_inputs(dataclasses.replace(SMALL, batch=4, kv_len=2000, seed=97))
+    ref, _ = run_oracle(oracle, inp)
+    clean, lse_clean, st = run_decode(api, inp)
+    assert st == 0 and api.last_decode_kernel() == api.KERNEL_TMA
+    check_bf16(clean, ref)
+    try:
+        api.debug_decode_timeout(2_000_000, 0)
+        _, _, st = run_decode(api, inp)
+    finally:
+        api.debug_decode_timeout(0, -1)
+    assert st == 1 << api.ERR_TIMEOUT
+    again, lse_again, st = run_decode(api, inp)
+    assert st == 0
+    assert np.array_equal(again, clean) and np.array_equal(lse_again, lse_clean)
 
 
 def test_tma_tail_rows_with_nan_garbage(api, oracle):
@@ -325,7 +409,7 @@ def test_config5_full_size_sampled_rows(api, oracle):
     check_lse(lse.cpu().numpy().astype(np.float64)[sel], lse_ref[sel], 2e-2, "cfg5 full size")
 
 
-def test_decode_from_and_to_host_memory(api, oracle):
+def test_decode_from_and_to_host_memory(api, oracle, fixed_owners):
     """diffqkv_decode_host: q in pinned host memory, the result back in pinned host memory, same numbers as
     diffqkv_decode on device buffers (bitwise) and within tolerance of the oracle."""
     inp = W.make_decode_inputs(SMALL)
@@ -349,3 +433,15 @@ def test_decode_from_and_to_host_memory(api, oracle):
         assert torch.equal(out_host, ref_out.cpu())
     ref, _ = run_oracle(oracle, inp)
     check_bf16(out_host.numpy().astype(np.float64), ref, "decode from host memory")
+
+
+def test_split_counts_beyond_the_combine_limit_are_refused_before_any_launch(api):
+    cfg = dataclasses.replace(W.CFG2, batch=1, kv_len=256)
+    inp = W.make_decode_inputs(cfg)
+    q, cache = W.to_torch(inp.q, "cuda"), device_cache(api, inp)
+    launches = api.launch_count()
+    with pytest.raises(api.DiffQKVError) as e:
+        api.diffqkv_decode(q, cache, cfg.n_k, cfg.n_v, cfg.scale, num_splits=8193,
+                           workspace=torch.zeros(1 << 20, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == api.ERR_UNSUPPORTED
+    assert api.launch_count() == launches

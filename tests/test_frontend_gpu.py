@@ -10,7 +10,7 @@ import pytest
 import torch
 
 from paper_2501_13629_b200 import workloads as W
-from helpers import check_bf16, device_cache, run_oracle
+from helpers import check_bf16, check_proj, device_cache, run_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -23,10 +23,7 @@ def api():
 
 
 def _check(out, ref, what):
-    err = np.abs(out - ref)
-    assert err.max() <= 1e-2 * np.abs(ref).max(), f"{what}: max err {err.max():.3e} vs max|ref| {np.abs(ref).max():.3e}"
-    rms = np.sqrt(np.mean(err ** 2)) / np.sqrt(np.mean(ref ** 2))
-    assert rms <= 4e-3, f"{what}: rms err / rms ref = {rms:.3e}"
+    check_proj(out, ref, what)
 
 
 def _tables(oracle, pos, d, theta):

@@ -1,5 +1,5 @@
 """GPU parity of diffqkv_prefill on the shapes its tensor-core kernel does not take (fp32 storage, head dimensions
-other than 64 and 128, d_qk != d_v): cache update + causal attention on the generic fp32-FMA kernel, against the float64
+other than (128, 128), (64, 64) and (64, 128)): cache update + causal attention on the generic fp32-FMA kernel, against the float64
 oracle through the C ABI.  bf16 storage: the bf16 tolerances of helpers.check_bf16; fp32 storage:
 max |err| / max |ref| <= 1e-5.  The cache contents after the call must equal the oracle's cache update bit for bit."""
 import numpy as np
@@ -54,7 +54,7 @@ def run_both(api, oracle, seed, batch, q_len, heads, d_qk, d_v, past, dtype):
     return out.cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64), ref, lse_ref
 
 
-@pytest.mark.parametrize("d_qk,d_v", [(192, 192), (64, 128), (128, 64), (32, 256)])
+@pytest.mark.parametrize("d_qk,d_v", [(192, 192), (128, 64), (32, 256)])
 @pytest.mark.parametrize("heads", [(8, 2, 4), (4, 4, 1)])
 def test_bf16_other_head_dimensions(api, oracle, d_qk, d_v, heads):
     out, lse, ref, lse_ref = run_both(api, oracle, 300 + d_qk + d_v, 2, 150, heads, d_qk, d_v, [0, 37], "bf16")

@@ -23,25 +23,27 @@ def api():
 class Case:
     """Seeded prefill problem with a contiguous [batch, head, S, d] cache holding `past` earlier tokens."""
 
-    def __init__(self, seed, batch, q_len, heads, past, S=None, q_std=1.0, garbage=None, d=D):
+    def __init__(self, seed, batch, q_len, heads, past, S=None, q_std=1.0, garbage=None, d=D, d_v=None):
         n_q, n_k, n_v = heads
         self.d = D = d
+        self.d_v = d_v or d
         self.batch, self.q_len, self.heads = batch, q_len, heads
         self.past = np.asarray(past, dtype=np.int32)
         self.S = S or int(self.past.max() + q_len)
         self.q = W.normal(seed, (batch, q_len, n_q, D), std=q_std)
         self.k_new = W.normal(seed + 1, (batch, q_len, n_k, D))
-        self.v_new = W.normal(seed + 2, (batch, q_len, n_v, D))
+        self.v_new = W.normal(seed + 2, (batch, q_len, n_v, self.d_v))
         self.k = W.normal(seed + 3, (batch, n_k, self.S, D))
-        self.v = W.normal(seed + 4, (batch, n_v, self.S, D))
+        self.v = W.normal(seed + 4, (batch, n_v, self.S, self.d_v))
         if garbage is not None:  # poison everything at and after the first new row
             for b in range(batch):
                 self.k[b, :, self.past[b]:] = garbage
                 self.v[b, :, self.past[b]:] = garbage
         self.scale = D ** -0.5
 
-    def strides(self, n):
-        return (n * self.S * self.d, self.S * self.d, self.d)
+    def strides(self, n, d=None):
+        d = d or self.d
+        return (n * self.S * d, self.S * d, d)
 
 
 def run_gpu(api, case, paged=None, out_dtype=torch.float32):
@@ -51,11 +53,11 @@ def run_gpu(api, case, paged=None, out_dtype=torch.float32):
     seqlens = torch.from_numpy(case.past).to(dev)
     if paged is None:
         k, v = W.to_torch(case.k.copy(), dev), W.to_torch(case.v.copy(), dev)
-        cache = api.KVCache(k, v, seqlens, case.S, k_strides=case.strides(n_k), v_strides=case.strides(n_v),
+        cache = api.KVCache(k, v, seqlens, case.S, k_strides=case.strides(n_k), v_strides=case.strides(n_v, case.d_v),
                             num_blocks=case.batch)
     else:
-        inp = W.DecodeInputs(W.DecodeConfig("t", case.batch, n_q, n_k, n_v, case.d, case.d, case.S), None, case.k, case.v,
-                             case.past, case.strides(n_k), case.strides(n_v), max_seqlen=case.S)
+        inp = W.DecodeInputs(W.DecodeConfig("t", case.batch, n_q, n_k, n_v, case.d, case.d_v, case.S), None, case.k, case.v,
+                             case.past, case.strides(n_k), case.strides(n_v, case.d_v), max_seqlen=case.S)
         pg = W.paginate(inp, paged, seed=99)
         k, v = W.to_torch(pg.k, dev), W.to_torch(pg.v, dev)
         cache = api.KVCache(k, v, seqlens, pg.max_seqlen, page_table=torch.from_numpy(pg.page_table).to(dev),
@@ -84,9 +86,9 @@ def run_gpu(api, case, paged=None, out_dtype=torch.float32):
 def run_oracle(oracle, case, rows=None):
     n_q, n_k, n_v = case.heads
     k, v = case.k.copy(), case.v.copy()
-    cache = oracle.Cache(k, v, case.strides(n_k), case.strides(n_v), case.past)
+    cache = oracle.Cache(k, v, case.strides(n_k), case.strides(n_v, case.d_v), case.past)
     oracle.cache_append(case.k_new, case.v_new, cache)
-    out, lse = oracle.prefill(case.q, case.past, cache, n_k, n_v, case.d, case.scale, rows=rows)
+    out, lse = oracle.prefill(case.q, case.past, cache, n_k, n_v, case.d_v, case.scale, rows=rows)
     return out, lse, k, v
 
 
@@ -159,6 +161,16 @@ def test_paged_cache_equals_contiguous_bitwise(api, oracle, page_size):
     check_bf16(out_p, ref, f"paged {page_size}")
 
 
+@pytest.mark.parametrize("scale", [-0.0884, 0.0])
+def test_non_positive_scale_matches_the_oracle(api, oracle, scale):
+    """A negative scale turns the softmax towards the smallest inner products; zero makes it uniform.  Either must give
+    what the definition gives (the tensor-core kernel orders raw scores, so these run on the generic kernel)."""
+    case = Case(950, 1, 200, (8, 2, 4), [30])
+    case.scale = scale
+    check_case(api, oracle, case, f"scale={scale}")
+    assert api.last_prefill_kernel() == 1
+
+
 def test_bf16_output(api, oracle):
     case = Case(900, 1, 200, (8, 2, 4), [0])
     ref, _, _, _ = run_oracle(oracle, case)
@@ -206,6 +218,21 @@ def test_config4_full_size_sampled_rows(api, oracle):
 def test_head_dimension_64_on_the_tensor_cores(api, oracle, q_len, past):
     """SIGMA-1.5B's head size: the same kernel with half-width tiles."""
     check_case(api, oracle, Case(800 + q_len, 2, q_len, (8, 2, 4), past, d=64), f"d=64 q_len={q_len} past={past}")
+    assert api.last_prefill_kernel() == 2
+
+
+@pytest.mark.parametrize("q_len,past", [(1, [0, 0]), (129, [0, 70]), (300, [257, 5]), (700, [0, 0])])
+def test_half_width_keys_on_the_tensor_cores(api, oracle, q_len, past):
+    """d_qk = 64 with d_v = 128 (keys cached at half the value width): half-width Q and K tiles, full-width V."""
+    check_case(api, oracle, Case(870 + q_len, 2, q_len, (8, 2, 4), past, d=64, d_v=128),
+               f"d 64/128 q_len={q_len} past={past}")
+    assert api.last_prefill_kernel() == 2
+
+
+@pytest.mark.parametrize("page", [16, 128])
+def test_half_width_keys_paged(api, oracle, page):
+    check_case(api, oracle, Case(880 + page, 2, 200, (32, 4, 16), [100, 0], d=64, d_v=128), f"d 64/128 page={page}",
+               paged=page)
     assert api.last_prefill_kernel() == 2
 
 

@@ -39,6 +39,14 @@ def _both_ways(api, inp, num_splits):
 
 def test_static_scratch_decode_matches_workspace_decode_twice(oracle):
     from paper_2501_13629_b200 import api
+    api.set_tail_reserve(0)  # fixed tile owners: the two entry points then differ in nothing but the scratch memory
+    try:
+        _twice(api, oracle)
+    finally:
+        api.set_tail_reserve(-1)
+
+
+def _twice(api, oracle):
     big = dataclasses.replace(W.CFG2, batch=3, kv_len=2500, seed=81)
     small = dataclasses.replace(W.CFG2, batch=2, n_q=8, n_k=2, n_v=2, kv_len=300, seed=82)
     first = W.make_decode_inputs(big, seqlens=np.array([2500, 1200, 9], np.int32))
@@ -69,3 +77,23 @@ def test_static_scratch_rejects_oversized_shapes():
         api.diffqkv_decode_static(q, cache, cfg.n_k, cfg.n_v, cfg.scale, out)
     assert e.value.status == api.ERR_WORKSPACE
     assert api.launch_count() == launches  # refused on the host, nothing was launched
+
+
+def test_static_scratch_agrees_with_decode_on_an_empty_batch():
+    """batch == 0 is a valid call that does nothing, through either entry point."""
+    from paper_2501_13629_b200 import api
+    z = lambda *s: torch.zeros(s, dtype=torch.bfloat16, device="cuda")  # noqa: E731
+    cache = api.KVCache(z(1, 2, 64, 128), z(1, 2, 64, 128), torch.zeros(1, dtype=torch.int32, device="cuda"), 64)
+    q = z(1, 8, 128)  # real storage behind the pointers; the shape says batch 0 (torch gives empty tensors a null pointer)
+    out = torch.zeros((1, 8, 128), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    shape = api.make_shape(0, 8, 2, 2, 128, 128, q.dtype, out.dtype, 0.1)
+    cs = cache.c_struct()
+    launches = api.launch_count()
+    import ctypes as C
+    st = api._lib.diffqkv_decode(q.data_ptr(), C.byref(cs), C.byref(shape), 0, ws.data_ptr(), ws.numel(), out.data_ptr(),
+                                 None, None, None)
+    assert st == api.OK
+    st = api._lib.diffqkv_decode_static(q.data_ptr(), C.byref(cs), C.byref(shape), 0, out.data_ptr(), None, None, None)
+    assert st == api.OK
+    assert api.launch_count() == launches
