@@ -343,6 +343,10 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
           report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
           ok = false;
         } else {
+          // Every lane has polled the barrier on its own: all of them must have seen the slot free before lane 0
+          // hands it to the consumers, whose release would otherwise complete the barrier's next phase under the
+          // lanes still polling for this one (they would then wait until their limit and report a timeout).
+          __syncwarp();
           if (lane == 0) {
             ctrl[stage] = 0;
             ptx::mbar_arrive(full0 + 8 * stage);

@@ -293,6 +293,23 @@ def test_tail_reserve_invariance(api, oracle, blocks, tail_reserve, heads, d_qk,
         assert np.abs(o - outs[0]).max() <= 5e-3
 
 
+def test_end_of_tail_marker_is_posted_once_every_lane_saw_the_slot_free(api, oracle, blocks, tail_reserve):
+    """Blocks with only a few tiles and a one-tile reserve reach the end-of-segment marker while their ring is full:
+    the producer's lanes must all have seen the slot free before it is handed on (a lane left polling would run
+    into its limit and report a timeout although every result is right).  Repeated, since it is a matter of timing."""
+    cfg = dataclasses.replace(SMALL, batch=5, n_q=32, n_k=4, n_v=16, d_qk=64, d_v=64, kv_len=3000, seed=91)
+    inp = W.make_decode_inputs(cfg, seqlens=np.array([3000, 64, 0, 1777, 1], dtype=np.int32))
+    ref, _ = run_oracle(oracle, inp)
+    for nb in (39, 40, 41):
+        blocks(nb)
+        for reserve in (1, -1):
+            tail_reserve(reserve)
+            for _ in range(8):
+                out, _, st = run_decode(api, inp)
+                assert st == 0, f"blocks={nb} reserve={reserve}: device status {st}"
+            check_bf16(out, ref, f"blocks={nb} reserve={reserve}")
+
+
 def test_tail_reserve_full_size_every_tile_drawn(api, oracle, tail_reserve):
     """The headline shape with every tile but one per segment handed out through the counters: a stress of the
     draw protocol at 148 blocks (the automatic reserve runs in test_full_size_bf16_and_gqa_twin)."""
