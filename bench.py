@@ -143,27 +143,28 @@ class DecodeCase:
             pt = None if inp.page_table is None else torch.from_numpy(inp.page_table).to(device)
             num_blocks = inp.num_pages if pt is not None else cfg.batch
             max_seqlen, ks, vs = inp.max_seqlen, inp.k_strides, inp.v_strides
-        else:  # large pools: same recipe (i.i.d. N(0,1) rounded to bf16), drawn on the device
+        else:  # large pools: same recipe (i.i.d. N(0,1) rounded to the storage type), drawn on the device
+            dt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
             g = torch.Generator(device=device)
             g.manual_seed(cfg.seed)
             self.seqlens_host = W.draw_lengths(cfg)
-            q = torch.randn((cfg.batch, cfg.n_q, cfg.d_qk), generator=g, device=device).to(torch.bfloat16)
+            q = torch.randn((cfg.batch, cfg.n_q, cfg.d_qk), generator=g, device=device).to(dt)
             if cfg.page_size:
                 table, num_blocks = W.shuffled_page_table(self.seqlens_host, cfg.page_size, cfg.seed)
                 pt = torch.from_numpy(table).to(device)
-                k = torch.empty((num_blocks, cfg.n_k, cfg.page_size, cfg.d_qk), dtype=torch.bfloat16, device=device)
-                v = torch.empty((num_blocks, cfg.n_v, cfg.page_size, cfg.d_v), dtype=torch.bfloat16, device=device)
+                k = torch.empty((num_blocks, cfg.n_k, cfg.page_size, cfg.d_qk), dtype=dt, device=device)
+                v = torch.empty((num_blocks, cfg.n_v, cfg.page_size, cfg.d_v), dtype=dt, device=device)
                 max_seqlen = int(table.shape[1]) * cfg.page_size
             else:
                 pt, num_blocks, max_seqlen = None, cfg.batch, cfg.kv_len
-                k = torch.empty((cfg.batch, cfg.n_k, cfg.kv_len, cfg.d_qk), dtype=torch.bfloat16, device=device)
-                v = torch.empty((cfg.batch, cfg.n_v, cfg.kv_len, cfg.d_v), dtype=torch.bfloat16, device=device)
+                k = torch.empty((cfg.batch, cfg.n_k, cfg.kv_len, cfg.d_qk), dtype=dt, device=device)
+                v = torch.empty((cfg.batch, cfg.n_v, cfg.kv_len, cfg.d_v), dtype=dt, device=device)
             for t in (k, v):  # fill in slices to bound temporary memory
                 flat = t.view(-1)
                 step = 1 << 28
                 for lo in range(0, flat.numel(), step):
                     n = min(step, flat.numel() - lo)
-                    flat[lo:lo + n] = torch.randn(n, generator=g, device=device).to(torch.bfloat16)
+                    flat[lo:lo + n] = torch.randn(n, generator=g, device=device).to(dt)
             ks = (k.stride(0), k.stride(1), k.stride(2))
             vs = (v.stride(0), v.stride(1), v.stride(2))
         self.bytes = kv_bytes(cfg, self.seqlens_host)
@@ -179,11 +180,11 @@ class DecodeCase:
                                            page_size=cfg.page_size, k_strides=ks, v_strides=vs,
                                            num_blocks=num_blocks))
         self.q = q
-        self.shape = api.make_shape(cfg.batch, cfg.n_q, cfg.n_k, cfg.n_v, cfg.d_qk, cfg.d_v, q.dtype,
-                                    torch.bfloat16, cfg.scale)
+        out_dt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+        self.shape = api.make_shape(cfg.batch, cfg.n_q, cfg.n_k, cfg.n_v, cfg.d_qk, cfg.d_v, q.dtype, out_dt, cfg.scale)
         nbytes = api.diffqkv_decode_workspace_bytes(self.shape, int(max_seqlen), 0)
         self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
-        self.out = torch.empty((cfg.batch, cfg.n_q, cfg.d_v), dtype=torch.bfloat16, device=device)
+        self.out = torch.empty((cfg.batch, cfg.n_q, cfg.d_v), dtype=out_dt, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self.working_set = pool_bytes * rotate
         self._i = 0
@@ -539,6 +540,18 @@ def time_context_sweep(api, W, device, steps):
     return rows
 
 
+def time_fp32_mode(api, W, device, steps):
+    """The fp32 mode beyond the second-level cache: config 1's heads (16 query / 2 K / 4 V, 64 channels, fp32 cache) at
+    batch 4 and 65536 tokens, 403 MB of cache per step, on the generic path's unit kernel (plain loads, fp32 FMAs,
+    every K and V row read once for the eight query heads of its unit) and its combine kernel."""
+    import dataclasses
+    cfg = dataclasses.replace(W.CFG1, name="fp32_b4_64k", batch=4, kv_len=65536, seed=1500)
+    case = DecodeCase(api, cfg, device)
+    ms = case.time_steps(steps, 5) / steps
+    return {"ms_per_step": ms, "GB/s": case.bytes / ms / 1e6, "kv_bytes": case.bytes, "rotate": case.rotate,
+            "shape": "batch 4, 16/2/4 heads, d 64, 65536 tokens, fp32 cache"}
+
+
 def time_topk(api, W, device, host, steps, topk=100):
     """Selective V fetching on the headline workload: the K cache is streamed once, of V only `topk` rows per query
     head are read.  Algorithmic bytes = K bytes + gathered V rows; the fp32 scores and the per-16-token maxima are
@@ -603,6 +616,8 @@ def summarize(line, peaks):
         for name in ("augq", "attention"):
             out["cfg4_" + name] = {"TFLOP/s": round(c4[name]["TFLOP/s"], 1), "ms": r3(c4[name]["ms"]),
                                    "of_measured_burst": r3(c4[name]["frac_of_measured_bf16_burst"])}
+    if "fp32_b4_64k" in o:
+        out["fp32_64k"] = gbs(o["fp32_b4_64k"]["GB/s"])
     if "cfg3_selective_v_top100" in o:
         out["cfg3_top100_us"] = r3(o["cfg3_selective_v_top100"]["ms_per_step"] * 1e3)
     if line.get("e2e"):
@@ -650,6 +665,10 @@ def run_ours(args):
         if rank == 0:
             print(json.dumps({"workload": "cfg4 widths, 4 / 16 / 64 rows",
                               **time_augq_decode(api, W, device, max(1, min(args.steps, 200)))}))
+        return
+    if args.workload == "fp32":  # the fp32 mode alone (the command profilers wrap)
+        if rank == 0:
+            print(json.dumps({"workload": "fp32_b4_64k", **time_fp32_mode(api, W, device, max(1, min(args.steps, 50)))}))
         return
     if args.workload == "topk":  # selective V fetching on the headline workload alone (the command profilers wrap)
         if rank == 0:
@@ -726,6 +745,8 @@ def run_ours(args):
                 c_ms = cs.time_steps(args.steps, args.warmup) / args.steps
                 others[c.name] = {"ms_per_step": c_ms, "GB/s": cs.bytes / c_ms / 1e6, "rotate": cs.rotate}
                 del cs
+            torch.cuda.empty_cache()
+            others["fp32_b4_64k"] = time_fp32_mode(api, W, device, max(5, min(args.steps, 50)))
             torch.cuda.empty_cache()
             c5 = DecodeCase(api, W.CFG5, device)
             n5 = max(5, min(args.steps, 30))
@@ -833,7 +854,7 @@ def main():
     ap.add_argument("--quick", action="store_true", help="headline workload only")
     ap.add_argument("--budget-s", type=float, default=150.0,
                     help="--impl reference: seconds of oracle time the whole run may take (sizes the per-step sample)")
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "topk", "augq_decode"],
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "topk", "augq_decode", "fp32"],
                     help="decode = the headline line (default); prefill = only the config 4 timings; "
                          "topk = only selective V fetching on the headline workload; augq_decode = only the projection "
                          "chain at decode row counts")

@@ -311,6 +311,16 @@ size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape *shape, int32_t m
 diffqkv_status diffqkv_decode_topk(const void *q, const diffqkv_cache *cache, const diffqkv_shape *shape, int32_t topk,
                                    void *workspace, size_t workspace_bytes, void *out, float *lse,
                                    int32_t *dev_status, void *stream);
+/*
+ * diffqkv_decode_topk_ids -- the same, and also says which tokens were kept (for callers that audit the selection or
+ * reuse it for a later step):
+ *   kept_ids  int32 [batch, n_q, topk]: the cached positions of the tokens whose V rows entered the output of each
+ *             query head, in no particular order, padded with -1 when the sequence has fewer than topk tokens; NULL
+ *             makes the call identical to diffqkv_decode_topk
+ */
+diffqkv_status diffqkv_decode_topk_ids(const void *q, const diffqkv_cache *cache, const diffqkv_shape *shape,
+                                       int32_t topk, void *workspace, size_t workspace_bytes, void *out, float *lse,
+                                       int32_t *kept_ids, int32_t *dev_status, void *stream);
 
 /* Static, never-null description of a status value. */
 const char *diffqkv_status_string(diffqkv_status status);

@@ -54,6 +54,14 @@ void diffqkv_profile_split_events(void *before_split, void *after_split);
 int64_t diffqkv_launch_count(void);
 
 /*
+ * Test hook (process-wide host state): the generic decode path (fp32 caches, bf16 shapes without a tensor map) has
+ * two kernels, one block per (split, unit of query heads, sequence) that reads every K and V row once for all heads of
+ * the unit, and one block per (split, query head, sequence) for head counts and dimensions the first does not take.
+ * A non-zero value makes it always take the second.  Both compute the same thing.
+ */
+void diffqkv_debug_decode_per_head_only(int32_t on);
+
+/*
  * Failure-path hook for tests.  Every wait of the library's kernels on a copy in flight is bounded: when it runs
  * out the block reports DIFFQKV_ERR_TIMEOUT in *dev_status, stops computing, lets copies already in flight land,
  * and returns; results of that call are undefined, the context stays usable.  This hook makes that path reachable

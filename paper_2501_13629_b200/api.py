@@ -33,7 +33,7 @@ EXPORTS = (
     "diffqkv_last_prefill_kernel", "diffqkv_force_tensor_gemm", "diffqkv_augq_rope", "diffqkv_project", "diffqkv_cache_append",
     "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes", "diffqkv_decode_frontend",
     "diffqkv_decode_frontend_workspace_bytes", "diffqkv_decode_host", "diffqkv_fold_k_up",
-    "diffqkv_set_tail_reserve", "diffqkv_debug_decode_timeout",
+    "diffqkv_set_tail_reserve", "diffqkv_debug_decode_timeout", "diffqkv_decode_topk_ids", "diffqkv_debug_decode_per_head_only",
 )
 
 
@@ -91,6 +91,9 @@ _lib.diffqkv_cache_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINT
                                       C.c_void_p, C.c_void_p]
 _lib.diffqkv_decode_topk_workspace_bytes.restype = C.c_size_t
 _lib.diffqkv_decode_topk_workspace_bytes.argtypes = [C.POINTER(ShapeStruct), C.c_int32, C.c_int32]
+_lib.diffqkv_decode_topk_ids.restype = C.c_int
+_lib.diffqkv_decode_topk_ids.argtypes = [C.c_void_p, C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_int32, C.c_void_p,
+                                         C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.diffqkv_decode_topk.restype = C.c_int
 _lib.diffqkv_decode_topk.argtypes = [C.c_void_p, C.POINTER(CacheStruct), C.POINTER(ShapeStruct), C.c_int32, C.c_void_p,
                                      C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -115,6 +118,8 @@ _lib.diffqkv_last_prefill_kernel.restype = C.c_int32
 _lib.diffqkv_last_prefill_kernel.argtypes = []
 _lib.diffqkv_topk_general_only.restype = None
 _lib.diffqkv_topk_general_only.argtypes = [C.c_int32]
+_lib.diffqkv_debug_decode_per_head_only.restype = None
+_lib.diffqkv_debug_decode_per_head_only.argtypes = [C.c_int32]
 _lib.diffqkv_debug_decode_timeout.restype = None
 _lib.diffqkv_debug_decode_timeout.argtypes = [C.c_int64, C.c_int64]
 _lib.diffqkv_set_tail_reserve.restype = None
@@ -161,6 +166,11 @@ KERNEL_NONE, KERNEL_GENERIC, KERNEL_TMA = 0, 1, 2
 def set_tail_reserve(tiles: int) -> None:
     """Tail balance of the TMA decode kernel: -1 automatic, 0 off (run-to-run bitwise reproducible), n tiles per block."""
     _lib.diffqkv_set_tail_reserve(int(tiles))
+
+
+def decode_per_head_only(on: bool) -> None:
+    """Test hook: the generic decode path never takes its unit kernel (one block per query head instead)."""
+    _lib.diffqkv_debug_decode_per_head_only(1 if on else 0)
 
 
 def debug_decode_timeout(wait_limit_ns: int = 0, skip_tile: int = -1) -> None:
@@ -504,8 +514,10 @@ def diffqkv_fold_k_up(q: torch.Tensor, W_kup: torch.Tensor, out: Optional[torch.
 def diffqkv_decode_topk(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: float, topk: int,
                         workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
                         lse: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
-                        out_dtype: Optional[torch.dtype] = None, stream: Optional[torch.cuda.Stream] = None):
-    """Decode that reads only the V rows of the `topk` highest scores of every query head."""
+                        out_dtype: Optional[torch.dtype] = None, stream: Optional[torch.cuda.Stream] = None,
+                        kept_ids: Optional[torch.Tensor] = None):
+    """Decode that reads only the V rows of the `topk` highest scores of every query head; ``kept_ids`` (int32
+    [batch, n_q, topk]) receives the kept tokens' positions, -1 padded."""
     batch, n_q, d_qk = q.shape
     d_v = cache.v.shape[-1]
     out_dtype = out_dtype or (out.dtype if out is not None else q.dtype)
@@ -516,8 +528,10 @@ def diffqkv_decode_topk(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, sca
     if out is None:
         out = torch.empty((batch, n_q, d_v), dtype=out_dtype, device=q.device)
     cs = cache.c_struct()
-    st = _lib.diffqkv_decode_topk(_p(q), C.byref(cs), C.byref(shape), int(topk), _p(workspace), workspace.numel(),
-                                  _p(out), _p(lse), _p(dev_status), _stream_ptr(stream))
+    if kept_ids is not None:
+        assert kept_ids.dtype == torch.int32 and kept_ids.is_contiguous() and tuple(kept_ids.shape) == (batch, n_q, topk)
+    st = _lib.diffqkv_decode_topk_ids(_p(q), C.byref(cs), C.byref(shape), int(topk), _p(workspace), workspace.numel(),
+                                      _p(out), _p(lse), _p(kept_ids), _p(dev_status), _stream_ptr(stream))
     if st != OK:
         raise DiffQKVError(st, "diffqkv_decode_topk")
     return out

@@ -12,12 +12,12 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 DecodePlan plan_decode(const diffqkv_shape& shape, int max_seqlen, int num_splits) {
   if (max_seqlen < 1) max_seqlen = 1;
   int want = num_splits;
-  if (want <= 0) {  // automatic: chunks of about 512 tokens, shorter when that leaves most SMs idle; at most 32 splits
+  if (want <= 0) {  // automatic: chunks of about 512 tokens, shorter when that leaves most SMs idle; at most 64 splits
     want = (max_seqlen + 511) / 512;
     const long long rows = (long long)shape.batch * shape.n_q;
     const long long fill = rows > 0 ? (592 + rows - 1) / rows : 1;  // about four blocks per SM
     if (want < fill) want = (int)fill;
-    if (want > 32) want = 32;
+    if (want > 64) want = 64;
   }
   if (want < 1) want = 1;
   int chunk = (max_seqlen + want - 1) / want;
@@ -186,6 +186,8 @@ size_t diffqkv_decode_workspace_bytes(const diffqkv_shape* shape, int32_t max_se
 void diffqkv_set_max_blocks(int32_t max_blocks) { set_tma_max_blocks(max_blocks); }
 
 void diffqkv_set_tail_reserve(int32_t tiles) { set_tma_tail_reserve(tiles); }
+
+void diffqkv_debug_decode_per_head_only(int32_t on) { set_decode_per_head_only(on); }
 
 void diffqkv_debug_decode_timeout(int64_t wait_limit_ns, int64_t skip_tile) {
   set_tma_debug_timeout(wait_limit_ns, skip_tile);
@@ -411,9 +413,9 @@ size_t diffqkv_decode_topk_workspace_bytes(const diffqkv_shape* shape, int32_t m
   return topk_decode_workspace_bytes(*shape, max_seqlen, topk);
 }
 
-diffqkv_status diffqkv_decode_topk(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape, int32_t topk,
-                                   void* workspace, size_t workspace_bytes, void* out, float* lse, int32_t* dev_status,
-                                   void* stream) {
+diffqkv_status diffqkv_decode_topk_ids(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape,
+                                       int32_t topk, void* workspace, size_t workspace_bytes, void* out, float* lse,
+                                       int32_t* kept_ids, int32_t* dev_status, void* stream) {
   diffqkv_status st = check_shape(shape);
   if (st != DIFFQKV_OK) return st;
   if (!q || !out || topk < 1) return DIFFQKV_ERR_INVALID_ARG;
@@ -426,9 +428,15 @@ diffqkv_status diffqkv_decode_topk(const void* q, const diffqkv_cache* cache, co
   if (!workspace || workspace_bytes < topk_decode_workspace_bytes(*shape, cache->max_seqlen, topk)) return DIFFQKV_ERR_WORKSPACE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DIFFQKV_ERR_ALIGNMENT;
   const cudaError_t err = launch_decode_topk(q, *cache, *shape, topk, box_tok, workspace, out, lse, dev_status,
-                                             static_cast<cudaStream_t>(stream));
+                                             static_cast<cudaStream_t>(stream), kept_ids);
   if (err == cudaErrorNotSupported) return DIFFQKV_ERR_UNSUPPORTED;
   return err == cudaSuccess ? DIFFQKV_OK : DIFFQKV_ERR_CUDA;
+}
+
+diffqkv_status diffqkv_decode_topk(const void* q, const diffqkv_cache* cache, const diffqkv_shape* shape, int32_t topk,
+                                   void* workspace, size_t workspace_bytes, void* out, float* lse, int32_t* dev_status,
+                                   void* stream) {
+  return diffqkv_decode_topk_ids(q, cache, shape, topk, workspace, workspace_bytes, out, lse, nullptr, dev_status, stream);
 }
 
 const char* diffqkv_status_string(diffqkv_status status) {

@@ -59,6 +59,7 @@ cudaError_t launch_prefill_generic(const DecodeParams& p, diffqkv_dtype dtype, i
 cudaError_t launch_combine(const float* o_partial, const float* lse_partial, int rows, int d_v, int splits,
                            diffqkv_dtype out_dtype, void* out, float* lse, cudaStream_t stream);
 void count_launch(int n = 1);
+void set_decode_per_head_only(int on);  // test hook: the generic decode never takes the unit kernel
 
 // Linear layers for at most kSkinnyMaxRows rows of x (weight-streaming kernel, linear_skinny.cu); same operands as the
 // tensor-core GEMM of augq.cu: C[M, N] = A[M, K] . B0[N, K]^T, with B1 silu(A.B0^T) * (A.B1^T), with rope_cos/rope_sin
@@ -127,6 +128,7 @@ bool topk_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, int t
 size_t topk_decode_workspace_bytes(const diffqkv_shape& s, int max_seqlen, int topk);
 void set_topk_general_only(int on);
 cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, int topk, int box_tok,
-                               void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream);
+                               void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream,
+                               int* kept_ids = nullptr);
 
 }  // namespace diffqkv

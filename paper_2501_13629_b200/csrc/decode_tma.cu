@@ -35,6 +35,8 @@
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "tmap.cuh"
+#include "walker.cuh"
 
 namespace diffqkv {
 namespace {
@@ -88,30 +90,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
-// Position in the flat (sequence, unit, tile) list.
-struct Walker {
-  long long g;  // flat tile index
-  int b, u, t, nt;
-  __device__ void seek(long long g0, const int* prefix, int batch, int n_units) {
-    g = g0;
-    int lo = 0, hi = batch;  // smallest b' with n_units * prefix[b'] > g; answer b = b' - 1
-    while (lo < hi) {
-      const int mid = (lo + hi) >> 1;
-      if ((long long)n_units * prefix[mid] > g0) hi = mid; else lo = mid + 1;
-    }
-    b = lo - 1;
-    nt = prefix[b + 1] - prefix[b];
-    const long long rem = g0 - (long long)n_units * prefix[b];
-    u = (int)(rem / nt);
-    t = (int)(rem % nt);
-  }
-  __device__ void next_sequence(const int* prefix, int batch) {
-    do {
-      ++b;
-      nt = b < batch ? prefix[b + 1] - prefix[b] : 1;
-    } while (b < batch && nt == 0);
-  }
-};
+using Walker = FlatWalker;  // position in the flat (sequence, unit, tile) list
 
 // SHARED: neighbouring units read the same K or V head (see k_shift / v_shift); the plain case keeps its own code.
 template <int D_QK, int D_V, int KPU, int VPU, bool SHARED = false>
@@ -745,27 +724,11 @@ combine_segments_kernel(const float* __restrict__ o_partial, const float* __rest
 }
 
 // ---------------------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = [] {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      ptr = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(ptr);
-  }();
-  return fn;
-}
-
 // Tensor map over one cache pool: dims (64 channels, token slot, channel half, head, block); one box
 // brings box_tok tokens x all halves of one head, each half landing as 128-byte swizzled rows.
 bool make_pool_map(CUtensorMap* map, const void* base, int d, long long tok_extent, int heads, long long blocks,
                    long long st_tok, long long st_head, long long st_blk, int box_tok) {
-  EncodeTiledFn fn = encode_fn();
+  TmapEncodeTiledFn fn = tmap_encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[5] = {64, (cuuint64_t)tok_extent, (cuuint64_t)(d / 64), (cuuint64_t)heads, (cuuint64_t)blocks};
   const cuuint64_t strides[4] = {(cuuint64_t)st_tok * 2, 128, (cuuint64_t)st_head * 2, (cuuint64_t)st_blk * 2};

@@ -19,6 +19,7 @@
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "walker.cuh"
 #include "tmap.cuh"
 
 namespace diffqkv {
@@ -50,37 +51,7 @@ struct ScoreParams {
   int* dev_status;
 };
 
-// Position in the flat (sequence, K head, tile) list.
-struct TileWalker {
-  long long g;
-  int b, u, t, nt;
-  __device__ void seek(long long g0, const int* prefix, int batch, int n_units) {
-    g = g0;
-    int lo = 0, hi = batch;  // smallest b' with n_units * prefix[b'] > g; answer b = b' - 1
-    while (lo < hi) {
-      const int mid = (lo + hi) >> 1;
-      if ((long long)n_units * prefix[mid] > g0) hi = mid; else lo = mid + 1;
-    }
-    b = lo - 1;
-    nt = prefix[b + 1] - prefix[b];
-    const long long rem = g0 - (long long)n_units * prefix[b];
-    u = (int)(rem / nt);
-    t = (int)(rem % nt);
-  }
-  __device__ void advance(const int* prefix, int batch, int n_units) {
-    ++g;
-    if (++t == nt) {
-      t = 0;
-      if (++u == n_units) {
-        u = 0;
-        do {
-          ++b;
-          nt = b < batch ? prefix[b + 1] - prefix[b] : 1;
-        } while (b < batch && nt == 0);
-      }
-    }
-  }
-};
+using TileWalker = FlatWalker;  // position in the flat (sequence, K head, tile) list
 
 template <int D_QK, int NG>  // NG: groups of 8 query heads per K head
 __global__ void __launch_bounds__(score_threads(NG), 1)
@@ -289,6 +260,7 @@ struct AttendParams {
   float* lse;
   int out_is_f32;
   int* dev_status;
+  int* kept_ids;  // [batch, n_q, topk] cached positions of the kept tokens (-1 padded), or NULL
 };
 
 // Larger float <=> larger key.
@@ -803,6 +775,8 @@ topk_attend_kernel(const AttendParams p) {
       else reinterpret_cast<__nv_bfloat16*>(p.out)[orow + ch] = __float2bfloat16_rn(0.f);
     }
     if (p.lse && tid == 0) p.lse[(long long)b * p.n_q + h] = -INFINITY;
+    if (p.kept_ids)
+      for (int i = tid; i < p.topk; i += kAttendThreads) p.kept_ids[(long long)blockIdx.x * p.topk + i] = -1;
     return;
   }
   const float* row = p.scores + (long long)blockIdx.x * p.lpad;
@@ -833,6 +807,9 @@ topk_attend_kernel(const AttendParams p) {
     for (int i = tid; i < k; i += kAttendThreads) sel_idx[i] = mtok[sel_idx[i]];
     __syncthreads();
   }
+
+  if (p.kept_ids)  // which tokens were kept (in no particular order), for callers that check or reuse the selection
+    for (int i = tid; i < p.topk; i += kAttendThreads) p.kept_ids[(long long)blockIdx.x * p.topk + i] = i < k ? sel_idx[i] : -1;
 
   // ---- softmax over the kept scores (base-2 domain)
   float m = -INFINITY;
@@ -972,7 +949,8 @@ static std::atomic<int> g_topk_general_only{0};  // test hook
 void set_topk_general_only(int on) { g_topk_general_only = on != 0; }
 
 cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diffqkv_shape& s, int topk, int box_tok,
-                               void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream) {
+                               void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream,
+                               int* kept_ids) {
   const int sms = sm_count_topk();
   if (sms <= 0) return cudaErrorUnknown;
   int dev = 0, max_smem = 0;
@@ -1056,6 +1034,7 @@ cudaError_t launch_decode_topk(const void* q, const diffqkv_cache& c, const diff
   ap.batch = s.batch; ap.n_q = s.n_q; ap.n_v = s.n_v; ap.d_v = s.d_v; ap.topk = topk;
   ap.out = out; ap.lse = lse; ap.out_is_f32 = s.out_dtype == DIFFQKV_F32;
   ap.dev_status = dev_status;
+  ap.kept_ids = kept_ids;
   cfg.gridDim = dim3((unsigned)rows);
   cfg.blockDim = dim3(kAttendThreads);
   cfg.dynamicSmemBytes =

@@ -462,3 +462,60 @@ def test_split_counts_beyond_the_combine_limit_are_refused_before_any_launch(api
                            workspace=torch.zeros(1 << 20, dtype=torch.uint8, device="cuda"))
     assert e.value.status == api.ERR_UNSUPPORTED
     assert api.launch_count() == launches
+
+
+@pytest.fixture
+def per_head_only(api):
+    """Switches the generic decode path to its one-block-per-query-head kernel and back."""
+    yield api.decode_per_head_only
+    api.decode_per_head_only(False)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("heads,d_qk,d_v", [((16, 2, 4), 64, 64), ((32, 4, 8), 128, 128), ((12, 6, 2), 128, 64),
+                                            ((8, 8, 1), 64, 256), ((8, 1, 8), 256, 128), ((4, 4, 4), 128, 128),
+                                            ((8, 2, 2), 64, 128)])
+def test_generic_unit_kernel_and_per_head_kernel(api, oracle, per_head_only, dtype, heads, d_qk, d_v):
+    """The generic path's unit kernel (every K and V row read once for all query heads of its unit) and its
+    one-block-per-head kernel against the oracle and each other: fp32 and bf16 storage, nested head groups in both
+    directions, mixed head dimensions, ragged and empty sequences, contiguous and paged, one and several splits."""
+    n_q, n_k, n_v = heads
+    cfg = dataclasses.replace(SMALL, batch=4, n_q=n_q, n_k=n_k, n_v=n_v, d_qk=d_qk, d_v=d_v, kv_len=1100, dtype=dtype,
+                              seed=77)
+    inp = W.make_decode_inputs(cfg, seqlens=np.array([1100, 1, 0, 517], dtype=np.int32))
+    ref, lse_ref = run_oracle(oracle, inp)
+    check = check_f32 if dtype == "f32" else check_bf16
+    for case in (inp, W.paginate(inp, 16, seed=5)):
+        for splits in (1, 5):
+            outs = []
+            for only in (False, True):
+                per_head_only(only)
+                out, lse, st = run_decode(api, case, num_splits=splits)
+                assert st == 0 and api.last_decode_kernel() == api.KERNEL_GENERIC
+                check(out, ref, f"{heads} {d_qk}/{d_v} {dtype} splits={splits} per_head={only}")
+                check_lse(lse, lse_ref, 1e-4 if dtype == "f32" else 2e-2)
+                assert np.all(out[2] == 0) and np.all(np.isneginf(lse[2]))
+                outs.append(out)
+            assert np.abs(outs[0] - outs[1]).max() <= (1e-5 if dtype == "f32" else 5e-3) * max(np.abs(ref).max(), 1.0)
+
+
+@pytest.mark.parametrize("heads,d", [((6, 3, 2), 64), ((16, 2, 4), 96), ((32, 1, 2), 64)])
+def test_generic_shapes_the_unit_kernel_does_not_take(api, oracle, heads, d):
+    """Head groups that do not nest, head dimensions other than 64 / 128 / 256 and more than eight query heads per
+    unit stay on the one-block-per-head kernel (fp32 storage)."""
+    n_q, n_k, n_v = heads
+    cfg = dataclasses.replace(SMALL, batch=2, n_q=n_q, n_k=n_k, n_v=n_v, d_qk=d, d_v=d, kv_len=600, dtype="f32", seed=78)
+    inp = W.make_decode_inputs(cfg, seqlens=np.array([600, 77], dtype=np.int32))
+    ref, lse_ref = run_oracle(oracle, inp)
+    out, lse, st = run_decode(api, inp)
+    assert st == 0
+    check_f32(out, ref, f"{heads} d={d}")
+    check_lse(lse, lse_ref, 1e-4)
+
+
+def test_unit_kernel_reports_pages_outside_the_pool(api):
+    cfg = dataclasses.replace(SMALL, batch=1, kv_len=256, dtype="f32")
+    inp = W.paginate(W.make_decode_inputs(cfg), 16, seed=1)
+    inp.page_table[0, 3] = inp.num_pages + 5
+    _, _, st = run_decode(api, inp)
+    assert st == 1 << api.ERR_INDEX

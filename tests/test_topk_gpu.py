@@ -182,3 +182,48 @@ def test_topk_argument_errors(api):
     with pytest.raises(api.DiffQKVError) as e:
         api.diffqkv_decode_topk(q, cache, 2, 4, 0.1, 10, workspace=torch.zeros(256, dtype=torch.uint8, device="cuda"))
     assert e.value.status == api.ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("topk,paged", [(1, 0), (7, 16), (100, 0), (100, 64), (1024, 0)])
+def test_kept_token_ids_are_a_valid_selection(api, oracle, topk, paged):
+    """diffqkv_decode_topk_ids returns which tokens entered each head's output.  Several sets can be right when
+    scores at the cut differ by less than fp32 scoring resolves, so the unique part is compared and the rest is
+    checked for validity: min(topk, len) distinct visible tokens; on rows the inputs decide (gap at the cut above
+    the scoring error) exactly the oracle's set; on the others every kept score at least every dropped score minus
+    the scoring error (scores from the definition, in float64); -1 padding behind short sequences."""
+    cfg = dataclasses.replace(SMALL, seed=95)
+    lens = np.array([3000, 129, 0], np.int32)
+    inp = W.make_decode_inputs(cfg, seqlens=lens)
+    # equal keys make equal scores: part of the selection is then decided by the tie rule alone
+    inp.k[0, :, 1000:1040] = inp.k[0, :, 1000:1001]
+    case = W.paginate(inp, paged, seed=3) if paged else inp
+    q, cache = W.to_torch(case.q, "cuda"), device_cache(api, case)
+    ids = torch.full((cfg.batch, cfg.n_q, topk), -7, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = api.diffqkv_decode_topk(q, cache, cfg.n_k, cfg.n_v, cfg.scale, topk, dev_status=status,
+                                  out_dtype=torch.float32, kept_ids=ids)
+    plain = api.diffqkv_decode_topk(q, cache, cfg.n_k, cfg.n_v, cfg.scale, topk, out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(out, plain)
+    ids = ids.cpu().numpy()
+    _, _, sel, margin = oracle.decode_topk(inp.q, oracle_cache(oracle, inp), cfg.n_q, cfg.n_k, cfg.n_v, cfg.d_qk,
+                                           cfg.d_v, cfg.scale, topk)
+    qf, kf = W.as_f64(inp.q), W.as_f64(inp.k)
+    for b in range(cfg.batch):
+        n = int(lens[b])
+        for h in range(cfg.n_q):
+            kept = ids[b, h]
+            k = min(topk, n)
+            got = kept[kept >= 0]
+            assert len(got) == k and np.all(kept[k:] == -1), (b, h)
+            assert len(set(got.tolist())) == k and (k == 0 or (got.min() >= 0 and got.max() < n)), (b, h)
+            if k == 0:
+                continue
+            want = set(sel[b, h][sel[b, h] >= 0].tolist())
+            if margin[b, h] > 2 * SCORE_EPS:
+                assert set(got.tolist()) == want, f"row ({b},{h}): kept set differs from the oracle's"
+            else:
+                s = cfg.scale * (kf[b, h * cfg.n_k // cfg.n_q, :n] @ qf[b, h])
+                dropped = np.setdiff1d(np.arange(n), got)
+                if len(dropped):
+                    assert s[got].min() >= s[dropped].max() - 2 * SCORE_EPS, f"row ({b},{h}): not a top-{topk} set"
