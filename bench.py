@@ -394,6 +394,19 @@ def time_prefill(api, W, device, peaks, steps):
     fl64 = 2.0 * cfg.batch * cfg.n_q * (cfg.seq * (cfg.seq + 1) / 2) * (2 * d64)
     res["attention_sigma1p5b_heads_d64"] = {"ms": ms64, "TFLOP/s": fl64 / ms64 / 1e9, "flops": fl64,
                                             "heads": "32 query / 4 K / 16 V, 64 channels"}
+    del q64, k64n, v64n, cache64, out64
+    # keys cached at half the value width (d_qk 64, d_v 128; queries folded through the K feed-forward layer first)
+    w_kup = rn(cfg.n_k, cfg.d_v, 64, std=64 ** -0.5)
+    qh = torch.empty(cfg.batch, cfg.seq, cfg.n_q, 64, dtype=torch.bfloat16, device=device)
+    kh_new = rn(cfg.batch, cfg.seq, cfg.n_k, 64)
+    cache_h = api.KVCache(torch.zeros(cfg.batch, cfg.n_k, cfg.seq, 64, dtype=torch.bfloat16, device=device), v,
+                          torch.zeros(cfg.batch, dtype=torch.int32, device=device), cfg.seq)
+    fold_ms = timed(lambda: api.diffqkv_fold_k_up(q4, w_kup, out=qh))
+    ms_h = timed(lambda: api.diffqkv_prefill(qh, kh_new, v_new, cache_h, cfg.scale, out=out, dev_status=status))
+    assert int(status.item()) == 0, "device status reported an error"
+    fl_h = 2.0 * cfg.batch * cfg.n_q * (cfg.seq * (cfg.seq + 1) / 2) * (64 + cfg.d_v)
+    res["attention_half_width_keys"] = {"ms": ms_h, "TFLOP/s": fl_h / ms_h / 1e9, "flops": fl_h, "fold_k_up_ms": fold_ms,
+                                        "heads": "32 query / 4 K / 8 V, d_qk 64, d_v 128"}
     return res
 
 

@@ -401,7 +401,7 @@ diffqkv_status diffqkv_fold_k_up(const void* q, const void* W_kup, int64_t T, in
                                  int32_t d_k, void* q_out, void* stream) {
   if (!q || !W_kup || !q_out) return DIFFQKV_ERR_INVALID_ARG;
   if (T < 0 || n_q <= 0 || n_k <= 0 || d_q <= 0 || d_k <= 0 || n_q % n_k != 0) return DIFFQKV_ERR_INVALID_ARG;
-  if (T * n_k > 0x7fffffffLL) return DIFFQKV_ERR_UNSUPPORTED;
+  if (T > 0x7fffffffLL) return DIFFQKV_ERR_UNSUPPORTED;
   if (T == 0) return DIFFQKV_OK;
   const cudaError_t err = launch_fold_kup(q, W_kup, T, n_q, n_k, d_q, d_k, q_out, static_cast<cudaStream_t>(stream));
   if (err == cudaErrorNotSupported) return DIFFQKV_ERR_UNSUPPORTED;
