@@ -722,7 +722,7 @@ def run_ours(args):
 
     e2e = None
     if not args.profile:  # every rank runs the end-to-end loop at the same time; the slowest one counts
-        n_e2e = min(args.steps, 500)
+        n_e2e = min(max(args.steps, 200), 500)  # a short --steps would leave this host-timed figure to a few samples
         if barrier:
             barrier()
         e2e_ms, h2d, d2h = case.time_e2e(n_e2e, min(args.warmup, 20))
@@ -735,7 +735,7 @@ def run_ours(args):
         print(json.dumps(line))
     elif rank == 0:
         # roofline of the dominant (split) kernel, timed alone by events the library records around it
-        k_ms = case.time_split_kernel(min(args.steps, 200))
+        k_ms = case.time_split_kernel(min(max(args.steps, 100), 200))
         ach = case.bytes / (k_ms * 1e-3) / 1e9
         line["roofline"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                             "frac": ach / peaks["hbm_gbs"], "traffic": split_kernel_dram_bytes(),
@@ -743,19 +743,20 @@ def run_ours(args):
                             "kernel_ms": k_ms, "peak_source": peaks["source"] + " (burst copy)"}
         line["e2e"] = e2e
         others = {}
+        so = max(args.steps, 300)  # steps for the other configurations: their figures should not hinge on a short --steps
         if not args.quick and world == 1:
             twin = DecodeCase(api, cfg.gqa_twin(), device, host_inputs=W.make_decode_inputs(cfg.gqa_twin()))
-            t_ms = twin.time_steps(args.steps, args.warmup) / args.steps
+            t_ms = twin.time_steps(so, args.warmup) / so
             others["cfg3_gqa_twin"] = {"ms_per_step": t_ms, "GB/s": twin.bytes / t_ms / 1e6,
                                        "tokens_per_s_per_layer": cfg.batch / (t_ms * 1e-3)}
             line["diffqkv_vs_gqa_speedup_32k"] = t_ms / ms_per_step
             del twin
-            tk = time_topk(api, W, device, host, min(args.steps, 300))
+            tk = time_topk(api, W, device, host, 300)
             tk["speedup_vs_full_v"] = ms_per_step / tk["ms_per_step"]
             others["cfg3_selective_v_top100"] = tk
             for c in (W.CFG2, W.CFG2.gqa_twin(), W.CFG1):
                 cs = DecodeCase(api, c, device, host_inputs=W.make_decode_inputs(c))
-                c_ms = cs.time_steps(args.steps, args.warmup) / args.steps
+                c_ms = cs.time_steps(so, args.warmup) / so
                 others[c.name] = {"ms_per_step": c_ms, "GB/s": cs.bytes / c_ms / 1e6, "rotate": cs.rotate}
                 del cs
             torch.cuda.empty_cache()
@@ -773,9 +774,9 @@ def run_ours(args):
             others["augq_at_decode"] = time_augq_decode(api, W, device, 200)
             others["decode_step_cfg3"] = time_decode_step(api, W, device, host, 200)
             torch.cuda.empty_cache()
-            others["sigma1p5b_vs_std_heads"] = time_sigma_table(api, W, device, max(20, min(args.steps, 300)))
+            others["sigma1p5b_vs_std_heads"] = time_sigma_table(api, W, device, 300)
             torch.cuda.empty_cache()
-            others["diffqkv_vs_gqa_over_context"] = time_context_sweep(api, W, device, max(20, min(args.steps, 200)))
+            others["diffqkv_vs_gqa_over_context"] = time_context_sweep(api, W, device, 200)
         line["others"] = others
         if world == 1:
             line["cpu_baseline"] = cpu_baseline(host, budget_s=12.0)
