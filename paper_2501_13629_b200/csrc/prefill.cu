@@ -19,8 +19,10 @@
 //                 (tcgen05.st), where the second product reads it; the first 64 tokens of P are announced on a
 //                 barrier of their own, so that half of the second product runs under the rest of the exponentials.
 //   fp32 scores, softmax statistics and output accumulation; P is rounded to bf16 for the second product.
-//   The kernel is a template on the head dimension (128 or 64 channels for Q/K and V alike): with 64 the tiles are
-//   half as wide, the first product takes four K steps instead of eight and O takes 64 TMEM columns per M-tile.
+//   The kernel is a template on the head dimensions (channels of Q/K and of V): (128, 128), (64, 64) with half-width
+//   tiles, four K steps in the first product and 64 TMEM columns of O per M-tile, and (64, 128) for keys cached at half
+//   the value width.  With 64-channel values P has tensor-memory columns of its own, and the next tile's scores are
+//   issued as soon as the softmax warps hold the current ones (see kSepP).
 // Every wait is bounded; on expiry the block reports DIFFQKV_ERR_TIMEOUT, drains and frees its TMEM.
 #include "common.cuh"
 #include "ptx.cuh"
@@ -82,6 +84,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   constexpr int kQBytes = kQT * kDQK * 2;   // a Q tile: [half][128 rows][128 B]
   constexpr int kKBytes = kKT * kDQK * 2;   // a K tile: [half][128 rows][128 B]
   constexpr int kTBytes = kKT * kD * 2;     // a V tile: [half][128 rows][128 B]
+  // With 64-channel values the two output accumulators take 128 of the 512 tensor-memory columns instead of 256, which
+  // leaves room for P outside the score columns: [S0 128][S1 128][O0 64][O1 64][P0 64][P1 64].  The next tile's
+  // scores can then be issued as soon as the softmax warps have taken the current ones into registers, instead of
+  // after the product that reads P, and the softmax warps find them ready when they come back.
+  constexpr bool kSepP = kD == 64;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* q_s = smem;                      // 2 M-tiles
@@ -95,7 +102,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   const uint32_t s_full0 = v_empty0 + 8 * kVSlots, p_full0 = s_full0 + 16, o_done0 = p_full0 + 16;
   const uint32_t drain = o_done0 + 16;
   const uint32_t p_half0 = drain + 8;  // the first 64 tokens of P_t are in place
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 + 2 * kKSlots + 2 * kVSlots + 6 + 2);
+  const uint32_t s_free0 = p_half0 + 16;  // (kSepP) the scores of M-tile t have been read out of tensor memory
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 + 2 * kKSlots + 2 * kVSlots + 6 + 2 + 2);
   volatile int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -114,6 +122,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       ptx::mbar_init(s_full0 + 8 * t, 1);
       ptx::mbar_init(p_full0 + 8 * t, 4);
       ptx::mbar_init(p_half0 + 8 * t, 4);
+      ptx::mbar_init(s_free0 + 8 * t, 4);
       ptx::mbar_init(o_done0 + 8 * t, 1);
     }
     ptx::mbar_init(drain, 1);
@@ -230,7 +239,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       // second half of P_t
       auto issue_pv = [&](int t, int slot, bool first, int half) {
         const uint32_t va = v_lo + slot * (kTBytes >> 4);
-        const uint32_t d = tmem_base + 256 + t * kD, pa = tmem_base + t * 128;
+        const uint32_t d = tmem_base + 256 + t * kD, pa = kSepP ? tmem_base + 384 + t * 64 : tmem_base + t * 128;
         constexpr int kSteps = kKT / 32;  // K steps of 16 tokens per half
         if (half == 0) {
           if (first) tc::mma_ts_halves<false>(d, pa, va, hi, idesc_pv);
@@ -254,6 +263,42 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       }
       int ks = 1 % kKSlots, vs = 0;  // slot of K tile j + 1, slot of V tile j
       uint32_t kph = 0, vph = 0;
+      if (kSepP) {
+        for (int j = 0; j < nkv_max && ok; ++j) {
+          // the next tile's scores first: their columns are free once the softmax warps hold the current ones
+          if (j + 1 < nkv_max) {
+            if (!ptx::mbar_wait(k_full0 + 8 * ks, kph, abort_flag)) { ok = false; break; }
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+              if (j + 1 < nkv[t]) {
+                if (!ptx::mbar_wait(s_free0 + 8 * t, j & 1, abort_flag)) { ok = false; break; }
+                tc::fence_after_sync();
+                issue_s(t, ks);
+              }
+            }
+            if (!ok) break;
+            tc::commit(k_empty0 + 8 * ks);
+          }
+#pragma unroll
+          for (int t = 0; t < 2; ++t) {
+            if (j < nkv[t]) {
+              if (!ptx::mbar_wait(p_half0 + 8 * t, j & 1, abort_flag) || !ptx::mbar_wait(v_full0 + 8 * vs, vph, abort_flag)) {
+                ok = false;
+                break;
+              }
+              tc::fence_after_sync();
+              issue_pv(t, vs, j == 0, 0);
+              if (!ptx::mbar_wait(p_full0 + 8 * t, j & 1, abort_flag)) { ok = false; break; }
+              tc::fence_after_sync();
+              issue_pv(t, vs, j == 0, 1);
+            }
+          }
+          if (!ok) break;
+          tc::commit(v_empty0 + 8 * vs);  // every MMA that reads V tile j has been issued
+          if (++ks == kKSlots) { ks = 0; kph ^= 1; }
+          if (++vs == kVSlots) { vs = 0; vph ^= 1; }
+        }
+      } else {
       for (int j = 0; j < nkv_max && ok; ++j) {
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
@@ -279,6 +324,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         if (++ks == kKSlots) { ks = 0; kph ^= 1; }
         if (++vs == kVSlots) { vs = 0; vph ^= 1; }
       }
+      }
       if (!ok) report(p.dev_status, DIFFQKV_ERR_TIMEOUT);
       tc::commit(drain);
     }
@@ -293,7 +339,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       const int qrow = q0 + t * kQT + r;
       const int qpos = past + qrow;
       const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-      const uint32_t s_taddr = lane_base + t * 128;  // scores, and P over their first 64 columns
+      const uint32_t s_taddr = lane_base + t * 128;  // scores, and (unless P has columns of its own) P over their first 64
+      const uint32_t p_taddr = kSepP ? lane_base + 384 + t * 64 : s_taddr;
       const uint32_t o_taddr = lane_base + 256 + t * kD;
       float m_ref = -INFINITY, l = 0.f;
       bool ok = true;
@@ -307,6 +354,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
 #pragma unroll
         for (int c = 0; c < 4; ++c) tc::ld_32x32b_x32(s_taddr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
         tc::wait_ld();
+        if (kSepP) {  // the score columns may take the next tile's scores from here on
+          tc::fence_before_sync();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(s_free0 + 8 * t);
+        }
         if (diag) {
 #pragma unroll
           for (int e = 0; e < 128; ++e)
@@ -360,6 +412,10 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         }
         // ---- P = 2^(S scale - m_ref) as packed bf16 over the first 64 score columns; fp32 row sum.  The first 64
         // tokens are announced on their own, so that their half of the product runs during the second half's work.
+        if (kSepP && j > 0) {  // P's own columns still hold the previous tile's P until its product is done
+          if (!wait_warp(o_done0 + 8 * t, (j - 1) & 1, abort_flag)) { ok = false; break; }
+          tc::fence_after_sync();
+        }
         float l0 = 0.f, l1 = 0.f;
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
@@ -372,7 +428,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             l0 += p0;
             l1 += p1;
           }
-          tc::st_32x32b_x32(s_taddr + c * 32, w);
+          tc::st_32x32b_x32(p_taddr + c * 32, w);
           if (c == 0) {
             tc::wait_st();
             tc::fence_before_sync();
