@@ -288,8 +288,10 @@ diffqkv_status diffqkv_decode_frontend(const void *h, const void *W_Q, const voi
  *   q      [T, n_q, d_q] bf16      W_kup [n_k, d_q, d_k] bf16      q_out [T, n_q, d_k] bf16 (fp32 accumulation)
  * Call sequence for the half-width cache: diffqkv_fold_k_up, then diffqkv_decode / diffqkv_prefill /
  * diffqkv_decode_topk with shape.d_qk = d_k (64 with d_v = 128 runs on the TMA and tensor-core kernels) and the
- * same scale the full-width scores would use.  (n_q / n_k) * d_q may not exceed 3072 and d_q must be a multiple of 4
- * (DIFFQKV_ERR_UNSUPPORTED otherwise).
+ * same scale the full-width scores would use.  Runs on the tensor cores when d_q is a multiple of 16 up to 256, d_k
+ * is 32, 64 or 128 and not above d_q, and the three pointers are 16-byte aligned; every other shape takes a plain
+ * kernel, for which (n_q / n_k) * d_q may not exceed 3072 and d_q must be a multiple of 4 (DIFFQKV_ERR_UNSUPPORTED
+ * otherwise).
  */
 diffqkv_status diffqkv_fold_k_up(const void *q, const void *W_kup, int64_t T, int32_t n_q, int32_t n_k, int32_t d_q,
                                  int32_t d_k, void *q_out, void *stream);

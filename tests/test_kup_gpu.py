@@ -51,15 +51,29 @@ def test_decode_over_half_width_keys(api, oracle, heads):
     check_lse(lse.cpu().numpy().astype(np.float64), lse_ref, 2e-2, f"heads {heads}")
 
 
-def test_folded_queries_match_the_definition(api):
-    """q' = W[hk]^T q per head, against the same product in float64 (every element, 2^-8 relative to the row)."""
-    n_q, n_k, d_q, d_k, T = 12, 3, 128, 64, 37
+@pytest.mark.parametrize("n_q,n_k,d_q,d_k,T", [
+    (12, 3, 128, 64, 37),     # tensor-core kernel, 148 rows per K head: one full 128-row tile and a ragged one
+    (32, 4, 128, 64, 1000),   # several tiles per block
+    (16, 16, 64, 32, 9),      # groups of one head, a single 16-row slab partly filled
+    (8, 2, 256, 128, 131),    # the widest layer the tensor-core kernel takes
+    (6, 2, 128, 32, 50),      # a group size that does not divide the slab height
+    (4, 4, 64, 64, 300),      # square layer
+    (8, 2, 96, 48, 21),       # d_k not a multiple of 32: the plain kernel
+    (12, 4, 100, 20, 13),     # d_q not a multiple of 16: the plain kernel
+    (8, 4, 64, 128, 40),      # a widening layer: the plain kernel
+])
+def test_folded_queries_match_the_definition(api, n_q, n_k, d_q, d_k, T):
+    """q' = W[hk]^T q per head, against the same product in float64: every element within one bf16 rounding of the
+    exact value (half a unit in the last of eight significant bits: 2^-8 relative) plus the fp32 accumulation's share."""
     q, w = W.normal(511, (T, n_q, d_q)), W.normal(512, (n_k, d_q, d_k), std=d_k ** -0.5)
-    got = api.diffqkv_fold_k_up(W.to_torch(q, "cuda"), W.to_torch(w, "cuda")).float().cpu().numpy().astype(np.float64)
+    out = torch.full((T, n_q, d_k), float("nan"), dtype=torch.bfloat16, device="cuda")
+    api.diffqkv_fold_k_up(W.to_torch(q, "cuda"), W.to_torch(w, "cuda"), out=out)
+    got = out.float().cpu().numpy().astype(np.float64)
     qf, wf = W.as_f64(q), W.as_f64(w)
     for h in range(n_q):
         ref = qf[:, h] @ wf[h // (n_q // n_k)]
-        assert np.abs(got[:, h] - ref).max() <= 2.0 ** -8 * np.abs(ref).max()
+        err = np.abs(got[:, h] - ref)
+        assert np.all(err <= 2.0 ** -8 * np.abs(ref) + 2e-5 * np.abs(ref).max()), (h, err.max())
 
 
 @pytest.mark.parametrize("q_len,past", [(300, [0, 0]), (257, [100, 31]), (1, [5, 0])])
