@@ -12,10 +12,13 @@
 //                 token-major tile); the two M-tiles alternate, so the tensor core works on one while the softmax
 //                 warps work on the other.  Operands are what bounds these products (about 100 bytes per cycle
 //                 reach the tensor core from shared memory), hence 128-wide tiles and P kept out of shared memory.
-//     warps 2-5   softmax of M-tile 0, warps 6-9 of M-tile 1: one thread per query row (= TMEM lane).  The thread
+//     warps 2-3   idle: they complete the first group of four warps, which hands most of its registers to the
+//                 softmax warps (setmaxnreg works on aligned groups of four warps)
+//     warps 4-7   softmax of M-tile 0, warps 8-11 of M-tile 1: one thread per query row (= TMEM lane).  The thread
 //                 reads its 128 scores into registers (tcgen05.ld), takes the row maximum (a running reference
 //                 maximum is only raised when exceeded by 2^8; then O is rescaled in TMEM), computes
-//                 P = 2^(S scale - m), sums it in fp32 and writes it as packed bf16 over the first 64 score columns
+//                 P = 2^(S scale - m) (scale-and-shift and row sum as packed fp32 pairs, to leave the issue slots
+//                 to the exponentials), sums it in fp32 and writes it as packed bf16 over the first 64 score columns
 //                 (tcgen05.st), where the second product reads it; the first 64 tokens of P are announced on a
 //                 barrier of their own, so that half of the second product runs under the rest of the exponentials.
 //   fp32 scores, softmax statistics and output accumulation; P is rounded to bf16 for the second product.
@@ -36,7 +39,11 @@ constexpr int kQT = 128;  // query rows per M-tile
 constexpr int kKT = 128;  // cached tokens per KV tile
 constexpr int kDMax = 128;  // channels per head (Q/K and V): the kernel is built for 128 and for 64
 constexpr int kKSlots = 3, kVSlots = 2;
-constexpr int kPrefillThreads = 320;
+// Three groups of four warps: {TMA producer, MMA issuer, two idle warps}, the softmax warps of M-tile 0 and those of
+// M-tile 1.  The first group hands most of its registers to the other two (setmaxnreg works on aligned groups of four
+// warps): 12 x 168 = 4 x 56 + 8 x 224.
+constexpr int kPrefillThreads = 384;
+constexpr int kSoftmaxWarp0 = 4;
 constexpr int kTmemCols = 512;         // S[t] (and P[t] over its first 64 columns) at 128 t, O[t] at 256 + D t
 // Shared memory is sized for D = 128 whatever D is: one block per SM, since a block takes all of the tensor memory.
 constexpr int kPrefillSmem = 1024 + 2 * (kQT * kDMax * 2) + (kKSlots + kVSlots) * (kKT * kDMax * 2) + 256;
@@ -71,6 +78,31 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return d;
 }
 
+// Packed fp32 pairs (one instruction, two lanes of the FMA pipe over two cycles: half the issue slots of the scalar
+// forms, which is what the softmax warps are short of next to their special-function instructions).
+__device__ __forceinline__ uint64_t pair(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ uint64_t pair(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpair(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity, abort_flag));
 }
@@ -158,6 +190,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   const int nkv_max = max(nkv[0], nkv[1]);
   const uint32_t q_u32 = ptx::smem_u32(q_s), k_u32 = ptx::smem_u32(k_s), v_u32 = ptx::smem_u32(v_s);
 
+  if (warp < kSoftmaxWarp0) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -329,9 +363,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       tc::commit(drain);
     }
     __syncwarp();
+  }
   } else {
     // ------------------------------------------------------------------ softmax warps
-    const int t = (warp - 2) >> 2;  // M-tile
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    const int t = (warp - kSoftmaxWarp0) >> 2;  // M-tile
     const int quarter = warp & 3;   // TMEM lanes this warp may touch
     const int r = quarter * 32 + lane;
     const int n = nkv[t];
@@ -416,17 +452,20 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           if (!wait_warp(o_done0 + 8 * t, (j - 1) & 1, abort_flag)) { ok = false; break; }
           tc::fence_after_sync();
         }
-        float l0 = 0.f, l1 = 0.f;
+        // Scale-and-shift and the row sum are packed: with a special-function instruction taking most of the issue
+        // slots of its eight cycles, the other instructions of the loop are what the exponentials wait for.
+        uint64_t l2 = 0;  // two partial row sums
+        const uint64_t scale2 = pair(p.scale_log2, p.scale_log2), negm2 = pair(neg_m, neg_m);
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           uint32_t w[32];
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            const float p0 = ex2(fmaf(__uint_as_float(s[c * 64 + 2 * e]), p.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(s[c * 64 + 2 * e + 1]), p.scale_log2, neg_m));
+            float x0, x1;
+            unpair(fma2(pair(s[c * 64 + 2 * e], s[c * 64 + 2 * e + 1]), scale2, negm2), x0, x1);
+            const float p0 = ex2(x0), p1 = ex2(x1);
             w[e] = pack2(p0, p1);
-            l0 += p0;
-            l1 += p1;
+            l2 = add2(l2, pair(p0, p1));
           }
           tc::st_32x32b_x32(p_taddr + c * 32, w);
           if (c == 0) {
@@ -436,6 +475,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             if (lane == 0) ptx::mbar_arrive(p_half0 + 8 * t);
           }
         }
+        float l0, l1;
+        unpair(l2, l0, l1);
         l += l0 + l1;
         tc::wait_st();
         tc::fence_before_sync();
