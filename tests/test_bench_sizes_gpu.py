@@ -214,3 +214,23 @@ def test_fused_gate_up_kernel_blocks_walk_many_tiles(api, oracle):
     ref = oracle.augq(h, *ws, rows=rows)
     got = q[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
     check_proj(got, ref, "aug-Q over 512 fused tiles")
+
+
+def test_fold_of_the_k_layer_at_config4_rows(api):
+    """diffqkv_fold_k_up over config 4's 16 384 query rows of 32 heads (every block of the tensor-core kernel walks
+    several 128-row tiles and the last block a ragged one: T is taken one row short): sampled rows, every head and
+    channel, against the float64 product (Section 2: K brought to the query width by a feed-forward layer)."""
+    n_q, n_k, d_q, d_k, T = 32, 4, 128, 64, 16383
+    q, w = W.normal(9101, (T, n_q, d_q)), W.normal(9102, (n_k, d_q, d_k), std=d_k ** -0.5)
+    out = torch.full((T, n_q, d_k), float("nan"), dtype=torch.bfloat16, device="cuda")
+    api.diffqkv_fold_k_up(W.to_torch(q, "cuda"), W.to_torch(w, "cuda"), out=out)
+    torch.cuda.synchronize()
+    rows = np.unique(np.concatenate([np.arange(0, 40), np.arange(8000, 8040), np.arange(T - 40, T),
+                                     np.random.default_rng(5).integers(0, T, 200)]))
+    got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+    assert not torch.isnan(out.float()).any(), "rows left unwritten"
+    qf, wf = W.as_f64(q[rows]), W.as_f64(w)
+    for h in range(n_q):
+        ref = qf[:, h] @ wf[h // (n_q // n_k)]
+        err = np.abs(got[:, h] - ref)
+        assert np.all(err <= 2.0 ** -8 * np.abs(ref) + 2e-5 * np.abs(ref).max()), (h, err.max())
