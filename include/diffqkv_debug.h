@@ -62,6 +62,17 @@ int64_t diffqkv_launch_count(void);
 void diffqkv_debug_decode_per_head_only(int32_t on);
 
 /*
+ * Test hook (process-wide host state) for the on-chip merge of the TMA decode kernel.  With few, short rows the
+ * blocks that share a (sequence, head group) row are launched as a thread-block cluster and the first of them merges
+ * the others' partial results out of their shared memory; no partials go through global memory and no combine kernel
+ * is launched.  Automatically this is done when the largest power of two of blocks per row (at most 8) fills four
+ * fifths of the SMs and the cache holds at most 160 MB for these rows; results differ from the two-kernel path only
+ * in fp32 summation order.
+ *   mode < 0  automatic (default)    mode = 0  never    mode > 0  whenever at least two blocks per row fit on the GPU
+ */
+void diffqkv_debug_decode_cluster(int32_t mode);
+
+/*
  * Failure-path hook for tests.  Every wait of the library's kernels on a copy in flight is bounded: when it runs
  * out the block reports DIFFQKV_ERR_TIMEOUT in *dev_status, stops computing, lets copies already in flight land,
  * and returns; results of that call are undefined, the context stays usable.  This hook makes that path reachable

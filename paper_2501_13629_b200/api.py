@@ -33,7 +33,7 @@ EXPORTS = (
     "diffqkv_last_prefill_kernel", "diffqkv_force_tensor_gemm", "diffqkv_augq_rope", "diffqkv_project", "diffqkv_cache_append",
     "diffqkv_decode_topk", "diffqkv_decode_topk_workspace_bytes", "diffqkv_decode_frontend",
     "diffqkv_decode_frontend_workspace_bytes", "diffqkv_decode_host", "diffqkv_fold_k_up",
-    "diffqkv_set_tail_reserve", "diffqkv_debug_decode_timeout", "diffqkv_decode_topk_ids", "diffqkv_debug_decode_per_head_only",
+    "diffqkv_set_tail_reserve", "diffqkv_debug_decode_timeout", "diffqkv_decode_topk_ids", "diffqkv_debug_decode_per_head_only", "diffqkv_debug_decode_cluster",
 )
 
 
@@ -120,6 +120,8 @@ _lib.diffqkv_topk_general_only.restype = None
 _lib.diffqkv_topk_general_only.argtypes = [C.c_int32]
 _lib.diffqkv_debug_decode_per_head_only.restype = None
 _lib.diffqkv_debug_decode_per_head_only.argtypes = [C.c_int32]
+_lib.diffqkv_debug_decode_cluster.restype = None
+_lib.diffqkv_debug_decode_cluster.argtypes = [C.c_int32]
 _lib.diffqkv_debug_decode_timeout.restype = None
 _lib.diffqkv_debug_decode_timeout.argtypes = [C.c_int64, C.c_int64]
 _lib.diffqkv_set_tail_reserve.restype = None
@@ -166,6 +168,11 @@ KERNEL_NONE, KERNEL_GENERIC, KERNEL_TMA = 0, 1, 2
 def set_tail_reserve(tiles: int) -> None:
     """Tail balance of the TMA decode kernel: -1 automatic, 0 off (run-to-run bitwise reproducible), n tiles per block."""
     _lib.diffqkv_set_tail_reserve(int(tiles))
+
+
+def decode_cluster(mode: int) -> None:
+    """Test hook: on-chip merge of the TMA decode kernel (-1 automatic, 0 never, 1 whenever the shape allows)."""
+    _lib.diffqkv_debug_decode_cluster(int(mode))
 
 
 def decode_per_head_only(on: bool) -> None:

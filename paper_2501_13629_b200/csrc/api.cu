@@ -188,6 +188,7 @@ void diffqkv_set_max_blocks(int32_t max_blocks) { set_tma_max_blocks(max_blocks)
 void diffqkv_set_tail_reserve(int32_t tiles) { set_tma_tail_reserve(tiles); }
 
 void diffqkv_debug_decode_per_head_only(int32_t on) { set_decode_per_head_only(on); }
+void diffqkv_debug_decode_cluster(int32_t mode) { set_tma_cluster_mode(mode); }
 
 void diffqkv_debug_decode_timeout(int64_t wait_limit_ns, int64_t skip_tile) {
   set_tma_debug_timeout(wait_limit_ns, skip_tile);

@@ -91,6 +91,7 @@ struct TmaPlan {
   int stages, grid, smem;
   long long slots;   // partial-result slots: grid + batch * units
   int reserve, reserve_auto;  // tail reserve per block in tiles (0 = none); auto: also at most a sixth of a block's share
+  int cluster;       // 0, or the blocks per (sequence, unit) row that merge through each other's shared memory
 };
 bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPlan* plan);
 size_t tma_decode_workspace_bytes(const diffqkv_shape& s, const TmaPlan& plan);
@@ -98,6 +99,7 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
                               void* workspace, void* out, float* lse, int* dev_status, cudaStream_t stream);
 void set_tma_max_blocks(int n);
 void set_tma_tail_reserve(int n);
+void set_tma_cluster_mode(int mode);  // -1 automatic, 0 never, 1 whenever the shape allows
 void set_tma_debug_timeout(long long wait_limit_ns, long long skip_tile);
 
 // Augmented-Q projection (augq.cu): three tcgen05 GEMMs, the gate/up pair fused with its silu-gate epilogue.

@@ -30,6 +30,7 @@
 #include <cuda.h>
 
 #include <atomic>
+#include <vector>
 #include <mutex>
 #include <random>
 
@@ -51,6 +52,7 @@ constexpr int kHeadsPerMma = 8;
 constexpr int kMaxBatchTma = 2048;  // the per-sequence tile prefix lives in shared memory
 // Hook state: process-wide, set and read from any calling thread, hence atomics.
 std::atomic<int> g_max_blocks{0};     // tuning / test hook: 0 = one block per SM
+std::atomic<int> g_cluster_mode{-1};  // test hook: -1 = automatic, 0 = never, 1 = whenever the shape allows
 std::atomic<int> g_tail_reserve{-1};  // tuning / test hook: -1 = automatic, 0 = no reserve, n = at most n tiles per block
 std::atomic<long long> g_wait_limit_ns{0};  // test hook: 0 = the default limit of every bounded wait
 std::atomic<long long> g_skip_tile{-1};     // test hook: flat tile whose copies are never issued (-1 = none)
@@ -77,6 +79,7 @@ struct TmaParams {
   int reserve_auto;           // 1: and never more than a sixth of a block's share
   unsigned long long wait_ns; // limit of every bounded wait
   long long skip_tile;        // test hook: flat tile whose copies the producer does not issue (-1 = none)
+  int cluster;                // 0, or blocks per (sequence, unit) row: the row's blocks form a cluster and merge on chip
   void* out;
   float* lse;
   int out_is_f32;
@@ -116,6 +119,10 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   int* prefix = const_cast<int*>(abort_flag) + 2;                                 // [batch + 1]
   int* lens_s = prefix + p.batch + 1;                                             // [batch] lengths, clamped
   volatile int* ctrl = lens_s + p.batch;  // [stages] tail phase: valid tokens of the tile in the stage, 0 = no more tiles
+  // (cluster mode) this block's share of its row for the on-chip merge: [8 heads][D_V] normalised outputs and their
+  // base-2 log-sum-exps, over the first stage of the ring, which is free once the block's last tile has been consumed
+  float* xo = reinterpret_cast<float*>(stage_base);
+  float* xl = xo + kHeadsPerMma * D_V;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t full0 = ptx::smem_u32(bars), empty0 = ptx::smem_u32(bars + p.stages);
@@ -168,20 +175,36 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   // Only min(grid, total) blocks take part, so that every participating block owns at least one tile
   // (the combine kernel relies on the blocks between a row's first and last owner all having written).
   const long long nblk = min((long long)gridDim.x, total);
-  if (blockIdx.x >= nblk) return;
-  const long long g_begin = (total * blockIdx.x) / nblk;
-  const long long g_end = (total * (blockIdx.x + 1)) / nblk;
+  if (!p.cluster && blockIdx.x >= nblk) return;
+  long long g_begin = 0, g_end = 0;
+  if (p.cluster) {
+    // Cluster mode (short rows): the p.cluster blocks of a cluster share one (sequence, unit) row, each takes an equal
+    // run of its tiles and the first block merges all of them out of the others' shared memory: no partials in global
+    // memory and no second kernel.  Every thread of every block reaches the two cluster barriers at the end.
+    const int row = (int)blockIdx.x / p.cluster, rank = (int)blockIdx.x % p.cluster;
+    const int b = row / p.n_units, u = row % p.n_units;
+    const long long nt = prefix[b + 1] - prefix[b];
+    const long long lo = (long long)p.n_units * prefix[b] + u * nt;
+    g_begin = lo + nt * rank / p.cluster;
+    g_end = lo + nt * (rank + 1) / p.cluster;
+  } else {
+    g_begin = (total * blockIdx.x) / nblk;
+    g_end = (total * (blockIdx.x + 1)) / nblk;
+  }
+  const bool have_tiles = g_begin < g_end;
 
   // ---- the tail reserve: the last R tiles of this block's last segment (never all of the segment)
-  const int reserve = p.reserve_auto ? (int)min((long long)p.reserve, (total / nblk) / 6) : p.reserve;
+  const int reserve = p.cluster ? 0 : (p.reserve_auto ? (int)min((long long)p.reserve, (total / nblk) / 6) : p.reserve);
   Walker wl;  // the row (sequence, unit) of the last segment
-  wl.seek(g_end - 1, prefix, p.batch, p.n_units);
+  wl.b = 0; wl.u = 0; wl.nt = 0; wl.t = 0; wl.g = 0;
+  if (have_tiles) wl.seek(g_end - 1, prefix, p.batch, p.n_units);
   const long long row_lo = (long long)p.n_units * prefix[wl.b] + (long long)wl.u * wl.nt, row_hi = row_lo + wl.nt;
   const int R = reserve > 0 ? min(reserve, (int)(g_end - max(g_begin, row_lo)) - 1) : 0;
   const long long g_stat = g_end - R;  // tiles [g_begin, g_stat) are this block's own
 
   Walker w;
-  w.seek(g_begin, prefix, p.batch, p.n_units);
+  w.b = 0; w.u = 0; w.nt = 0; w.t = 0; w.g = g_begin;
+  if (have_tiles) w.seek(g_begin, prefix, p.batch, p.n_units);
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer warp
@@ -346,6 +369,10 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         const int uses = (issued - s + p.stages - 1) / p.stages;
         ptx::mbar_wait(full0 + 8 * s, (uint32_t)(uses - 1) & 1u, nullptr, p.wait_ns);
       }
+    }
+    if (p.cluster) {  // the two barriers of the on-chip merge (see the end of the kernel)
+      ptx::cluster_sync();
+      ptx::cluster_sync();
     }
     return;
   }
@@ -565,7 +592,12 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         }
         const float inv = 1.f / L;
         const float lse2 = M + log2f(L);
-        if (whole) {
+        if (p.cluster) {  // this block's share of the row, for the first block of the cluster to merge
+          float* dst = xo + col * D_V + ch0;
+#pragma unroll
+          for (int e = 0; e < CPT; ++e) dst[e] = o[e] * inv;
+          if (ch0 == 0) xl[col] = lse2;
+        } else if (whole) {
           const long long orow = ((long long)w.b * p.n_q + (long long)w.u * p.U + col) * D_V + ch0;
           if (p.out_is_f32) {
             float* dst = reinterpret_cast<float*>(p.out) + orow;
@@ -595,6 +627,57 @@ decode_tma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
       w.t = 0;
       if (++w.u == p.n_units) { w.u = 0; w.next_sequence(prefix, p.batch); }
     }
+  }
+
+  if (p.cluster) {
+    // ---- on-chip merge of the row's shares.  A block without tiles (fewer tiles than blocks, an empty sequence)
+    // contributes log-sum-exp -inf.  First barrier: every share is in place; then the first block of the cluster reads
+    // them out of its peers' shared memory (same weights as the combine kernel: 2^(lse_r - max)) and writes the row;
+    // second barrier: nobody leaves, and gives up its shared memory, before that is done.
+    constexpr int TPH = (kConsumerWarps * 32) / kHeadsPerMma;
+    constexpr int CPT = D_V / TPH;
+    const int col = tid / TPH, ch0 = (tid % TPH) * CPT;
+    if (!have_tiles && tid < kHeadsPerMma) xl[tid] = -INFINITY;
+    ptx::cluster_sync();
+    const int row = (int)blockIdx.x / p.cluster, rank = (int)blockIdx.x % p.cluster;
+    if (rank == 0 && col < p.U) {
+      const uint32_t xl_u32 = ptx::smem_u32(xl + col), xo_u32 = ptx::smem_u32(xo + col * D_V + ch0);
+      float M = -INFINITY;
+      for (int r = 0; r < p.cluster; ++r) M = fmaxf(M, ptx::ld_cluster_f32(ptx::cluster_map(xl_u32, r)));
+      float L = 0.f, o[CPT];
+#pragma unroll
+      for (int e = 0; e < CPT; ++e) o[e] = 0.f;
+      if (M > -INFINITY) {
+        for (int r = 0; r < p.cluster; ++r) {
+          const float lr = ptx::ld_cluster_f32(ptx::cluster_map(xl_u32, r));
+          if (lr == -INFINITY) continue;
+          const float wgt = exp2f(lr - M);
+          L += wgt;
+          const uint32_t src = ptx::cluster_map(xo_u32, r);
+#pragma unroll
+          for (int e = 0; e < CPT; e += 4) {
+            const float4 v = ptx::ld_cluster_f32x4(src + e * 4);
+            o[e] = fmaf(wgt, v.x, o[e]); o[e + 1] = fmaf(wgt, v.y, o[e + 1]);
+            o[e + 2] = fmaf(wgt, v.z, o[e + 2]); o[e + 3] = fmaf(wgt, v.w, o[e + 3]);
+          }
+        }
+      }
+      const float inv = L > 0.f ? 1.f / L : 0.f;
+      const int b = row / p.n_units, u = row % p.n_units;
+      const long long orow = ((long long)b * p.n_q + (long long)u * p.U + col) * D_V + ch0;
+      if (p.out_is_f32) {
+        float* dst = reinterpret_cast<float*>(p.out) + orow;
+#pragma unroll
+        for (int e = 0; e < CPT; ++e) dst[e] = o[e] * inv;
+      } else {
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + orow;
+#pragma unroll
+        for (int e = 0; e < CPT; ++e) dst[e] = __float2bfloat16_rn(o[e] * inv);
+      }
+      if (p.lse && ch0 == 0)
+        p.lse[(long long)b * p.n_q + (long long)u * p.U + col] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+    }
+    ptx::cluster_sync();
   }
 }
 
@@ -786,6 +869,39 @@ bool pick_variant(int d_qk, int d_v, int kpu, int vpu, Variant* v) {
   return false;
 }
 
+// How many clusters of `size` blocks of this kernel (one block per SM at `smem` bytes) the GPU runs at once; asked of
+// the driver once per (kernel, shared memory, size) and device.
+int max_active_clusters(KernelFn fn, int smem, int size) {
+  struct Entry { KernelFn fn; int smem, size, dev, n; };
+  static std::mutex mu;
+  static std::vector<Entry> seen;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  std::lock_guard<std::mutex> lock(mu);
+  for (const Entry& e : seen)
+    if (e.fn == fn && e.smem == smem && e.size == size && e.dev == dev) return e.n;
+  int n = 0;
+  if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) == cudaSuccess) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)size);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess) {
+      n = 0;
+      cudaGetLastError();  // not an error of the call being served
+    }
+  }
+  seen.push_back(Entry{fn, smem, size, dev, n});
+  return n;
+}
+
 }  // namespace
 
 bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPlan* plan) {
@@ -854,11 +970,67 @@ bool tma_decode_supported(const diffqkv_shape& s, const diffqkv_cache& c, TmaPla
   const int tail_reserve = g_tail_reserve.load();
   plan->reserve = tail_reserve < 0 ? kAutoReserve : tail_reserve;
   plan->reserve_auto = tail_reserve < 0;
+  // Cluster mode: with few, short rows the step is mostly fixed costs (the partials' trip through global memory, the
+  // second launch and its dependency, about 4 us), and a row's blocks can merge through each other's shared memory
+  // instead.  The blocks per row are chosen (2 to 8, the portable cluster size) to cover as many SMs as possible with
+  // all clusters resident at once (one block takes a whole SM's shared memory, and a cluster has to fit one GPC: the
+  // driver says how many clusters of each size can run together).  It is taken when the streaming time lost on the
+  // SMs left idle is less than those 4 us; lengths are not known here, so the cache's capacity stands in for them.
+  plan->cluster = 0;
+  const int mode = g_cluster_mode.load();
+  // blocks per row for units of `u_heads` query heads on kernel `fn`, 0 when the mode does not pay
+  auto blocks_per_row = [&](int u_heads, KernelFn fn, int smem, int stage_bytes) -> int {
+    const long long rows = (long long)s.batch * (s.n_q / u_heads);
+    if (mode == 0 || max_blocks > 0 || !fn || rows * 2 > di.sms) return 0;
+    int best = 0;
+    for (int per_row = 8; per_row >= 2; --per_row) {
+      if (rows * per_row > di.sms || per_row <= best) continue;
+      if (rows <= max_active_clusters(fn, smem, per_row)) best = per_row;
+    }
+    if (best < 2) return 0;
+    const double cover = (double)(rows * best) / di.sms;
+    const double cap_bytes = (double)rows * c.max_seqlen * (stage_bytes / kTT);
+    // (below 0.85 of the SMs the rows' tiles also divide badly over the blocks: 16 rows of 64 tiles on 7 blocks
+    // each measured slower than the two-kernel path on all 148 SMs)
+    return (mode > 0 || (cover >= 0.85 && cap_bytes * (1.0 / cover - 1.0) <= 26e6)) ? best : 0;
+  };
+  int per_row = blocks_per_row(U, (k_shift || v_shift) ? v.fn_shared : v.fn, plan->smem, v.stage_bytes);
+  if (per_row == 0 && mode != 0 && U % 2 == 0) {
+    // Too few rows: halve the units.  Each half takes half of the unit's K and V heads, or shares the head when the
+    // unit has only one (its two halves then stream that head twice, the second time mostly out of L2: they run at
+    // the same time in neighbouring clusters).  Worth it only here, where the step is not bound by bandwidth.
+    int kpu2 = kpu, vpu2 = vpu, ks2 = k_shift, vs2 = v_shift;
+    if (kpu2 % 2 == 0) kpu2 /= 2; else if (kpu2 == 1) ++ks2; else kpu2 = 0;
+    if (vpu2 % 2 == 0) vpu2 /= 2; else if (vpu2 == 1) ++vs2; else vpu2 = 0;
+    Variant v2;
+    if (kpu2 > 0 && vpu2 > 0 && pick_variant(s.d_qk, s.d_v, kpu2, vpu2, &v2) && (!(ks2 || vs2) || v2.fn_shared)) {
+      int stages2 = (di.max_smem - fixed) / v2.stage_bytes;
+      if (stages2 > 8) stages2 = 8;
+      const int smem2 = fixed + stages2 * v2.stage_bytes;
+      const int pr2 = stages2 >= 2 ? blocks_per_row(U / 2, (ks2 || vs2) ? v2.fn_shared : v2.fn, smem2, v2.stage_bytes) : 0;
+      if (pr2 > 0) {
+        per_row = pr2;
+        U /= 2;
+        plan->U = U; plan->kpu = kpu2; plan->vpu = vpu2; plan->k_shift = ks2; plan->v_shift = vs2;
+        plan->stages = stages2;
+        plan->smem = smem2;
+      }
+    }
+  }
+  if (per_row > 0) {
+    const long long rows = (long long)s.batch * (s.n_q / U);
+    plan->cluster = per_row;
+    plan->grid = (int)(rows * per_row);
+    plan->slots = plan->grid + rows;
+    plan->reserve = 0;
+    plan->reserve_auto = 0;
+  }
   return true;
 }
 
 void set_tma_max_blocks(int n) { g_max_blocks = n > 0 ? n : 0; }
 void set_tma_tail_reserve(int n) { g_tail_reserve = n < 0 ? -1 : (n > 4096 ? 4096 : n); }
+void set_tma_cluster_mode(int mode) { g_cluster_mode = mode < 0 ? -1 : (mode > 0 ? 1 : 0); }
 void set_tma_debug_timeout(long long wait_limit_ns, long long skip_tile) {
   g_wait_limit_ns = wait_limit_ns > 0 ? wait_limit_ns : 0;
   g_skip_tile = skip_tile >= 0 ? skip_tile : -1;
@@ -919,6 +1091,7 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
   const long long wait_ns = g_wait_limit_ns.load();
   p.wait_ns = wait_ns > 0 ? (unsigned long long)wait_ns : ptx::kWaitLimitNs;
   p.skip_tile = g_skip_tile.load();
+  p.cluster = plan.cluster;
   p.out = out; p.lse = lse; p.out_is_f32 = s.out_dtype == DIFFQKV_F32;
   p.dev_status = dev_status;
 
@@ -928,13 +1101,17 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
   if (err != cudaSuccess) return err;
   // both kernels may start before their predecessor in the stream has finished; each waits on the device
   // before it touches anything the predecessor may still be producing
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = (unsigned)(plan.cluster > 0 ? plan.cluster : 1);
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.stream = stream;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = plan.cluster > 0 ? 2 : 1;
   cfg.gridDim = dim3((unsigned)plan.grid);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = (size_t)plan.smem;
@@ -942,6 +1119,8 @@ cudaError_t launch_decode_tma(const void* q, const diffqkv_cache& c, const diffq
   if (err != cudaSuccess) return err;
   count_launch();
   profile_after_split(stream);
+  if (plan.cluster > 0) return cudaGetLastError();  // the rows were merged on chip
+  cfg.numAttrs = 1;
   const long long rows = (long long)s.batch * s.n_q;
   cfg.gridDim = dim3((unsigned)rows);
   cfg.blockDim = dim3(128);

@@ -519,3 +519,81 @@ def test_unit_kernel_reports_pages_outside_the_pool(api):
     inp.page_table[0, 3] = inp.num_pages + 5
     _, _, st = run_decode(api, inp)
     assert st == 1 << api.ERR_INDEX
+
+
+@pytest.fixture
+def cluster_mode(api):
+    """Sets the on-chip-merge mode of the TMA kernel and always restores the automatic choice."""
+    yield api.decode_cluster
+    api.decode_cluster(-1)
+
+
+@pytest.mark.parametrize("heads,d_qk,d_v", [((16, 2, 4), 128, 128), ((32, 4, 16), 64, 64), ((8, 4, 1), 128, 128),
+                                            ((32, 1, 2), 128, 128), ((16, 2, 4), 64, 128), ((8, 8, 8), 128, 128)])
+def test_rows_merged_on_chip_by_a_cluster(api, oracle, cluster_mode, heads, d_qk, d_v):
+    """The blocks of a (sequence, unit) row as a thread-block cluster whose first block merges the others' shares out
+    of their shared memory: one launch, no partials in global memory.  Against the oracle and against the two-kernel
+    path, with rows of 47 tiles, of one tile (fewer tiles than blocks: most blocks of the cluster have none), of one
+    token and empty ones, NaN bit patterns behind every sequence end, contiguous and paged."""
+    n_q, n_k, n_v = heads
+    cfg = dataclasses.replace(SMALL, batch=5, n_q=n_q, n_k=n_k, n_v=n_v, d_qk=d_qk, d_v=d_v, kv_len=3000, seed=93)
+    lens = np.array([3000, 64, 0, 1777, 1], dtype=np.int32)
+    inp = W.make_decode_inputs(cfg, seqlens=lens)
+    for b, n in enumerate(lens):
+        inp.k[b, :, n:] = 0x7FC0  # bf16 NaN
+        inp.v[b, :, n:] = 0x7FC0
+    ref, lse_ref = run_oracle(oracle, inp)
+    for paged in (0, 16, 128):
+        case = W.paginate(inp, paged, seed=7) if paged else inp
+        cluster_mode(0)
+        n0 = api.launch_count()
+        out2, lse2, st2 = run_decode(api, case)
+        two = api.launch_count() - n0
+        cluster_mode(1)
+        n0 = api.launch_count()
+        out, lse, st = run_decode(api, case)
+        one = api.launch_count() - n0
+        what = f"{heads} d={d_qk}/{d_v} paged={paged}"
+        assert st == 0 and st2 == 0 and api.last_decode_kernel() == api.KERNEL_TMA, what
+        assert (one, two) == (1, 2), what + f": launches {one} / {two}"
+        check_bf16(out, ref, what)
+        check_lse(lse, lse_ref, 2e-2, what)
+        assert np.all(out[2] == 0) and np.all(np.isneginf(lse[2])), what
+        assert np.abs(out - out2).max() <= 5e-3, what
+
+
+def test_cluster_merge_is_chosen_for_short_rows_only(api, oracle, cluster_mode):
+    """Left to itself the library merges on chip where the fixed costs dominate (16 sequences of 4096 tokens: 32 rows of
+    four blocks) and keeps the two-kernel path where the SMs it would leave idle cost more (the same heads at 8 times
+    the capacity)."""
+    short = dataclasses.replace(SMALL, batch=16, n_q=16, n_k=2, n_v=4, d_qk=128, d_v=128, kv_len=4096, seed=94)
+    inp = W.make_decode_inputs(short)
+    n0 = api.launch_count()
+    out, lse, st = run_decode(api, inp)
+    assert st == 0 and api.launch_count() - n0 == 1
+    pairs = np.array([(0, 0), (3, 7), (15, 15), (9, 4)], dtype=np.int32)
+    ref, _ = run_oracle(oracle, inp, pairs=pairs)
+    check_bf16(out[pairs[:, 0], pairs[:, 1]], ref[pairs[:, 0], pairs[:, 1]], "short rows")
+    # four sequences of the long-context heads have 16 rows, too few for clusters that fill the GPU: the units are
+    # halved (two halves share their K head), which makes 32 rows of four blocks
+    halves = dataclasses.replace(SMALL, batch=4, n_q=32, n_k=4, n_v=8, d_qk=128, d_v=128, kv_len=4096, seed=95)
+    inp = W.make_decode_inputs(halves, seqlens=np.array([4096, 4000, 77, 2049], dtype=np.int32))
+    n0 = api.launch_count()
+    out, lse, st = run_decode(api, inp)
+    assert st == 0 and api.launch_count() - n0 == 1
+    ref, lse_ref = run_oracle(oracle, inp)
+    check_bf16(out, ref, "halved units")
+    check_lse(lse, lse_ref, 2e-2, "halved units")
+    cluster_mode(0)
+    out2, _, _ = run_decode(api, inp)
+    cluster_mode(-1)
+    assert np.abs(out - out2).max() <= 5e-3
+    long_rows = dataclasses.replace(short, batch=2, kv_len=262144)
+    q = torch.zeros(2, 16, 128, dtype=torch.bfloat16, device="cuda")
+    cache = api.KVCache(torch.zeros(2, 2, 262144, 128, dtype=torch.bfloat16, device="cuda"),
+                        torch.zeros(2, 4, 262144, 128, dtype=torch.bfloat16, device="cuda"),
+                        torch.tensor([5000, 262144], dtype=torch.int32, device="cuda"), 262144)
+    n0 = api.launch_count()
+    api.diffqkv_decode(q, cache, 2, 4, long_rows.scale)
+    torch.cuda.synchronize()
+    assert api.launch_count() - n0 == 2
