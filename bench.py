@@ -230,6 +230,13 @@ class DecodeCase:
         n = 1 if first >= min_total_ms else int(min(max_groups, np.ceil(min_total_ms / max(first, 1e-6))))
         return [first] + [reduce_max(self.time_steps(steps, 0, barrier)) for _ in range(n - 1)]
 
+    def launches_per_step(self):
+        """Kernels the library launches for one step (2: split + combine; 1: the rows are merged on chip)."""
+        n0 = self.api.launch_count()
+        self.step()
+        self.torch.cuda.synchronize()
+        return self.api.launch_count() - n0
+
     def time_split_and_combine(self, steps):
         """Mean durations of the split kernel and of the combine kernel, each timed alone: the library records an
         event before and after the split kernel, a third event follows the call.  The events between the two
@@ -525,12 +532,17 @@ def time_sigma_table(api, W, device, steps):
             case = DecodeCase(api, cfg, device)
             ms = case.time_steps(steps, 20) / steps
             split_ms, combine_ms = case.time_split_and_combine(min(steps, 100))
-            row[name] = {"us_per_step": ms * 1e3, "split_us": split_ms * 1e3, "combine_us": combine_ms * 1e3,
+            kernels = case.launches_per_step()
+            row[name] = {"us_per_step": ms * 1e3, "split_us": split_ms * 1e3,
+                         "combine_us": combine_ms * 1e3 if kernels > 1 else None, "kernels_per_step": kernels,
                          "GB/s": case.bytes / ms / 1e6, "kv_bytes": case.bytes, "rotate": case.rotate}
+            if kernels == 1:
+                row[name]["note"] = "the rows' blocks merge on chip (thread-block clusters): no combine kernel"
             del case
         for key, out in (("us_per_step", "time_reduction_pct"), ("split_us", "split_reduction_pct"),
                          ("combine_us", "combine_reduction_pct")):
-            row[out] = 100.0 * (1.0 - row["sigma"][key] / row["std"][key])
+            a, b = row["sigma"][key], row["std"][key]
+            row[out] = 100.0 * (1.0 - a / b) if a is not None and b is not None else None
         row["bytes_reduction_pct"] = 100.0 * (1.0 - row["sigma"]["kv_bytes"] / row["std"]["kv_bytes"])
         rows.append(row)
     return rows
@@ -546,7 +558,8 @@ def time_context_sweep(api, W, device, steps):
         for name, cfg in (("diffqkv", W.CFG3), ("gqa", W.CFG3.gqa_twin())):
             case = DecodeCase(api, dataclasses.replace(cfg, name=f"{name}_{ctx}", kv_len=ctx), device)
             ms = case.time_steps(steps, 20) / steps
-            row[name] = {"us_per_step": ms * 1e3, "GB/s": case.bytes / ms / 1e6, "rotate": case.rotate}
+            row[name] = {"us_per_step": ms * 1e3, "GB/s": case.bytes / ms / 1e6, "rotate": case.rotate,
+                         "kernels_per_step": case.launches_per_step()}
             del case
         row["speedup"] = row["gqa"]["us_per_step"] / row["diffqkv"]["us_per_step"]
         rows.append(row)
@@ -757,7 +770,8 @@ def run_ours(args):
             for c in (W.CFG2, W.CFG2.gqa_twin(), W.CFG1):
                 cs = DecodeCase(api, c, device, host_inputs=W.make_decode_inputs(c))
                 c_ms = cs.time_steps(so, args.warmup) / so
-                others[c.name] = {"ms_per_step": c_ms, "GB/s": cs.bytes / c_ms / 1e6, "rotate": cs.rotate}
+                others[c.name] = {"ms_per_step": c_ms, "GB/s": cs.bytes / c_ms / 1e6, "rotate": cs.rotate,
+                                  "kernels_per_step": cs.launches_per_step()}
                 del cs
             torch.cuda.empty_cache()
             others["fp32_b4_64k"] = time_fp32_mode(api, W, device, max(5, min(args.steps, 50)))

@@ -113,7 +113,10 @@ size_t diffqkv_decode_workspace_bytes(const diffqkv_shape *shape, int32_t max_se
  *   out        [batch, n_q, d_v]   shape.out_dtype
  *   lse        [batch, n_q] fp32 natural-log log-sum-exp of the scaled scores, or NULL
  *   dev_status one int32 the kernels OR (1 << diffqkv_status) bits into, or NULL; the caller zeroes it
- * Runs the split kernel and then the combine kernel on `stream`.
+ * Runs the split kernel and then the combine kernel on `stream`.  With few, short rows (the blocks that share a
+ * (sequence, head group) row fill at least 0.85 of the SMs as clusters of 2 to 8 and the cache's capacity for them is
+ * small enough that the idle SMs cost less than a second launch) the TMA kernel's blocks of a row form a thread-block
+ * cluster and merge on chip instead: one launch, the workspace is not used.
  */
 diffqkv_status diffqkv_decode(const void *q, const diffqkv_cache *cache, const diffqkv_shape *shape,
                               int32_t num_splits, void *workspace, size_t workspace_bytes, void *out,
