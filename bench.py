@@ -692,6 +692,18 @@ def run_ours(args):
             print(json.dumps({"workload": "cfg4 widths, 4 / 16 / 64 rows",
                               **time_augq_decode(api, W, device, max(1, min(args.steps, 200)))}))
         return
+    if args.workload == "cfg2":  # config 2 and its GQA twin alone (short rows: merged on chip; the command profilers wrap)
+        if rank == 0:
+            res = {"workload": W.CFG2.name}
+            steps = max(1, min(args.steps, 2000))
+            for c in (W.CFG2, W.CFG2.gqa_twin()):
+                cs = DecodeCase(api, c, device, host_inputs=W.make_decode_inputs(c))
+                c_ms = cs.time_steps(steps, args.warmup) / steps
+                res[c.name] = {"ms_per_step": c_ms, "GB/s": cs.bytes / c_ms / 1e6, "kv_bytes": cs.bytes,
+                               "rotate": cs.rotate, "kernels_per_step": cs.launches_per_step()}
+                del cs
+            print(json.dumps(res))
+        return
     if args.workload == "fp32":  # the fp32 mode alone (the command profilers wrap)
         if rank == 0:
             print(json.dumps({"workload": "fp32_b4_64k", **time_fp32_mode(api, W, device, max(1, min(args.steps, 50)))}))
@@ -882,10 +894,10 @@ def main():
     ap.add_argument("--quick", action="store_true", help="headline workload only")
     ap.add_argument("--budget-s", type=float, default=150.0,
                     help="--impl reference: seconds of oracle time the whole run may take (sizes the per-step sample)")
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "topk", "augq_decode", "fp32"],
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "topk", "augq_decode", "fp32", "cfg2"],
                     help="decode = the headline line (default); prefill = only the config 4 timings; "
                          "topk = only selective V fetching on the headline workload; augq_decode = only the projection "
-                         "chain at decode row counts")
+                         "chain at decode row counts; fp32 = only the fp32 mode; cfg2 = only config 2 and its GQA twin")
     ap.add_argument("--tail-reserve", type=int, default=-1,
                     help="tail balance of the TMA decode kernel: -1 automatic (default), 0 off, n tiles per block")
     ap.add_argument("--profile", action="store_true",
