@@ -30,8 +30,19 @@ def _heads(rng):
     return n_q, int(rng.choice(divs)), int(rng.choice(divs))
 
 
+@pytest.mark.parametrize("cluster", [-1, 1])
 @pytest.mark.parametrize("it", range(20))
-def test_random_decode(api, oracle, it):
+def test_random_decode(api, oracle, it, cluster):
+    """cluster = 1 forces the on-chip merge of a row's blocks wherever at least two blocks per row fit on the GPU
+    (left to itself the library takes it for some of these shapes only)."""
+    api.decode_cluster(cluster)
+    try:
+        _random_decode(api, oracle, it)
+    finally:
+        api.decode_cluster(-1)
+
+
+def _random_decode(api, oracle, it):
     rng = _rng(1, it)
     n_q, n_k, n_v = _heads(rng)
     d_qk, d_v = int(rng.choice([64, 128])), int(rng.choice([64, 128]))
