@@ -291,6 +291,31 @@ def diffqkv_decode(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: f
                    out_dtype, stream)
 
 
+def bind_decode(q: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: float, workspace: torch.Tensor,
+                out: torch.Tensor, num_splits: int = 0, lse: Optional[torch.Tensor] = None,
+                dev_status: Optional[torch.Tensor] = None, gqa: bool = False):
+    """diffqkv_decode (or gqa_decode) with its argument structs built once: returns a function of no arguments that
+    makes the library call on the current stream, as a C caller that keeps its diffqkv_shape / diffqkv_cache around
+    does (a decode step of a few microseconds is otherwise bounded by the marshalling here, not by the GPU).  The
+    tensors must stay alive and unmoved while the function is in use."""
+    batch, n_q, d_qk = q.shape
+    shape = make_shape(batch, n_q, n_k, n_v, d_qk, cache.v.shape[-1], q.dtype, out.dtype, scale)
+    cs = cache.c_struct()
+    fn = _lib.gqa_decode if gqa else _lib.diffqkv_decode
+    name = "gqa_decode" if gqa else "diffqkv_decode"
+    args = (_p(q), C.byref(cs), C.byref(shape), int(num_splits), _p(workspace),
+            workspace.numel() * workspace.element_size(), _p(out), _p(lse), _p(dev_status))
+    keep = (shape, cs, q, cache, workspace, out, lse, dev_status)
+
+    def call():
+        st = fn(*args, C.c_void_p(torch.cuda.current_stream().cuda_stream))
+        if st != OK:
+            raise DiffQKVError(st, name)
+        return keep[5]
+
+    return call
+
+
 def diffqkv_decode_host(q_host: torch.Tensor, q_dev: torch.Tensor, cache: KVCache, n_k: int, n_v: int, scale: float,
                         workspace: torch.Tensor, out_dev: torch.Tensor, out_host: torch.Tensor, num_splits: int = 0,
                         lse: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,

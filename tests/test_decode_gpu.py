@@ -597,3 +597,19 @@ def test_cluster_merge_is_chosen_for_short_rows_only(api, oracle, cluster_mode):
     api.diffqkv_decode(q, cache, 2, 4, long_rows.scale)
     torch.cuda.synchronize()
     assert api.launch_count() - n0 == 2
+
+
+def test_bound_call_is_the_same_call(api, fixed_owners):
+    """bind_decode builds the argument structs once; what it launches is the plain call."""
+    inp = W.make_decode_inputs(SMALL)
+    cfg = inp.cfg
+    q, cache = W.to_torch(inp.q, "cuda"), device_cache(api, inp)
+    ref = api.diffqkv_decode(q, cache, cfg.n_k, cfg.n_v, cfg.scale)
+    shape = api.make_shape(cfg.batch, cfg.n_q, cfg.n_k, cfg.n_v, cfg.d_qk, cfg.d_v, q.dtype, q.dtype, cfg.scale)
+    ws = torch.empty(api.diffqkv_decode_workspace_bytes(shape, cache.max_seqlen, 0), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(ref, float("nan"))
+    call = api.bind_decode(q, cache, cfg.n_k, cfg.n_v, cfg.scale, ws, out)
+    for _ in range(3):
+        assert call() is out
+    torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.uint16), ref.view(torch.uint16))
